@@ -1,0 +1,250 @@
+"""fp64 CPU oracle of the TARDIS partially linear FFN forward (arXiv 2501.10054).
+
+TEST INFRASTRUCTURE, NOT PRODUCT CODE.  Only the test-suite, the smoke check and
+the CPU-baseline / reference arm of the benchmark may import this module.  It
+shares no code with the CUDA library and never calls it; the CUDA library never
+calls this.  Everything here is plain numpy in float64, written in the order
+and notation of the paper so it can be checked against the paper by eye.
+
+Notation bridge.  The paper writes row vectors, FFN(x) = sigma(x W1) W2 with
+W1 in R^{d x h}, W2 in R^{h x d}; neuron n is column n of W1 and row n of W2
+(Section 3.1, Section 5.1).  This module uses the nn.Linear storage layout:
+
+    W1[h, d]  row j    = neuron j's input weights   (paper: column j of W1)
+    W2[d, h]  column j = neuron j's output weights  (paper: row j of W2)
+
+so W_f = W2 diag(a) W1 is the transpose of the paper's folded matrix C and
+b_f is the paper's B (with the biases b1, b2 the paper drops for presentation,
+Section 3.1 footnote).  Slope/intercept (a_j, c_j) are the paper's (a, b) of
+the per-neuron linear function on the half-open range [l1, l2) = [lo_j, hi_j)
+(Section 5.1.1).
+
+Pins (tests, CPU only): the worked two-neuron example of Section 4.2, the fold
+example of Section 3.1, the linear-activation identity, the all-flagged = dense
+GELU FFN identity, brute force over every flag subset for d, h <= 16, the
+exact-predictor special case, closed forms of GELU, the packing convention.
+No function in this file is "parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+ACT_GELU_TANH = 0
+ACT_GELU_ERF = 1
+
+_F64 = np.float64
+
+
+def _as64(v):
+    return np.ascontiguousarray(np.asarray(v, dtype=_F64))
+
+
+# --------------------------------------------------------------------------
+# activation
+# --------------------------------------------------------------------------
+def gelu(z, act=ACT_GELU_TANH):
+    """GELU in float64.  The paper only says "GELU" (Section 3.2); both common
+    forms are provided: tanh form 0.5 z (1 + tanh(sqrt(2/pi)(z + 0.044715 z^3)))
+    and the exact form z * Phi(z) with Phi the standard normal CDF."""
+    z = np.asarray(z, dtype=_F64)
+    if act == ACT_GELU_TANH:
+        u = math.sqrt(2.0 / math.pi) * (z + 0.044715 * z * z * z)
+        return 0.5 * z * (1.0 + np.tanh(u))
+    if act == ACT_GELU_ERF:
+        from scipy.special import erf          # library primitive: the error function
+        return 0.5 * z * (1.0 + erf(z / math.sqrt(2.0)))
+    raise ValueError("unknown activation %r" % (act,))
+
+
+# --------------------------------------------------------------------------
+# predictor state format
+# --------------------------------------------------------------------------
+def unpack_codes(codes_u32, d, bits=2):
+    """Expand packed predictor codes to one integer per weight.
+
+    Packed layout: for neuron j, word w of row j holds the codes of input
+    channels k = w*(32/bits) ... , channel order ascending, lowest bits first.
+    Returns uint8 [h, d]."""
+    codes_u32 = np.asarray(codes_u32, dtype=np.uint32)
+    per = 32 // bits
+    h, nw = codes_u32.shape
+    if nw * per != d:
+        raise ValueError("codes row has %d words, expected %d" % (nw, d // per))
+    q = np.empty((h, d), dtype=np.uint8)
+    mask = np.uint32((1 << bits) - 1)
+    for p in range(per):
+        q[:, p::per] = ((codes_u32 >> np.uint32(bits * p)) & mask).astype(np.uint8)
+    return q
+
+
+def predictor_score(x, codes_u32, scale, zero, group, b1=None, bits=2):
+    """Predictor score of Section 5.3: the pre-activation computed from the
+    compressed (quantised) copy of W1 instead of W1 itself.
+
+        zhat[t, j] = b1_j + sum_g s[j,g] * sum_{k in g} (q[j,k] - zp[j,g]) * x[t,k]
+
+    x [n, d]; codes packed uint32 [h, d*bits/32]; scale, zero [h, d/group]."""
+    x = _as64(x)
+    n, d = x.shape
+    q = unpack_codes(codes_u32, d, bits).astype(_F64)
+    h = q.shape[0]
+    scale = _as64(scale)
+    zero = _as64(zero)
+    ng = d // group
+    if scale.shape != (h, ng) or zero.shape != (h, ng):
+        raise ValueError("scale/zero must be [h, d/group]")
+    zhat = np.zeros((n, h), dtype=_F64)
+    for g in range(ng):
+        ks = slice(g * group, (g + 1) * group)
+        centred = q[:, ks] - zero[:, g:g + 1]            # (q - zp), [h, group]
+        zhat += (x[:, ks] @ centred.T) * scale[:, g][None, :]
+    if b1 is not None:
+        zhat += _as64(b1)[None, :]
+    return zhat
+
+
+def flags_from_score(zhat, lo, hi):
+    """A neuron is flagged when its (predicted) pre-activation is outside the
+    half-open linear range [lo, hi) of Section 5.1.1.  Written as the negation
+    of the in-range test so that NaN scores are flagged."""
+    zhat = _as64(zhat)
+    lo = _as64(lo)[None, :]
+    hi = _as64(hi)[None, :]
+    with np.errstate(invalid="ignore"):
+        inside = (lo <= zhat) & (zhat < hi)
+    return ~inside
+
+
+def near_threshold(zhat, lo, hi, band=1e-6):
+    """Neurons whose score lies within `band` of either range end; their flag
+    is excluded from bit-exact comparison and reported instead."""
+    zhat = _as64(zhat)
+    return (np.abs(zhat - _as64(lo)[None, :]) < band) | (np.abs(zhat - _as64(hi)[None, :]) < band)
+
+
+# --------------------------------------------------------------------------
+# offline: constant folding (Section 5.2)
+# --------------------------------------------------------------------------
+def fold(W1, W2, a, c, b1=None, b2=None):
+    """Constant folding.  Per neuron CF gives (a_j * outer(W2[:,j], W1[j,:]),
+    c_j * W2[:,j]); summed over neurons:
+
+        W_f[i,k] = sum_j W2[i,j] a_j W1[j,k]
+        b_f[i]   = sum_j W2[i,j] (a_j b1_j + c_j) + b2_i
+    """
+    W1 = _as64(W1)
+    W2 = _as64(W2)
+    a = _as64(a)
+    c = _as64(c)
+    h, d = W1.shape
+    b1v = np.zeros(h) if b1 is None else _as64(b1)
+    b2v = np.zeros(d) if b2 is None else _as64(b2)
+    Wf = (W2 * a[None, :]) @ W1
+    bf = W2 @ (a * b1v + c) + b2v
+    return Wf, bf
+
+
+def fold_rows(rows, W1, W2, a):
+    """Rows `rows` of W_f only (for sampled checks at sizes where the whole
+    d x d fold is too slow on a CPU)."""
+    W1 = _as64(W1)
+    a = _as64(a)
+    W2r = _as64(np.asarray(W2)[np.asarray(rows)])
+    return (W2r * a[None, :]) @ W1
+
+
+# --------------------------------------------------------------------------
+# online: speculate, then fix (Section 5.4)
+# --------------------------------------------------------------------------
+def speculate(Wf, bf, x):
+    """Speculative approximation: every neuron assumed in range, y0 = W_f x + b_f."""
+    return _as64(x) @ _as64(Wf).T + _as64(bf)[None, :]
+
+
+def fix(y0, x, F, W1, W2, a, c, b1=None, act=ACT_GELU_TANH):
+    """Result fixing.  For every flagged neuron j of token t: recompute the true
+    pre-activation z_j from the original W1 row, take away the linear value that
+    the folded product already contains and add the true activation:
+
+        y[t,:] += W2[:,j] * (GELU(z_j) - a_j z_j - c_j)
+
+    The predictor's flags define the result: a flagged neuron is replaced even
+    if its true z_j is inside the range, an unflagged one keeps the linear value."""
+    x = _as64(x)
+    W1 = _as64(W1)
+    W2 = _as64(W2)
+    a = _as64(a)
+    c = _as64(c)
+    F = np.asarray(F, dtype=bool)
+    y = _as64(y0).copy()
+    for t in range(x.shape[0]):
+        idx = np.nonzero(F[t])[0]
+        if idx.size == 0:
+            continue
+        z = W1[idx] @ x[t]
+        if b1 is not None:
+            z = z + _as64(b1)[idx]
+        delta = gelu(z, act) - a[idx] * z - c[idx]
+        y[t] += W2[:, idx] @ delta
+    return y
+
+
+def tardis_ffn(x, W1, W2, a, c, lo, hi, codes_u32, scale, zero, group,
+               b1=None, b2=None, act=ACT_GELU_TANH, bits=2, folded=None):
+    """The whole path in the paper's order: fold (offline), predictor score,
+    flag, speculative folded product, result fixing.  Returns (y, F, zhat).
+    `folded` may carry a previously computed (W_f, b_f)."""
+    if folded is None:
+        folded = fold(W1, W2, a, c, b1, b2)
+    Wf, bf = folded
+    zhat = predictor_score(x, codes_u32, scale, zero, group, b1, bits)
+    F = flags_from_score(zhat, lo, hi)
+    y0 = speculate(Wf, bf, x)
+    y = fix(y0, x, F, W1, W2, a, c, b1, act)
+    return y, F, zhat
+
+
+# --------------------------------------------------------------------------
+# definitions the path is checked against
+# --------------------------------------------------------------------------
+def dense_ffn(x, W1, W2, b1=None, b2=None, act=ACT_GELU_TANH):
+    """The original FFN, W2 GELU(W1 x + b1) + b2 (Section 3.1)."""
+    x = _as64(x)
+    z = x @ _as64(W1).T
+    if b1 is not None:
+        z = z + _as64(b1)[None, :]
+    y = gelu(z, act) @ _as64(W2).T
+    if b2 is not None:
+        y = y + _as64(b2)[None, :]
+    return y
+
+
+def direct_partially_linear(x, F, W1, W2, a, c, b1=None, b2=None, act=ACT_GELU_TANH):
+    """The partially linear FFN with no folding at all: neuron j contributes
+    W2[:,j] * phi_j(z_j), phi_j = GELU when flagged, a_j z + c_j otherwise
+    (Section 5.1.1 with the predictor's flags standing in for the range test).
+    Costs 4 d h per token and needs no d x d matrix, so it also serves as the
+    per-token check at full problem sizes."""
+    x = _as64(x)
+    z = x @ _as64(W1).T
+    if b1 is not None:
+        z = z + _as64(b1)[None, :]
+    F = np.asarray(F, dtype=bool)
+    phi = np.where(F, gelu(z, act), _as64(a)[None, :] * z + _as64(c)[None, :])
+    y = phi @ _as64(W2).T
+    if b2 is not None:
+        y = y + _as64(b2)[None, :]
+    return y
+
+
+def rel_error(y, y_ref):
+    """Per-element error |y - y_ref| / max(|y_ref|, rms(y_ref[t,:])); the maximum
+    of this over all elements is the "max relative error" of the parity gate."""
+    y = _as64(y)
+    y_ref = _as64(y_ref)
+    rms = np.sqrt(np.mean(y_ref * y_ref, axis=-1, keepdims=True))
+    den = np.maximum(np.abs(y_ref), rms)
+    den = np.where(den > 0, den, 1.0)
+    return np.abs(y - y_ref) / den

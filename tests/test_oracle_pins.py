@@ -1,0 +1,303 @@
+"""Pins of the fp64 oracle against what the paper and the mathematics fix.
+CPU only.  Each test states which plausible mistake it is meant to catch."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import tardis_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def read_golden(name):
+    out = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, *v = line.split()
+            out[k] = np.array([float(t) for t in v])
+    return out
+
+
+def Phi(z):
+    """Standard normal CDF through erfc (independent of the oracle's erf call)."""
+    return 0.5 * math.erfc(-z / math.sqrt(2.0))
+
+
+# ------------------------------------------------------------------ GELU
+def test_gelu_closed_forms():
+    # exact form: GELU(z) = z Phi(z); GELU(-2) = -2 Phi(-2) = -0.0455002639...
+    assert O.gelu(-2.0, O.ACT_GELU_ERF) == pytest.approx(-2.0 * Phi(-2.0), abs=1e-15)
+    assert -2.0 * Phi(-2.0) == pytest.approx(-0.04550026389635842, abs=1e-12)
+    for act in (O.ACT_GELU_TANH, O.ACT_GELU_ERF):
+        assert O.gelu(0.0, act) == 0.0
+        z = np.linspace(-6, 6, 49)
+        # odd-part identity GELU(z) - GELU(-z) = z (Phi(z) + Phi(-z) = 1; tanh is odd)
+        np.testing.assert_allclose(O.gelu(z, act) - O.gelu(-z, act), z, atol=1e-14)
+        assert O.gelu(30.0, act) == pytest.approx(30.0, abs=1e-12)
+        assert abs(float(O.gelu(-30.0, act))) < 1e-12
+    # the tanh form is the published approximation of the exact one: they agree to < 1e-3
+    z = np.linspace(-8, 8, 4001)
+    assert np.max(np.abs(O.gelu(z, O.ACT_GELU_TANH) - O.gelu(z, O.ACT_GELU_ERF))) < 1e-3
+    # tanh-form value at -2 quoted to six digits (-0.045402)
+    assert float(O.gelu(-2.0, O.ACT_GELU_TANH)) == pytest.approx(-0.0454023, abs=2e-7)
+    # derivative at 0 is 1/2 for both forms (catches a dropped 0.5 or a wrong inner constant sign)
+    for act in (O.ACT_GELU_TANH, O.ACT_GELU_ERF):
+        e = 1e-6
+        assert (float(O.gelu(e, act)) - float(O.gelu(-e, act))) / (2 * e) == pytest.approx(0.5, abs=1e-9)
+    # second-order coefficient of the tanh form: GELU(z) ~ z/2 + z^2 sqrt(2/pi)/2 near 0
+    e = 1e-3
+    curv = (float(O.gelu(e)) + float(O.gelu(-e))) / (e * e)
+    assert curv == pytest.approx(math.sqrt(2 / math.pi), rel=1e-5)
+
+
+# ------------------------------------------------------------------ worked example (Section 4.2)
+def _worked():
+    g = read_golden("worked_example.txt")
+    # nn.Linear layout: W1[h,d] row j = neuron j (paper's column j); W2[d,h] column j = paper's row j
+    W1 = np.stack([g["W1_col1"], g["W1_col2"]])
+    W2 = np.stack([g["W2_row1"], g["W2_row2"]]).T
+    a = np.array([g["slope_intercept1"][0], g["slope_intercept2"][0]])
+    c = np.array([g["slope_intercept1"][1], g["slope_intercept2"][1]])
+    lo = np.array([g["range1"][0], g["range2"][0]])
+    hi = np.array([g["range1"][1], g["range2"][1]])
+    return g, W1, W2, a, c, lo, hi
+
+
+def test_worked_example_fold_and_speculate():
+    g, W1, W2, a, c, lo, hi = _worked()
+    Wf, bf = O.fold(W1, W2, a, c)
+    # paper convention C = W_f^T; values derived from the printed numbers
+    np.testing.assert_allclose(Wf.T, [[-0.65, 0.1], [0.45, 0.2]], atol=1e-15)
+    np.testing.assert_allclose(bf, [0.1, 0.2], atol=1e-15)
+    y0 = O.speculate(Wf, bf, g["x"][None, :])
+    np.testing.assert_allclose(y0[0], g["xC_plus_B"], atol=1e-15)   # printed: (0.3, -0.1)
+
+
+def test_worked_example_flags_and_fix():
+    g, W1, W2, a, c, lo, hi = _worked()
+    x = g["x"][None, :]
+    z = x @ W1.T
+    np.testing.assert_allclose(z[0], g["z"][1:], atol=0)
+    F = O.flags_from_score(z, lo, hi)
+    assert F[0].tolist() == [bool(v) for v in g["flagged"]]          # neuron one flagged, two not
+    Wf, bf = O.fold(W1, W2, a, c)
+    y = O.fix(O.speculate(Wf, bf, x), x, F, W1, W2, a, c, act=O.ACT_GELU_ERF)
+    # printed steps: (0.3,-0.1) - (0.4,0) + GELU(-2) (-1,0)
+    gelu_m2 = -2.0 * Phi(-2.0)
+    expect = g["xC_plus_B"] - g["subtracted"] + gelu_m2 * g["W2_row1"]
+    np.testing.assert_allclose(y[0], expect, atol=1e-15)
+    np.testing.assert_allclose(y[0], [-0.1 + 0.04550026389635842, -0.1], atol=1e-12)
+    # the subtracted term itself: (a1 z1 + c1) * W2 row 1 = (0.4, 0)
+    np.testing.assert_allclose((a[0] * z[0, 0] + c[0]) * W2[:, 0], g["subtracted"], atol=1e-15)
+
+
+def test_fold_example_section_3_1():
+    g = read_golden("fold_example.txt")
+    W1 = np.stack([g["W1_col1"], g["W1_col2"]])
+    W2 = np.stack([g["W2_row1"], g["W2_row2"]]).T
+    prod = np.stack([g["W1W2_row1"], g["W1W2_row2"]])            # paper's W1 W2
+    for slope in (1.0, 0.3, -2.0):
+        Wf, bf = O.fold(W1, W2, np.full(2, slope), np.zeros(2))
+        np.testing.assert_allclose(Wf.T, slope * prod, atol=1e-15)
+        np.testing.assert_allclose(bf, 0, atol=0)
+        x = np.array([[0.7, -1.3]])
+        np.testing.assert_allclose(O.speculate(Wf, bf, x)[0],
+                                   [slope * (-2 * 0.7 + 3 * -1.3), slope * (0.7 + 2 * -1.3)], atol=1e-15)
+    d, h = 7, 28
+    assert 1 - d * d / (2 * d * h) == g["param_reduction_h4d"][0]
+
+
+# ------------------------------------------------------------------ invariants on random small problems
+def _random_problem(rng, d, h, n, group=None, bias=True):
+    W1 = rng.normal(size=(h, d))
+    W2 = rng.normal(size=(d, h))
+    b1 = rng.normal(size=h) if bias else None
+    b2 = rng.normal(size=d) if bias else None
+    a = rng.uniform(-0.2, 1.2, size=h)
+    c = rng.normal(size=h) * 0.1
+    x = rng.normal(size=(n, d))
+    return W1, W2, b1, b2, a, c, x
+
+
+def _loops_partially_linear(x, F, W1, W2, b1, b2, a, c, act):
+    """The definition as scalar Python loops (brute force; no numpy contraction)."""
+    n, d, h = len(x), len(x[0]), len(W1)
+    y = [[0.0] * d for _ in range(n)]
+    for t in range(n):
+        for j in range(h):
+            z = sum(W1[j][k] * x[t][k] for k in range(d)) + (b1[j] if b1 is not None else 0.0)
+            if F[t][j]:
+                u = math.sqrt(2.0 / math.pi) * (z + 0.044715 * z ** 3)
+                phi = 0.5 * z * (1.0 + math.tanh(u)) if act == O.ACT_GELU_TANH else z * Phi(z)
+            else:
+                phi = a[j] * z + c[j]
+            for i in range(d):
+                y[t][i] += W2[i][j] * phi
+        if b2 is not None:
+            for i in range(d):
+                y[t][i] += b2[i]
+    return np.array(y)
+
+
+@pytest.mark.parametrize("bias", [True, False])
+def test_linear_activation_identity(bias):
+    """With every activation replaced by its neuron's linear map the unfolded FFN equals
+    W_f x + b_f (catches a transposed operand, a dropped a_j b1_j / c_j / b2 term)."""
+    rng = np.random.default_rng(1)
+    W1, W2, b1, b2, a, c, x = _random_problem(rng, 5, 11, 4, bias=bias)
+    Wf, bf = O.fold(W1, W2, a, c, b1, b2)
+    none = np.zeros((4, 11), dtype=bool)
+    ref = _loops_partially_linear(x.tolist(), none, W1.tolist(), W2.tolist(),
+                                  None if b1 is None else b1.tolist(), None if b2 is None else b2.tolist(),
+                                  a.tolist(), c.tolist(), O.ACT_GELU_TANH)
+    np.testing.assert_allclose(O.speculate(Wf, bf, x), ref, rtol=0, atol=1e-12)
+    # no neuron flagged: fixing changes nothing
+    np.testing.assert_array_equal(O.fix(O.speculate(Wf, bf, x), x, none, W1, W2, a, c, b1), O.speculate(Wf, bf, x))
+
+
+@pytest.mark.parametrize("act", [O.ACT_GELU_TANH, O.ACT_GELU_ERF])
+def test_all_flagged_equals_dense_ffn(act):
+    rng = np.random.default_rng(2)
+    W1, W2, b1, b2, a, c, x = _random_problem(rng, 6, 13, 5)
+    Wf, bf = O.fold(W1, W2, a, c, b1, b2)
+    allf = np.ones((5, 13), dtype=bool)
+    y = O.fix(O.speculate(Wf, bf, x), x, allf, W1, W2, a, c, b1, act)
+    ref = _loops_partially_linear(x.tolist(), allf, W1.tolist(), W2.tolist(), b1.tolist(), b2.tolist(),
+                                  a.tolist(), c.tolist(), act)
+    np.testing.assert_allclose(y, ref, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(O.dense_ffn(x, W1, W2, b1, b2, act), ref, rtol=0, atol=1e-12)
+
+
+def test_brute_force_every_flag_subset():
+    """d = 3, h = 8: for each of the 2^8 flag subsets fold + speculate + fix equals the scalar-loop
+    definition, and so does the unfolded numpy definition."""
+    rng = np.random.default_rng(3)
+    d, h = 3, 8
+    W1, W2, b1, b2, a, c, x = _random_problem(rng, d, h, 1)
+    Wf, bf = O.fold(W1, W2, a, c, b1, b2)
+    y0 = O.speculate(Wf, bf, x)
+    for bits in itertools.product([False, True], repeat=h):
+        F = np.array([bits])
+        ref = _loops_partially_linear(x.tolist(), F, W1.tolist(), W2.tolist(), b1.tolist(), b2.tolist(),
+                                      a.tolist(), c.tolist(), O.ACT_GELU_TANH)
+        np.testing.assert_allclose(O.fix(y0, x, F, W1, W2, a, c, b1), ref, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(O.direct_partially_linear(x, F, W1, W2, a, c, b1, b2), ref, rtol=0, atol=1e-12)
+
+
+def test_brute_force_d16_h16_random_subsets():
+    rng = np.random.default_rng(4)
+    d = h = 16
+    W1, W2, b1, b2, a, c, x = _random_problem(rng, d, h, 3)
+    Wf, bf = O.fold(W1, W2, a, c, b1, b2)
+    for _ in range(40):
+        F = rng.random((3, h)) < rng.random()
+        ref = _loops_partially_linear(x.tolist(), F, W1.tolist(), W2.tolist(), b1.tolist(), b2.tolist(),
+                                      a.tolist(), c.tolist(), O.ACT_GELU_TANH)
+        np.testing.assert_allclose(O.fix(O.speculate(Wf, bf, x), x, F, W1, W2, a, c, b1), ref, rtol=0, atol=1e-11)
+
+
+def test_fold_rows_matches_fold():
+    rng = np.random.default_rng(5)
+    W1, W2, b1, b2, a, c, x = _random_problem(rng, 9, 20, 1)
+    Wf, _ = O.fold(W1, W2, a, c, b1, b2)
+    np.testing.assert_allclose(O.fold_rows([7, 0, 3], W1, W2, a), Wf[[7, 0, 3]], atol=1e-13)
+    # element-wise definition W_f[i,k] = sum_j W2[i,j] a_j W1[j,k]
+    i, k = 4, 2
+    assert Wf[i, k] == pytest.approx(sum(W2[i, j] * a[j] * W1[j, k] for j in range(20)), abs=1e-13)
+
+
+# ------------------------------------------------------------------ predictor
+def test_unpack_convention():
+    # channel 0 in the two lowest bits, channel 15 in the two highest
+    word = sum(v << (2 * p) for p, v in enumerate([1, 2, 3, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 3]))
+    q = O.unpack_codes(np.array([[word, 0b11]], dtype=np.uint32), 32)
+    assert q[0, :4].tolist() == [1, 2, 3, 0] and q[0, 15] == 3 and q[0, 16] == 3 and q[0, 17:].sum() == 0
+
+
+def _pack(q):
+    h, d = q.shape
+    w = np.zeros((h, d // 16), dtype=np.uint64)
+    for p in range(16):
+        w |= q[:, p::16].astype(np.uint64) << np.uint64(2 * p)
+    return w.astype(np.uint32)
+
+
+def test_predictor_hand_case():
+    # 2 neurons, d = 16 = one group.  neuron 0: codes k%4, s = 0.5, zp = 1; neuron 1: all 3, s = 2, zp = 0
+    q = np.stack([np.arange(16) % 4, np.full(16, 3)]).astype(np.uint8)
+    x = np.arange(16, dtype=np.float64)[None, :] - 4.0
+    s = np.array([[0.5], [2.0]])
+    zp = np.array([[1], [0]], dtype=np.uint8)
+    b1 = np.array([0.25, -1.0])
+    zhat = O.predictor_score(x, _pack(q), s, zp, 16, b1)
+    e0 = 0.25 + 0.5 * sum((k % 4 - 1) * (k - 4.0) for k in range(16))
+    e1 = -1.0 + 2.0 * 3 * sum(k - 4.0 for k in range(16))
+    np.testing.assert_allclose(zhat[0], [e0, e1], atol=1e-13)
+
+
+def test_predictor_exact_special_case_is_a_gemv():
+    """With unit scales, zero zero-points and integer weights in 0..3 the predictor's
+    "compressed W1" is W1 itself, so the score is the textbook GEMV W1 x + b1."""
+    rng = np.random.default_rng(6)
+    h, d, G = 12, 64, 16
+    q = rng.integers(0, 4, size=(h, d)).astype(np.uint8)
+    x = rng.normal(size=(5, d))
+    b1 = rng.normal(size=h)
+    zhat = O.predictor_score(x, _pack(q), np.ones((h, d // G)), np.zeros((h, d // G), dtype=np.uint8), G, b1)
+    ref = np.array([[sum(float(q[j, k]) * x[t, k] for k in range(d)) + b1[j] for j in range(h)] for t in range(5)])
+    np.testing.assert_allclose(zhat, ref, atol=1e-12)
+
+
+def test_predictor_groups_scales_zero_points_and_linearity():
+    rng = np.random.default_rng(7)
+    h, d, G = 6, 96, 32
+    q = rng.integers(0, 4, size=(h, d)).astype(np.uint8)
+    s = rng.uniform(0.01, 0.05, size=(h, d // G))
+    zp = rng.integers(0, 4, size=(h, d // G)).astype(np.uint8)
+    x = rng.normal(size=(3, d))
+    zhat = O.predictor_score(x, _pack(q), s, zp, G)
+    ref = np.zeros((3, h))
+    for t in range(3):
+        for j in range(h):
+            for k in range(d):
+                ref[t, j] += s[j, k // G] * (float(q[j, k]) - float(zp[j, k // G])) * x[t, k]
+    np.testing.assert_allclose(zhat, ref, atol=1e-12)
+    z2 = O.predictor_score(2.5 * x[:1] - x[1:2], _pack(q), s, zp, G)
+    np.testing.assert_allclose(z2, 2.5 * zhat[:1] - zhat[1:2], atol=1e-12)
+
+
+def test_flag_rule_half_open_and_nan():
+    lo = np.array([-1.0, -1.0, -1.0, -1.0, -1.0])
+    hi = np.array([2.0, 2.0, 2.0, 2.0, 2.0])
+    z = np.array([[-1.0, 2.0, 0.0, np.nan, np.nextafter(2.0, 0.0)]])
+    assert O.flags_from_score(z, lo, hi)[0].tolist() == [False, True, False, True, False]
+    z = np.array([[-1.0 - 5e-7, 2.0 + 2e-6, 0.0, 1.0, -1.0 + 2e-6]])
+    assert O.near_threshold(z, lo, hi)[0].tolist() == [True, False, False, False, False]
+
+
+def test_full_path_composition():
+    """tardis_ffn = the five steps in order; its output equals the unfolded definition under its own flags."""
+    rng = np.random.default_rng(8)
+    h, d, G = 32, 32, 16
+    W1, W2, b1, b2, a, c, x = _random_problem(rng, d, h, 6)
+    q = rng.integers(0, 4, size=(h, d)).astype(np.uint8)
+    s = rng.uniform(0.3, 0.9, size=(h, d // G))
+    zp = rng.integers(0, 4, size=(h, d // G)).astype(np.uint8)
+    lo = rng.uniform(-6, -1, size=h)
+    hi = rng.uniform(1, 6, size=h)
+    y, F, zhat = O.tardis_ffn(x, W1, W2, a, c, lo, hi, _pack(q), s, zp, G, b1, b2)
+    assert 0 < F.mean() < 1
+    np.testing.assert_array_equal(F, ~((lo <= zhat) & (zhat < hi)))
+    np.testing.assert_allclose(y, O.direct_partially_linear(x, F, W1, W2, a, c, b1, b2), atol=1e-11)
+
+
+def test_rel_error_metric():
+    y_ref = np.array([[3.0, 4.0, 0.0, 0.0]])            # rms = 2.5
+    y = y_ref + np.array([[0.3, 0.0, 0.25, 0.0]])
+    np.testing.assert_allclose(O.rel_error(y, y_ref)[0], [0.1, 0.0, 0.1, 0.0])
