@@ -1,0 +1,157 @@
+/*
+ * libtardis — C ABI of the partially linear FFN forward (TARDIS, arXiv 2501.10054)
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The paper's system has an offline part that turns an FFN (weights W1, W2, a
+ * per-neuron linear range and linear fit, a compressed copy of W1 used as a
+ * predictor) into a constant-folded matrix (Section 5.2, Section 5.3), and an
+ * online part that maps an FFN input to the FFN output by speculative
+ * approximation and result fixing (Section 5.4).  tardis_fold is the offline
+ * part, tardis_ffn_forward the online part, tardis_stats the paper's
+ * memory-footprint accounting (Section 5.4, "Memory Footprint") plus run
+ * counters.
+ *
+ * Notation.  The paper writes row vectors, FFN(x) = sigma(x W1) W2 with neuron n
+ * = column n of W1 and row n of W2.  This interface takes the nn.Linear storage
+ * layout: W1[d_ff, d_model] (row j = neuron j) and W2[d_model, d_ff] (column j
+ * = neuron j); W_f = W2 diag(a) W1 is then the transpose of the paper's C and
+ * b_f = W2 (a .* b1 + c) + b2 is the paper's B.  (a_j, c_j) are the paper's
+ * slope and intercept, [lo_j, hi_j) its half-open range [l1, l2) (Section 5.1.1).
+ *
+ * All pointers named "device" are CUDA device pointers of the current device;
+ * no argument is a host array unless it says so.  No function throws, aborts
+ * or prints; every failure is a status code.  A handle is not thread-safe;
+ * distinct handles are independent.
+ */
+#ifndef TARDIS_H_
+#define TARDIS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tardis_handle_s* tardis_handle_t;   /* opaque; owns device memory */
+typedef void* tardis_stream_t;                      /* a cudaStream_t (0 = default stream) */
+
+typedef enum {
+  TARDIS_OK = 0,
+  TARDIS_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, negative size, bad enum */
+  TARDIS_ERR_UNSUPPORTED = 2,   /* valid request this build has no kernel for (see tardis_fold) */
+  TARDIS_ERR_ALLOC = 3,         /* device allocation failed */
+  TARDIS_ERR_CUDA = 4,          /* a CUDA call failed; text via tardis_last_error */
+  TARDIS_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out */
+  TARDIS_ERR_CORRUPT = 6        /* handle magic / guard words damaged */
+} tardis_status_t;
+
+typedef enum { TARDIS_F32 = 0, TARDIS_BF16 = 1 } tardis_dtype_t;
+typedef enum { TARDIS_ACT_GELU_TANH = 0, TARDIS_ACT_GELU_ERF = 1 } tardis_act_t;
+
+/* Inputs of the offline fold.  Every array is read on `stream` during
+ * tardis_fold and copied or transformed into handle-owned memory; once that
+ * stream has drained the caller may free all of them. */
+typedef struct {
+  int32_t d_model;            /* d; multiple of 8 and of pred_group                       */
+  int32_t d_ff;               /* h; multiple of 32                                        */
+  int32_t dtype;              /* tardis_dtype_t: type of W1, W2, pred_scale, x and y      */
+  int32_t act;                /* tardis_act_t                                             */
+  const void* W1;             /* device [d_ff, d_model] row-major; row j = neuron j       */
+  const void* W2;             /* device [d_model, d_ff] row-major; column j = neuron j    */
+  const float* b1;            /* device [d_ff]    or NULL (= 0)                           */
+  const float* b2;            /* device [d_model] or NULL (= 0)                           */
+  const float* lo;            /* device [d_ff]; neuron j is in range iff lo <= z < hi     */
+  const float* hi;            /* device [d_ff]                                            */
+  const float* a;             /* device [d_ff]; linear fit a*z + c on the range           */
+  const float* c;             /* device [d_ff]                                            */
+  int32_t pred_bits;          /* 2                                                        */
+  int32_t pred_group;         /* G: channels per quantisation group; multiple of 16       */
+  const uint32_t* pred_codes; /* device [d_ff, d_model*pred_bits/32]; channel k of row j in
+                                 word k/16, bits 2*(k%16) .. 2*(k%16)+1                   */
+  const void* pred_scale;     /* device [d_ff, d_model/G], type `dtype`                   */
+  const uint8_t* pred_zero;   /* device [d_ff, d_model/G], integer zero-point 0..3        */
+  uint32_t flags;             /* reserved, 0                                              */
+} tardis_fold_desc_t;
+
+/* Counters and sizes.  Byte counts are the resident state of the handle,
+ * following the paper's footprint components: folded matrix + bias, predictor,
+ * original weights kept for fixing (here: all of W1 and W2^T, any neuron can
+ * be flagged), per-neuron tables, scratch. */
+typedef struct {
+  uint64_t calls;               /* tardis_ffn_forward calls that launched work             */
+  uint64_t tokens;              /* tokens processed                                        */
+  uint64_t flagged_total;       /* sum over tokens of flagged neurons                      */
+  uint64_t flagged_max;         /* largest flagged count of a single token                 */
+  uint64_t last_path;           /* 0 none, 1 generic, 2 fused decode, 3 batched/prefill    */
+  uint64_t bytes_folded;        /* W_f and b_f                                             */
+  uint64_t bytes_predictor;     /* codes + scales + zero-points as stored                  */
+  uint64_t bytes_tables;        /* lo, hi, a, c, b1                                        */
+  uint64_t bytes_w1;
+  uint64_t bytes_w2t;
+  uint64_t bytes_scratch;
+  uint64_t device_error;        /* sticky device-side error word, 0 = none                 */
+  uint64_t exact_rechecks;      /* predictor scores re-evaluated by the exact slow path    */
+} tardis_stats_t;
+
+/* Offline part (Section 5.2 constant folding, Section 5.3 predictor set-up).
+ * Computes W_f = W2 diag(a) W1 and b_f = W2 (a .* b1 + c) + b2 with accumulation
+ * in at least fp32 and one rounding to `dtype`, stores W2 transposed, keeps a
+ * copy of W1 and of the predictor.  Asynchronous on `stream` after the device
+ * allocations; *out is valid on return with TARDIS_OK.
+ * Errors: INVALID_ARG (NULL desc/out/required array, pointer not 16-byte
+ * aligned, d_model % 8, d_model % pred_group, pred_group % 16, d_ff % 32,
+ * non-positive sizes, unknown enum), UNSUPPORTED (pred_bits != 2), ALLOC, CUDA. */
+tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stream,
+                            tardis_handle_t* out);
+
+/* Online part (Section 5.4): y[t,:] = W_f x[t,:] + b_f
+ *      + sum over neurons j flagged for token t of W2[:,j] (GELU(z_j) - a_j z_j - c_j),
+ * z_j = W1[j,:] x[t,:] + b1_j recomputed from the original row; neuron j is
+ * flagged for token t when the predictor score
+ *      zhat = b1_j + sum_g scale[j,g] sum_{k in g} (code[j,k] - zero[j,g]) x[t,k]
+ * is not in [lo_j, hi_j) (NaN counts as outside).
+ * x, y: device [n_tokens, d_model] row-major in the handle's dtype, 16-byte
+ * aligned, not overlapping; y is fully overwritten.  Asynchronous on `stream`,
+ * allocates nothing, does not synchronise.  n_tokens == 0 returns TARDIS_OK
+ * without launching.  The kernel path depends on n_tokens and the handle only.
+ * Calls on one handle must be stream-ordered with respect to each other (they
+ * share the handle's scratch).
+ * Errors: INVALID_ARG (NULL/destroyed handle, NULL or misaligned x/y,
+ * n_tokens < 0), CUDA. */
+tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* y,
+                                   int64_t n_tokens, tardis_stream_t stream);
+
+/* Synchronises the stream of the handle's most recent call, then fills *out
+ * (host memory).  Returns TIMEOUT / CORRUPT when the device error word says so. */
+tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out);
+
+/* Debug capture for parity checks: when set, every later forward call also
+ * writes, for its tokens, the flag bitmap (device uint32 [n_tokens, d_ff/32],
+ * bit j%32 of word j/32 = neuron j flagged) and/or the predictor scores as the
+ * kernel decided on them (device double [n_tokens, d_ff]).  Either may be NULL;
+ * both NULL switches capture off.  The buffers must cover the largest n_tokens
+ * passed while capture is on. */
+tardis_status_t tardis_set_debug_capture(tardis_handle_t handle, uint32_t* flag_bitmap,
+                                         double* scores);
+
+/* Copies the folded state out for inspection: Wf device [d_model, d_model]
+ * row-major in the handle's dtype (row i = output channel i, i.e. W_f itself,
+ * the transpose of the paper's C), bf device float [d_model].  Either may be NULL. */
+tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf,
+                                     tardis_stream_t stream);
+
+/* Chooses the kernel path: 0 = automatic (default), 1 = always the generic
+ * kernels.  For testing one path against the other. */
+tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
+
+/* Frees everything the handle owns (synchronises the device first). */
+tardis_status_t tardis_destroy(tardis_handle_t handle);
+
+const char* tardis_status_string(tardis_status_t status);
+/* Text of the most recent CUDA error seen by this thread in the library ("" if none). */
+const char* tardis_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TARDIS_H_ */

@@ -1,0 +1,163 @@
+"""Python binding of libtardis (the C ABI in include/tardis.h): argument marshalling only.
+
+Every step of the partially linear FFN forward (TARDIS, arXiv 2501.10054: constant folding,
+predictor, speculative folded product, result fixing) runs inside the CUDA library; this
+module turns torch tensors into device pointers and status codes into exceptions.  There is
+no CPU fallback: importing works anywhere, but any call needs libtardis.so and a CUDA device.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtardis.so")
+
+TARDIS_OK = 0
+TARDIS_F32, TARDIS_BF16 = 0, 1
+TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF = 0, 1
+
+EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_stats", "tardis_set_debug_capture",
+           "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_status_string",
+           "tardis_last_error"]
+
+
+class TardisError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(what)
+
+
+class FoldDesc(ctypes.Structure):
+    _fields_ = [("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("act", ctypes.c_int32), ("W1", ctypes.c_void_p), ("W2", ctypes.c_void_p),
+                ("b1", ctypes.c_void_p), ("b2", ctypes.c_void_p), ("lo", ctypes.c_void_p),
+                ("hi", ctypes.c_void_p), ("a", ctypes.c_void_p), ("c", ctypes.c_void_p),
+                ("pred_bits", ctypes.c_int32), ("pred_group", ctypes.c_int32),
+                ("pred_codes", ctypes.c_void_p), ("pred_scale", ctypes.c_void_p),
+                ("pred_zero", ctypes.c_void_p), ("flags", ctypes.c_uint32)]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint64) for n in
+                ("calls", "tokens", "flagged_total", "flagged_max", "last_path", "bytes_folded",
+                 "bytes_predictor", "bytes_tables", "bytes_w1", "bytes_w2t", "bytes_scratch",
+                 "device_error", "exact_rechecks")]
+
+    def as_dict(self):
+        return {n: int(getattr(self, n)) for n, _ in self._fields_}
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Loads libtardis.so (built in-tree by paper_2501_10054_b200.build).  Fails loudly if absent."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise TardisError(-1, "libtardis.so not found at %s: run `python -m paper_2501_10054_b200.build` "
+                              "(there is no CPU fallback)" % p)
+    lib = ctypes.CDLL(p)
+    vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
+    lib.tardis_fold.argtypes = [ctypes.POINTER(FoldDesc), vp, ctypes.POINTER(vp)]
+    lib.tardis_ffn_forward.argtypes = [vp, vp, vp, i64, vp]
+    lib.tardis_stats.argtypes = [vp, ctypes.POINTER(Stats)]
+    lib.tardis_set_debug_capture.argtypes = [vp, vp, vp]
+    lib.tardis_export_folded.argtypes = [vp, vp, vp, vp]
+    lib.tardis_set_path.argtypes = [vp, i32]
+    lib.tardis_destroy.argtypes = [vp]
+    for name in EXPORTS[:7]:
+        getattr(lib, name).restype = ctypes.c_int
+    lib.tardis_status_string.argtypes = [ctypes.c_int]
+    lib.tardis_status_string.restype = ctypes.c_char_p
+    lib.tardis_last_error.argtypes = []
+    lib.tardis_last_error.restype = ctypes.c_char_p
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _check(status: int, what: str):
+    if status != TARDIS_OK:
+        lib = load_library()
+        msg = lib.tardis_status_string(status).decode()
+        detail = lib.tardis_last_error().decode()
+        raise TardisError(status, "%s: %s%s" % (what, msg, (" [" + detail + "]") if detail and status == 4 else ""))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise TardisError(1, "tensors must be contiguous CUDA tensors")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return TARDIS_F32
+    if dt == torch.bfloat16:
+        return TARDIS_BF16
+    raise TardisError(1, "dtype must be float32 or bfloat16")
+
+
+def tardis_fold(W1, W2, lo, hi, a, c, pred_codes, pred_scale, pred_zero, pred_group, b1=None, b2=None,
+                act=TARDIS_ACT_GELU_TANH, pred_bits=2, stream=None) -> int:
+    """tardis_fold of the C ABI.  Returns the opaque handle (an integer)."""
+    lib = load_library()
+    h, d = W1.shape
+    desc = FoldDesc(d, h, _dtype_code(W1.dtype), act, _ptr(W1), _ptr(W2), _ptr(b1), _ptr(b2), _ptr(lo), _ptr(hi),
+                    _ptr(a), _ptr(c), pred_bits, pred_group, _ptr(pred_codes), _ptr(pred_scale), _ptr(pred_zero), 0)
+    out = ctypes.c_void_p()
+    _check(lib.tardis_fold(ctypes.byref(desc), _stream(stream), ctypes.byref(out)), "tardis_fold")
+    return out.value
+
+
+def tardis_ffn_forward(handle: int, x: torch.Tensor, y: torch.Tensor, n_tokens: Optional[int] = None, stream=None):
+    lib = load_library()
+    n = x.shape[0] if n_tokens is None else n_tokens
+    _check(lib.tardis_ffn_forward(handle, _ptr(x), _ptr(y), n, _stream(stream)), "tardis_ffn_forward")
+    return y
+
+
+def tardis_stats(handle: int) -> dict:
+    lib = load_library()
+    st = Stats()
+    _check(lib.tardis_stats(handle, ctypes.byref(st)), "tardis_stats")
+    return st.as_dict()
+
+
+def tardis_set_debug_capture(handle: int, flag_bitmap: Optional[torch.Tensor], scores: Optional[torch.Tensor]):
+    _check(load_library().tardis_set_debug_capture(handle, _ptr(flag_bitmap), _ptr(scores)), "tardis_set_debug_capture")
+
+
+def tardis_export_folded(handle: int, Wf: Optional[torch.Tensor], bf: Optional[torch.Tensor], stream=None):
+    _check(load_library().tardis_export_folded(handle, _ptr(Wf), _ptr(bf), _stream(stream)), "tardis_export_folded")
+
+
+def tardis_set_path(handle: int, path: int):
+    _check(load_library().tardis_set_path(handle, path), "tardis_set_path")
+
+
+def tardis_destroy(handle: int):
+    _check(load_library().tardis_destroy(handle), "tardis_destroy")
+
+
+def fold_layer(layer, stream=None) -> int:
+    """Convenience: tardis_fold from an object with the fields W1, W2, b1, b2, lo, hi, a, c, codes, scale,
+    zero and cfg.group / cfg.act / cfg.bits (all CUDA tensors)."""
+    return tardis_fold(layer.W1, layer.W2, layer.lo, layer.hi, layer.a, layer.c, layer.codes, layer.scale,
+                       layer.zero, layer.cfg.group, b1=layer.b1, b2=layer.b2, act=layer.cfg.act,
+                       pred_bits=layer.cfg.bits, stream=stream)

@@ -1,0 +1,199 @@
+// C ABI of libtardis: argument validation, handle life cycle, dispatch.
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+namespace tardis {
+
+static thread_local char g_last_error[256] = "";
+
+void set_last_error(cudaError_t e, const char* where) {
+  snprintf(g_last_error, sizeof(g_last_error), "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static Handle* check(tardis_handle_t h) {
+  Handle* H = reinterpret_cast<Handle*>(h);
+  if (!H || H->magic != kMagic) return nullptr;
+  return H;
+}
+
+template <typename T>
+static tardis_status_t dev_alloc(T** p, size_t count, size_t* tally) {
+  *p = nullptr;
+  size_t bytes = count * sizeof(T);
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes ? bytes : 16);
+  if (e != cudaSuccess) {
+    set_last_error(e, "cudaMalloc");
+    cudaGetLastError();
+    return TARDIS_ERR_ALLOC;
+  }
+  if (tally) *tally += bytes;
+  return TARDIS_OK;
+}
+
+static void free_all(Handle* H) {
+  decode_release(H);
+  void* ptrs[] = {H->W1, H->W2T, H->C, H->bf, H->lo, H->hi, H->a, H->c, H->b1, H->codes, H->scale,
+                  H->zero, H->yacc, H->bitmap, H->counters};
+  for (void* p : ptrs)
+    if (p) cudaFree(p);
+  H->magic = 0;
+  delete H;
+}
+
+}  // namespace tardis
+
+using namespace tardis;
+
+extern "C" {
+
+tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stream, tardis_handle_t* out) {
+  if (!desc || !out) return TARDIS_ERR_INVALID_ARG;
+  *out = nullptr;
+  const int d = desc->d_model, h = desc->d_ff, G = desc->pred_group;
+  if (d <= 0 || h <= 0 || G <= 0) return TARDIS_ERR_INVALID_ARG;
+  if (desc->dtype != TARDIS_F32 && desc->dtype != TARDIS_BF16) return TARDIS_ERR_INVALID_ARG;
+  if (desc->act != TARDIS_ACT_GELU_TANH && desc->act != TARDIS_ACT_GELU_ERF) return TARDIS_ERR_INVALID_ARG;
+  if (desc->flags != 0) return TARDIS_ERR_INVALID_ARG;
+  if (d % 8 || h % 32 || G % 16 || d % G) return TARDIS_ERR_INVALID_ARG;
+  if (desc->pred_bits != 2) return desc->pred_bits > 0 && desc->pred_bits <= 8 ? TARDIS_ERR_UNSUPPORTED : TARDIS_ERR_INVALID_ARG;
+  const void* required[] = {desc->W1, desc->W2, desc->lo, desc->hi, desc->a, desc->c,
+                            desc->pred_codes, desc->pred_scale, desc->pred_zero};
+  for (const void* p : required)
+    if (!p) return TARDIS_ERR_INVALID_ARG;
+  const void* al[] = {desc->W1, desc->W2, desc->pred_codes, desc->pred_scale};
+  for (const void* p : al)
+    if (!aligned16(p)) return TARDIS_ERR_INVALID_ARG;
+
+  Handle* H = new (std::nothrow) Handle();
+  if (!H) return TARDIS_ERR_ALLOC;
+  memset(H, 0, sizeof(*H));
+  H->magic = kMagic;
+  H->d = d; H->h = h; H->dtype = desc->dtype; H->act = desc->act; H->G = G; H->ngroups = d / G;
+  H->esize = desc->dtype == TARDIS_F32 ? 4 : 2;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  H->last_stream = s;
+  cudaError_t e = cudaGetDevice(&H->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&H->num_sms, cudaDevAttrMultiProcessorCount, H->device);
+  if (e != cudaSuccess) { set_last_error(e, "device query"); delete H; return TARDIS_ERR_CUDA; }
+
+  const size_t hd = size_t(h) * d;
+  tardis_status_t st = TARDIS_OK;
+  auto A = [&](auto** p, size_t count, size_t* tally) { if (st == TARDIS_OK) st = dev_alloc(p, count, tally); };
+  A(reinterpret_cast<char**>(&H->W1), hd * H->esize, &H->bytes_w1);
+  A(reinterpret_cast<char**>(&H->W2T), hd * H->esize, &H->bytes_w2t);
+  A(reinterpret_cast<char**>(&H->C), size_t(d) * d * H->esize, &H->bytes_folded);
+  A(&H->bf, size_t(d), &H->bytes_folded);
+  A(&H->lo, size_t(h), &H->bytes_tables);
+  A(&H->hi, size_t(h), &H->bytes_tables);
+  A(&H->a, size_t(h), &H->bytes_tables);
+  A(&H->c, size_t(h), &H->bytes_tables);
+  A(&H->b1, size_t(h), &H->bytes_tables);
+  A(&H->codes, hd / 16, &H->bytes_predictor);
+  A(reinterpret_cast<char**>(&H->scale), size_t(h) * H->ngroups * H->esize, &H->bytes_predictor);
+  A(&H->zero, size_t(h) * H->ngroups, &H->bytes_predictor);
+  A(&H->yacc, size_t(kGenericChunk) * d, &H->bytes_scratch);
+  A(&H->bitmap, size_t(kGenericChunk) * (h / 32), &H->bytes_scratch);
+  A(&H->counters, size_t(CTR_COUNT), &H->bytes_scratch);
+  if (st != TARDIS_OK) { free_all(H); return st; }
+
+  st = launch_fold(H, desc, s);
+  if (st == TARDIS_OK && H->dtype == TARDIS_BF16) st = decode_prepare(H, s);
+  if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
+  *out = reinterpret_cast<tardis_handle_t>(H);
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* y, int64_t n_tokens,
+                                   tardis_stream_t stream) {
+  Handle* H = check(handle);
+  if (!H) return TARDIS_ERR_INVALID_ARG;
+  if (n_tokens < 0) return TARDIS_ERR_INVALID_ARG;
+  if (n_tokens == 0) return TARDIS_OK;
+  if (!x || !y || !aligned16(x) || !aligned16(y)) return TARDIS_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  H->last_stream = s;
+  tardis_status_t st;
+  const bool fused = H->path_override == 0 && H->codes_mma != nullptr && n_tokens <= kDecodeMaxTokens;
+  if (fused) {
+    st = launch_decode_forward(H, x, y, int(n_tokens), s);
+    H->last_path = 2;
+  } else {
+    st = launch_generic_forward(H, x, y, n_tokens, s);
+    H->last_path = 1;
+  }
+  if (st == TARDIS_OK) { H->calls += 1; H->tokens += uint64_t(n_tokens); }
+  return st;
+}
+
+tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
+  Handle* H = check(handle);
+  if (!H || !out) return TARDIS_ERR_INVALID_ARG;
+  TARDIS_CUDA_TRY(cudaStreamSynchronize(H->last_stream));
+  unsigned long long ctr[CTR_COUNT];
+  TARDIS_CUDA_TRY(cudaMemcpy(ctr, H->counters, sizeof(ctr), cudaMemcpyDeviceToHost));
+  memset(out, 0, sizeof(*out));
+  out->calls = H->calls; out->tokens = H->tokens; out->last_path = H->last_path;
+  out->flagged_total = ctr[CTR_FLAGGED_TOTAL]; out->flagged_max = ctr[CTR_FLAGGED_MAX];
+  out->device_error = ctr[CTR_ERROR]; out->exact_rechecks = ctr[CTR_RECHECKS];
+  out->bytes_folded = H->bytes_folded; out->bytes_predictor = H->bytes_predictor;
+  out->bytes_tables = H->bytes_tables; out->bytes_w1 = H->bytes_w1; out->bytes_w2t = H->bytes_w2t;
+  out->bytes_scratch = H->bytes_scratch;
+  if (ctr[CTR_ERROR] == 1) return TARDIS_ERR_TIMEOUT;
+  if (ctr[CTR_ERROR] != 0) return TARDIS_ERR_CORRUPT;
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_set_debug_capture(tardis_handle_t handle, uint32_t* flag_bitmap, double* scores) {
+  Handle* H = check(handle);
+  if (!H) return TARDIS_ERR_INVALID_ARG;
+  H->dbg_bitmap = flag_bitmap;
+  H->dbg_scores = scores;
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf, tardis_stream_t stream) {
+  Handle* H = check(handle);
+  if (!H) return TARDIS_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  H->last_stream = s;
+  return launch_export_folded(H, Wf, bf, s);
+}
+
+tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path) {
+  Handle* H = check(handle);
+  if (!H || path < 0 || path > 1) return TARDIS_ERR_INVALID_ARG;
+  H->path_override = path;
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_destroy(tardis_handle_t handle) {
+  Handle* H = check(handle);
+  if (!H) return TARDIS_ERR_INVALID_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  free_all(H);
+  if (e != cudaSuccess) { set_last_error(e, "cudaDeviceSynchronize"); return TARDIS_ERR_CUDA; }
+  return TARDIS_OK;
+}
+
+const char* tardis_status_string(tardis_status_t status) {
+  switch (status) {
+    case TARDIS_OK: return "ok";
+    case TARDIS_ERR_INVALID_ARG: return "invalid argument";
+    case TARDIS_ERR_UNSUPPORTED: return "unsupported configuration";
+    case TARDIS_ERR_ALLOC: return "device allocation failed";
+    case TARDIS_ERR_CUDA: return "CUDA error";
+    case TARDIS_ERR_TIMEOUT: return "device-side wait timed out";
+    case TARDIS_ERR_CORRUPT: return "handle corrupt";
+  }
+  return "unknown status";
+}
+
+const char* tardis_last_error(void) { return g_last_error; }
+
+}  // extern "C"

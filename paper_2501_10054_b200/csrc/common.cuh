@@ -1,0 +1,94 @@
+// Shared declarations of libtardis (internal; the public interface is include/tardis.h).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tardis.h"
+
+namespace tardis {
+
+constexpr uint64_t kMagic = 0x7A2D15F01DULL;
+constexpr int kGenericChunk = 256;   // tokens per pass of the generic kernels (scratch is sized for this)
+constexpr int kDecodeMaxTokens = 8;  // largest batch the fused decode kernel takes
+
+// device counter slots
+enum { CTR_FLAGGED_TOTAL = 0, CTR_FLAGGED_MAX = 1, CTR_ERROR = 2, CTR_RECHECKS = 3, CTR_TICKET = 4, CTR_COUNT = 8 };
+
+struct Handle {
+  uint64_t magic;
+  int d, h, dtype, act, G, ngroups;
+  size_t esize;
+  int device;
+  // state (device)
+  void* W1;        // [h, d]   original rows (result fixing recomputes z_j from these)
+  void* W2T;       // [h, d]   W2 transposed: row j = output weights of neuron j
+  void* C;         // [d, d]   C[k, i] = W_f[i, k]  (the paper's folded matrix, row k = input channel k)
+  float* bf;       // [d]
+  float *lo, *hi, *a, *c, *b1;   // [h]; b1 is zeros when the layer has no bias
+  uint32_t* codes; // [h, d/16]
+  void* scale;     // [h, d/G]
+  uint8_t* zero;   // [h, d/G]
+  // fused-decode state (bf16 only; null otherwise)
+  uint32_t* codes_mma;   // predictor codes re-packed into tensor-core fragment order
+  float2* pmeta;         // [h/16 tiles][ngroups][16 rows] (scale, scale*zero)
+  // scratch (device)
+  float* yacc;           // [kGenericChunk, d] fp32 accumulator
+  uint32_t* bitmap;      // [kGenericChunk, h/32]
+  unsigned long long* counters;  // [CTR_COUNT]
+  void* dscratch;        // fused decode scratch (see decode.cu)
+  size_t dscratch_bytes;
+  // debug capture (caller-owned)
+  uint32_t* dbg_bitmap;
+  double* dbg_scores;
+  // host-side bookkeeping
+  uint64_t calls, tokens, last_path;
+  cudaStream_t last_stream;
+  int path_override;
+  size_t bytes_folded, bytes_predictor, bytes_tables, bytes_w1, bytes_w2t, bytes_scratch;
+  int num_sms;
+};
+
+void set_last_error(cudaError_t e, const char* where);
+
+#define TARDIS_CUDA_TRY(expr)                                  \
+  do {                                                         \
+    cudaError_t e__ = (expr);                                  \
+    if (e__ != cudaSuccess) {                                  \
+      ::tardis::set_last_error(e__, #expr);                    \
+      return TARDIS_ERR_CUDA;                                  \
+    }                                                          \
+  } while (0)
+
+// ---- kernels' host launchers (each returns after enqueueing on `s`) ----
+tardis_status_t launch_fold(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);
+tardis_status_t launch_export_folded(Handle* H, void* Wf, float* bf, cudaStream_t s);
+tardis_status_t launch_generic_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
+tardis_status_t decode_prepare(Handle* H, cudaStream_t s);                 // builds codes_mma, pmeta, scratch
+tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
+void decode_release(Handle* H);
+
+// ---- small device helpers ----
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float gelu_f32(float z, int act) {
+  if (act == TARDIS_ACT_GELU_TANH) {
+    float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
+    return 0.5f * z * (1.0f + tanhf(u));
+  }
+  return 0.5f * z * (1.0f + erff(z * 0.7071067811865476f));
+}
+__device__ __forceinline__ double gelu_f64(double z, int act) {
+  if (act == TARDIS_ACT_GELU_TANH) {
+    double u = 0.7978845608028654 * (z + 0.044715 * z * z * z);
+    return 0.5 * z * (1.0 + tanh(u));
+  }
+  return 0.5 * z * (1.0 + erf(z * 0.7071067811865476));
+}
+
+}  // namespace tardis

@@ -1,0 +1,137 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle on the same seeded
+inputs.  Flags bit-exact outside the 1e-6 score band; outputs within 1e-5 (fp32) / 2e-2 (bf16)
+max relative error |dy| / max(|y_ref|, rms(y_ref[t,:]))."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2501_10054_b200 as T
+import workloads as W
+from oracle import tardis_oracle as O
+from tests import helpers as Hp
+
+pytestmark = pytest.mark.gpu
+
+
+def _layer(cfg, seed=0):
+    return Hp.to_cuda(W.make_layer(cfg, seed))
+
+
+def _run(cfg, n, calls=None, seed=0, path=0, full_fold=True):
+    L = _layer(cfg, seed)
+    s = L.numpy64()
+    x = W.make_tokens(cfg, n, seed).cuda()
+    h = T.fold_layer(L)
+    try:
+        T.tardis_set_path(h, path)
+        y, F, S = Hp.gpu_forward(h, L, x, calls)
+        info = Hp.assert_parity(L, s, x, y, F, S, full_fold=full_fold, label=cfg.name)
+        st = T.tardis_stats(h)
+        assert st["tokens"] == n and st["device_error"] == 0
+        assert st["flagged_total"] == int(F.sum())
+        assert st["flagged_max"] == int(F.sum(1).max()) if n else True
+    finally:
+        T.tardis_destroy(h)
+    return info
+
+
+def test_tiny_f32_config_all_tokens():
+    cfg = W.CONFIGS["tiny_f32"]
+    info = _run(cfg, 64)
+    assert 0.02 < info["flag_frac"] < 0.4
+
+
+def test_tiny_f32_fold_matches_oracle_elementwise():
+    cfg = W.CONFIGS["tiny_f32"]
+    L = _layer(cfg)
+    s = L.numpy64()
+    h = T.fold_layer(L)
+    Wf = torch.empty(cfg.d_model, cfg.d_model, dtype=torch.float32, device="cuda")
+    bf = torch.empty(cfg.d_model, dtype=torch.float32, device="cuda")
+    T.tardis_export_folded(h, Wf, bf)
+    torch.cuda.synchronize()
+    Wf_ref, bf_ref = O.fold(s["W1"], s["W2"], s["a"], s["c"], s["b1"], s["b2"])
+    assert np.abs(Wf.double().cpu().numpy() - Wf_ref).max() <= 1e-5 * np.abs(Wf_ref).max()
+    assert np.abs(bf.double().cpu().numpy() - bf_ref).max() <= 1e-5 * np.abs(bf_ref).max()
+    st = T.tardis_stats(h)
+    # footprint accounting: folded matrix d^2 against the 2 d h original weights = 12.5 % at h = 4 d,
+    # 2-bit codes = 6.25 % of the original weights
+    assert (st["bytes_folded"] - 4 * cfg.d_model) / (st["bytes_w1"] + st["bytes_w2t"]) == 0.125
+    assert (cfg.d_ff * cfg.d_model // 4) / st["bytes_w1"] == 2 / 32            # 2-bit codes against fp32 W1
+    T.tardis_destroy(h)
+
+
+@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("shape", [(512, 2048, 64), (1136, 4544, 16), (768, 3072, 128)])
+def test_bf16_small_shapes_ragged_batches(shape, path):
+    d, hh, G = shape
+    cfg = W.LayerConfig("small_%d" % d, d, hh, group=G, n_calib=512, bias=(d != 1136),
+                        tokens="mixture" if d == 1136 else "student_t")
+    calls = [1, 1, 3, 8, 9, 0, 2, 64, 65, 5]
+    info = _run(cfg, sum(calls), calls, path=path)
+    assert 0.02 < info["flag_frac"] < 0.5
+
+
+def test_erf_activation_and_other_seed():
+    cfg = W.LayerConfig("erf", 256, 1024, dtype="bf16", act=W.ACT_GELU_ERF, n_calib=512)
+    _run(cfg, 17, [1, 16], seed=5)
+    cfg = W.LayerConfig("erf32", 128, 512, dtype="f32", act=W.ACT_GELU_ERF, n_calib=512)
+    _run(cfg, 9, seed=6)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_degenerate_ranges_all_and_none_flagged(dtype):
+    cfg = W.LayerConfig("deg_" + dtype, 256, 1024, dtype=dtype, n_calib=256)
+    L = _layer(cfg)
+    x = W.make_tokens(cfg, 5, 1).cuda()
+    inf = torch.full_like(L.lo, float("inf"))
+    for lo, hi, frac in ((inf, inf, 1.0), (-inf, inf, 0.0)):
+        L2 = W.Layer(**{**L.__dict__, "lo": lo, "hi": hi})
+        s = L2.numpy64()
+        h = T.fold_layer(L2)
+        y, F, S = Hp.gpu_forward(h, L2, x, [1, 4])
+        assert F.mean() == frac
+        Hp.assert_parity(L2, s, x, y, F, S, label="degenerate")
+        if frac == 1.0:   # every neuron flagged: the original GELU FFN
+            dense = O.dense_ffn(x.double().cpu().numpy(), s["W1"], s["W2"], s["b1"], s["b2"], s["act"])
+            assert O.rel_error(y.double().cpu().numpy(), dense).max() <= Hp.TOL[dtype]
+        T.tardis_destroy(h)
+
+
+def test_nan_token_is_flagged_everywhere_and_propagates():
+    cfg = W.LayerConfig("nan", 256, 1024, dtype="bf16", n_calib=256)
+    L = _layer(cfg)
+    x = W.make_tokens(cfg, 3, 2).cuda()
+    x[1, 7] = float("nan")
+    h = T.fold_layer(L)
+    y, F, S = Hp.gpu_forward(h, L, x, [3])
+    assert F[1].all() and torch.isnan(y[1]).all()
+    assert not torch.isnan(y[0]).any() and not torch.isnan(y[2]).any()
+    T.tardis_destroy(h)
+
+
+def test_forward_argument_errors_and_empty_call():
+    cfg = W.LayerConfig("args", 128, 512, dtype="bf16", n_calib=256)
+    L = _layer(cfg)
+    h = T.fold_layer(L)
+    lib = T.load_library()
+    x = W.make_tokens(cfg, 2, 0).cuda()
+    y = torch.empty_like(x)
+    assert lib.tardis_ffn_forward(h, x.data_ptr(), y.data_ptr(), -1, None) == 1
+    assert lib.tardis_ffn_forward(h, None, y.data_ptr(), 1, None) == 1
+    assert lib.tardis_ffn_forward(h, x.data_ptr() + 2, y.data_ptr(), 1, None) == 1
+    assert lib.tardis_ffn_forward(h, None, None, 0, None) == 0          # empty call is a no-op
+    assert T.tardis_stats(h)["calls"] == 0
+    T.tardis_destroy(h)
+
+
+def test_run_to_run_flags_identical():
+    cfg = W.LayerConfig("rep", 512, 2048, n_calib=512)
+    L = _layer(cfg)
+    x = W.make_tokens(cfg, 8, 0).cuda()
+    h = T.fold_layer(L)
+    y1, F1, S1 = Hp.gpu_forward(h, L, x, [8])
+    y2, F2, S2 = Hp.gpu_forward(h, L, x, [8])
+    assert (F1 == F2).all() and (S1 == S2).all()
+    assert (y1.float() - y2.float()).abs().max() <= 2e-2 * y1.float().abs().max()
+    T.tardis_destroy(h)
