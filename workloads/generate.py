@@ -65,9 +65,9 @@ class LayerConfig:
 # The five configurations the benchmark definition names.
 CONFIGS = {
     "tiny_f32": LayerConfig("tiny_f32", 256, 1024, dtype="f32", n_calib=4096, q_lo=0.05, q_hi=0.95),
-    "decode_7b": LayerConfig("decode_7b", 4096, 16384, n_calib=2048, target_flag_frac=0.10),
+    "decode_7b": LayerConfig("decode_7b", 4096, 16384, n_calib=2048, target_flag_frac=0.10, group=128),
     "falcon_7b": LayerConfig("falcon_7b", 4544, 18176, bias=False, tokens="mixture", n_calib=2048),
-    "prefill_7b": LayerConfig("prefill_7b", 4096, 16384, n_calib=2048, target_flag_frac=0.10),
+    "prefill_7b": LayerConfig("prefill_7b", 4096, 16384, n_calib=2048, target_flag_frac=0.10, group=128),
     "large_8k": LayerConfig("large_8k", 8192, 32768, n_calib=2048, target_flag_frac=0.10, group=128),
 }
 # quantile pairs of the Falcon-shaped sweep (flagged fraction about 5/10/20/30 %)
