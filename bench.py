@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the partially linear FFN forward (TARDIS, arXiv 2501.10054) on B200.
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+    python bench.py --impl reference --steps K --warmup W    # the fp64 CPU oracle on the host cores
+
+Workload (default): the 7B-class decode configuration - one FFN layer shape d_model = 4096,
+d_ff = 16384, bf16, about 10 % of the neurons flagged per token - run as batch-1 decode.  One
+"step" is 512 successive tokens, each one call of tardis_ffn_forward (predictor, flagging, folded
+product, result fixing).  Calls rotate over `--layers` independently seeded layers so that the
+state a call touches (about 80 MB) has left the 126 MB L2 by the time its layer comes round again.
+Prints ONE JSON line; see the design doc for the meaning of every key.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tardis_ffn_tokens_per_s"
+UNIT = "tokens/s"
+L2_BYTES = 126e6
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="tardis", choices=["tardis", "reference"])
+    ap.add_argument("--workload", default="decode_7b")
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--tokens", type=int, default=512, help="tokens per step")
+    ap.add_argument("--layers", type=int, default=8, help="independent layers the calls rotate over (L2-cold)")
+    ap.add_argument("--graph", type=int, default=0, help="replay one step as a CUDA graph")
+    ap.add_argument("--no-context", action="store_true", help="skip the dense-FFN / batch-64 / oracle context legs")
+    ap.add_argument("--cpu-sample-tokens", type=int, default=16)
+    return ap.parse_args()
+
+
+def algorithmic_bytes(cfg, batch, union_flagged):
+    """Bytes one call must move (bf16): folded matrix + predictor codes + group metadata (4 B per
+    neuron and group) + W1 row and W2^T row of every flagged neuron + per-neuron tables + bias + x, y."""
+    d, h, G = cfg.d_model, cfg.d_ff, cfg.group
+    return (2 * d * d + h * d // 4 + 4 * h * (d // G) + union_flagged * 4 * d + 12 * h + 8 * union_flagged
+            + 4 * d + 4 * batch * d)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown if hasattr(nv, "nvmlClocksEventReasonHwSlowdown") else 0x8,
+                 "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4, "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def oracle_sample(cfg, layer64, x64, reps=1):
+    """The oracle as it stands on the host cores: fold once (offline part), then the online part
+    (predictor score, flags, folded product, fixing) on the sample tokens.  Returns (tokens/s, fold_s, cores)."""
+    from threadpoolctl import threadpool_info
+    from oracle import tardis_oracle as O
+    s = layer64
+    t0 = time.perf_counter()
+    folded = O.fold(s["W1"], s["W2"], s["a"], s["c"], s["b1"], s["b2"])
+    fold_s = time.perf_counter() - t0
+    best = float("inf")
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        O.tardis_ffn(x64, s["W1"], s["W2"], s["a"], s["c"], s["lo"], s["hi"], s["codes"], s["scale"], s["zero"],
+                     s["group"], s["b1"], s["b2"], s["act"], s["bits"], folded=folded)
+        best = min(best, time.perf_counter() - t0)
+    cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    return x64.shape[0] / best, fold_s, cores
+
+
+def run_reference(args):
+    """--impl reference: the fp64 oracle on the host cores, same metric and workload, bounded sample."""
+    import workloads as W
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = W.CONFIGS[args.workload]
+    L = W.make_layer(cfg, 0)
+    s = L.numpy64()
+    n = max(1, min(args.cpu_sample_tokens, 8))
+    x64 = W.make_tokens(cfg, n, 0).double().numpy()
+    from oracle import tardis_oracle as O
+    folded = O.fold(s["W1"], s["W2"], s["a"], s["c"], s["b1"], s["b2"])
+
+    def step():
+        O.tardis_ffn(x64, s["W1"], s["W2"], s["a"], s["c"], s["lo"], s["hi"], s["codes"], s["scale"], s["zero"],
+                     s["group"], s["b1"], s["b2"], s["act"], s["bits"], folded=folded)
+
+    steps, warm = max(1, min(args.steps, 5)), max(1, min(args.warmup, 2))
+    for _ in range(warm):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    from threadpoolctl import threadpool_info
+    cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    val = n / dt
+    sample = "%d tokens per step, %d steps, batch-1 semantics (tokens independent), fold excluded (offline)" % (n, steps)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s batch-%d decode, d_model=%d d_ff=%d" % (cfg.name, args.batch, cfg.d_model, cfg.d_ff)},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    import torch.distributed as dist
+    import paper_2501_10054_b200 as T
+    from paper_2501_10054_b200 import build as tbuild
+    import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        tbuild.build()
+    if world > 1:
+        dist.barrier()
+    lib = T.load_library()
+
+    cfg = W.CONFIGS[args.workload]
+    d, h, B, NT = cfg.d_model, cfg.d_ff, args.batch, args.tokens
+    assert NT % B == 0
+    # ---- set-up: independent layers (weak scaling: every rank has its own layers and tokens) ----
+    handles, dense = [], []
+    layer0_64 = None
+    for l in range(args.layers):
+        L = W.make_layer(cfg, seed=rank * 1000 + l, device=dev)
+        handles.append(T.fold_layer(L))
+        dense.append((L.W1, L.W2, L.b1, L.b2))
+        if l == 0 and rank == 0 and not args.no_context:
+            layer0_64 = L.numpy64()
+    x_all = W.make_tokens(cfg, NT, seed=rank, device=dev)
+    y_all = torch.empty_like(x_all)
+    torch.cuda.synchronize()
+    touched = algorithmic_bytes(cfg, B, int(0.1 * h))
+    stream = torch.cuda.current_stream()
+    sptr = stream.cuda_stream or None
+    esz = x_all.element_size()
+    fwd = lib.tardis_ffn_forward
+
+    def make_step(batch, xs, ys):
+        calls = [(handles[i % len(handles)], xs.data_ptr() + i * batch * d * esz, ys.data_ptr() + i * batch * d * esz)
+                 for i in range(NT // batch)]
+
+        def step():
+            for hdl, xp, yp in calls:
+                st = fwd(hdl, xp, yp, batch, sptr)
+                if st:
+                    raise RuntimeError("tardis_ffn_forward status %d" % st)
+        return step
+
+    def timed(step, steps, warm, sampler=None, graph=False):
+        runner = step
+        if graph:
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step()
+            torch.cuda.current_stream().wait_stream(side)
+            with torch.cuda.graph(g):
+                step()
+            runner = g.replay
+        for _ in range(max(3, warm)):
+            runner()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ctx = sampler if sampler is not None else _Null()
+        with ctx:
+            e0.record()
+            for _ in range(steps):
+                runner()
+            e1.record()
+            torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    # ---- device-resident timing (the headline `value`) ----
+    st0 = [T.tardis_stats(hd) for hd in handles]
+    sampler = ClockSampler(local)
+    step = make_step(B, x_all, y_all)
+    if args.graph:
+        # the graph path captures on torch's capture stream: rebuild the call list inside timed()
+        def step_graph():
+            s2 = torch.cuda.current_stream().cuda_stream or None
+            for i in range(NT // B):
+                st = fwd(handles[i % len(handles)], x_all.data_ptr() + i * B * d * esz, y_all.data_ptr() + i * B * d * esz, B, s2)
+                if st:
+                    raise RuntimeError("tardis_ffn_forward status %d" % st)
+        ms = timed(step_graph, args.steps, args.warmup, sampler, graph=True)
+    else:
+        ms = timed(step, args.steps, args.warmup, sampler)
+    st1 = [T.tardis_stats(hd) for hd in handles]
+    if any(s["device_error"] for s in st1):
+        raise SystemExit("device error word set: %r" % [s["device_error"] for s in st1])
+    tokens_done = sum(b["tokens"] - a["tokens"] for a, b in zip(st0, st1))
+    flagged = sum(b["flagged_total"] - a["flagged_total"] for a, b in zip(st0, st1)) / max(1, tokens_done)
+    launches_per_step = sum(b["launches"] - a["launches"] for a, b in zip(st0, st1)) / (max(3, args.warmup) + args.steps)
+    value = world * NT / (ms * 1e-3)
+
+    # ---- end to end: host buffers, H2D of the step's tokens and D2H of its outputs inside the timed region ----
+    xh = x_all.cpu().pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    xd = torch.empty_like(x_all)
+    yd = torch.empty_like(x_all)
+    inner = make_step(B, xd, yd)
+
+    def e2e_step():
+        xd.copy_(xh, non_blocking=True)
+        inner()
+        yh.copy_(yd, non_blocking=True)
+
+    ms_e2e = timed(e2e_step, max(3, args.steps // 4), 3)
+    e2e_value = world * NT / (ms_e2e * 1e-3)
+
+    # ---- roofline of the dominant kernel ----
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_src = "measured" if "hbm_gbs" in peaks else "fallback"
+    calls_per_step = NT // B
+    union = flagged if B == 1 else h * (1 - (1 - flagged / h) ** B)
+    alg = algorithmic_bytes(cfg, B, union)
+    dur_s = ms * 1e-3 / calls_per_step
+    achieved = alg / dur_s / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_source": peak_src, "kernel": "k_decode" if B <= 8 else "generic",
+                "algorithmic_bytes_per_launch": alg, "avg_launch_us": dur_s * 1e6,
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+    prof = os.path.join(ROOT, "profiles", "k_decode_traffic.json")
+    if os.path.exists(prof):
+        try:
+            roofline["traffic"] = json.load(open(prof)).get(args.workload)
+        except Exception:
+            pass
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype,
+        "data": "synthetic",
+        "config": {"workload": "%s batch-%d decode, d_model=%d d_ff=%d, %d tokens/step" % (cfg.name, B, d, h, NT),
+                   "flagged_per_token": flagged, "flagged_frac": flagged / h, "pred_group": cfg.group,
+                   "l2": "inputs larger than L2: calls rotate over %d independent layers (%.0f MB touched per call, %.0f MB per round)"
+                         % (len(handles), touched / 1e6, touched * len(handles) / 1e6),
+                   "cuda_graph": bool(args.graph)},
+        "clocks": sampler.summary(),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": xh.numel() * esz, "d2h_bytes_per_step": yh.numel() * esz,
+                "ms_per_step": ms_e2e},
+        "gpu_launches": int(round(launches_per_step * args.steps)),
+        "roofline": roofline,
+    }
+
+    # ---- context legs (rank 0, N = 1 semantics): batch 64, dense FFN, oracle on the host cores ----
+    if not args.no_context:
+        if NT % 64 == 0 and B != 64:
+            s0 = [T.tardis_stats(hd) for hd in handles]
+            ms64 = timed(make_step(64, x_all, y_all), max(3, args.steps // 4), 3)
+            out["batch64"] = {"value": world * NT / (ms64 * 1e-3), "unit": UNIT, "ms_per_step": ms64,
+                              "path": T.tardis_stats(handles[0])["last_path"]}
+
+        def dense_step():
+            for i in range(NT // B):
+                W1, W2, b1, b2 = dense[i % len(dense)]
+                xb = x_all[i * B:(i + 1) * B]
+                hid = torch.nn.functional.gelu(torch.nn.functional.linear(xb, W1, None if b1 is None else b1.to(W1.dtype)),
+                                               approximate="tanh" if cfg.act == 0 else "none")
+                torch.nn.functional.linear(hid, W2, None if b2 is None else b2.to(W2.dtype))
+
+        msd = timed(dense_step, max(3, args.steps // 4), 3)
+        out["dense_ffn_context"] = {"value": world * NT / (msd * 1e-3), "unit": UNIT, "ms_per_step": msd,
+                                    "what": "torch bf16 linear-gelu-linear, same rotation, same GPU",
+                                    "bytes_per_call": 4 * d * h}
+        out["paper_context"] = {"e2e_speedup_vllm": 1.59, "e2e_speedup_hf": 1.39, "ffn_speedup": 1.86,
+                                "hardware": "RTX 4090D, Falcon-7B, 80% FFN compression (paper Section 7.4)"}
+        if rank == 0 and layer0_64 is not None:
+            n = args.cpu_sample_tokens
+            x64 = x_all[:n].double().cpu().numpy()
+            v, fold_s, cores = oracle_sample(cfg, layer0_64, x64)
+            out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                   "sample": "online path on %d tokens of layer 0 (fold excluded: offline, %.1f s)" % (n, fold_s),
+                                   "fold_s": fold_s}
+    if rank == 0:
+        print(json.dumps(out))
+    for hd in handles:
+        T.tardis_destroy(hd)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+class _Null:
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        return False
+
+
+if __name__ == "__main__":
+    main()

@@ -144,6 +144,7 @@ tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
   out->bytes_folded = H->bytes_folded; out->bytes_predictor = H->bytes_predictor;
   out->bytes_tables = H->bytes_tables; out->bytes_w1 = H->bytes_w1; out->bytes_w2t = H->bytes_w2t;
   out->bytes_scratch = H->bytes_scratch;
+  out->launches = H->launches;
   if (ctr[CTR_ERROR] == 1) return TARDIS_ERR_TIMEOUT;
   if (ctr[CTR_ERROR] != 0) return TARDIS_ERR_CORRUPT;
   return TARDIS_OK;

@@ -42,7 +42,7 @@ struct Handle {
   uint32_t* dbg_bitmap;
   double* dbg_scores;
   // host-side bookkeeping
-  uint64_t calls, tokens, last_path;
+  uint64_t calls, tokens, last_path, launches;
   cudaStream_t last_stream;
   int path_override;
   size_t bytes_folded, bytes_predictor, bytes_tables, bytes_w1, bytes_w2t, bytes_scratch;

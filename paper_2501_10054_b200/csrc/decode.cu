@@ -697,6 +697,7 @@ tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, 
     p.dbg_bitmap = H->dbg_bitmap ? H->dbg_bitmap + size_t(t) * (H->h / 32) : nullptr;
     p.dbg_scores = H->dbg_scores ? H->dbg_scores + size_t(t) * H->h : nullptr;
     k_decode<<<H->num_sms, NTHREADS, S->smem_bytes, s>>>(p);
+    H->launches += 1;
   }
   TARDIS_CUDA_TRY(cudaGetLastError());
   return TARDIS_OK;

@@ -198,6 +198,7 @@ static tardis_status_t generic_typed(Handle* H, const T* x, T* y, int64_t n_tota
     k_fix<T, Acc><<<dim3(n, (h + 1023) / 1024), 256, size_t(d) * sizeof(float), s>>>(
         static_cast<const T*>(H->W1), static_cast<const T*>(H->W2T), H->b1, H->a, H->c, xc, H->bitmap, H->yacc, d, h, H->act);
     k_store_y<T><<<unsigned((cnt + 255) / 256), 256, 0, s>>>(H->yacc, y + size_t(t0) * d, cnt);
+    H->launches += 6;
   }
   TARDIS_CUDA_TRY(cudaGetLastError());
   return TARDIS_OK;
