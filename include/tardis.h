@@ -82,7 +82,8 @@ typedef struct {
   uint64_t tokens;              /* tokens processed                                        */
   uint64_t flagged_total;       /* sum over tokens of flagged neurons                      */
   uint64_t flagged_max;         /* largest flagged count of a single token                 */
-  uint64_t last_path;           /* 0 none, 1 generic, 2 fused decode, 3 batched/prefill    */
+  uint64_t last_path;           /* 0 none, 1 generic, 2 fused decode, 3 batched/prefill,
+                                   4 generic kernels on the library's built-in scratch     */
   uint64_t bytes_folded;        /* W_f and b_f                                             */
   uint64_t bytes_predictor;     /* codes + scales + zero-points as stored                  */
   uint64_t bytes_tables;        /* lo, hi, a, c, b1                                        */
@@ -121,6 +122,30 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
  * n_tokens < 0), CUDA. */
 tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* y,
                                    int64_t n_tokens, tardis_stream_t stream);
+
+/* The online part for callers that must not allocate device memory.  (The paper has no counterpart of
+ * this call; it exists for the way this library gets embedded.)  Some hosts of this code cannot go
+ * to the CUDA allocator once they are running: a serving process that handed all device memory to
+ * its own pool at start-up, a control loop with a "no driver allocation after initialisation" rule,
+ * code that runs while a stream is being captured.  tardis_ffn_forward already takes its scratch
+ * from the handle; this variant takes it from neither the handle nor the allocator: the fp32 output
+ * accumulator and the flag bitmap of the call live in a fixed 4 MiB array that is part of the
+ * library image (every GPU that loads the library holds those 4 MiB until the process exits).  It
+ * calls no cudaMalloc, cudaFree or other allocating routine.
+ * Same arguments, result and error behaviour as tardis_ffn_forward, computed by the generic
+ * kernels, with these differences:
+ *   - n_tokens <= 64 and n_tokens * (4 * d_model + d_ff / 8) <= 4 MiB (each of the two terms rounded
+ *     up to 256 bytes), else TARDIS_ERR_UNSUPPORTED with the reason in tardis_last_error; the
+ *     handle's device must be the current device, else TARDIS_ERR_INVALID_ARG;
+ *   - the first call on a device asks the runtime for the array's device address
+ *     (cudaGetSymbolAddress) and keeps it; make that first call before any stream capture starts;
+ *   - the array is shared by every call and every handle in the process and keeps what the last
+ *     call left in it.  A call overwrites all of the part it uses before reading it, so stale
+ *     contents are harmless, but two calls that overlap in time on the GPU (different streams, or
+ *     one of them tardis_ffn_forward_static and the other any work still using the array) race:
+ *     order them on one stream or with events. */
+tardis_status_t tardis_ffn_forward_static(tardis_handle_t handle, const void* x, void* y,
+                                          int64_t n_tokens, tardis_stream_t stream);
 
 /* Synchronises the stream of the handle's most recent call, then fills *out
  * (host memory).  Returns TIMEOUT / CORRUPT when the device error word says so. */

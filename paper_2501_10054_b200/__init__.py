@@ -20,9 +20,9 @@ TARDIS_OK = 0
 TARDIS_F32, TARDIS_BF16 = 0, 1
 TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF = 0, 1
 
-EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_stats", "tardis_set_debug_capture",
-           "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_status_string",
-           "tardis_last_error"]
+EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_stats",
+           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy",
+           "tardis_status_string", "tardis_last_error"]
 
 
 class TardisError(RuntimeError):
@@ -67,12 +67,13 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
     lib.tardis_fold.argtypes = [ctypes.POINTER(FoldDesc), vp, ctypes.POINTER(vp)]
     lib.tardis_ffn_forward.argtypes = [vp, vp, vp, i64, vp]
+    lib.tardis_ffn_forward_static.argtypes = [vp, vp, vp, i64, vp]
     lib.tardis_stats.argtypes = [vp, ctypes.POINTER(Stats)]
     lib.tardis_set_debug_capture.argtypes = [vp, vp, vp]
     lib.tardis_export_folded.argtypes = [vp, vp, vp, vp]
     lib.tardis_set_path.argtypes = [vp, i32]
     lib.tardis_destroy.argtypes = [vp]
-    for name in EXPORTS[:7]:
+    for name in EXPORTS[:8]:
         getattr(lib, name).restype = ctypes.c_int
     lib.tardis_status_string.argtypes = [ctypes.c_int]
     lib.tardis_status_string.restype = ctypes.c_char_p
@@ -129,6 +130,18 @@ def tardis_ffn_forward(handle: int, x: torch.Tensor, y: torch.Tensor, n_tokens: 
     lib = load_library()
     n = x.shape[0] if n_tokens is None else n_tokens
     _check(lib.tardis_ffn_forward(handle, _ptr(x), _ptr(y), n, _stream(stream)), "tardis_ffn_forward")
+    return y
+
+
+def tardis_ffn_forward_static(handle: int, x: torch.Tensor, y: torch.Tensor, n_tokens: Optional[int] = None, stream=None):
+    """tardis_ffn_forward_static of the C ABI: the same forward for callers that may not allocate device
+    memory; its scratch is a fixed array inside the library (at most 64 tokens, 4 MiB of scratch)."""
+    lib = load_library()
+    n = x.shape[0] if n_tokens is None else n_tokens
+    st = lib.tardis_ffn_forward_static(handle, _ptr(x), _ptr(y), n, _stream(stream))
+    if st == 2:
+        raise TardisError(st, "tardis_ffn_forward_static: %s" % lib.tardis_last_error().decode())
+    _check(st, "tardis_ffn_forward_static")
     return y
 
 

@@ -131,6 +131,28 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   return st;
 }
 
+tardis_status_t tardis_ffn_forward_static(tardis_handle_t handle, const void* x, void* y, int64_t n_tokens,
+                                         tardis_stream_t stream) {
+  Handle* H = check(handle);
+  if (!H) return TARDIS_ERR_INVALID_ARG;
+  if (n_tokens < 0) return TARDIS_ERR_INVALID_ARG;
+  if (n_tokens == 0) return TARDIS_OK;
+  if (!x || !y || !aligned16(x) || !aligned16(y)) return TARDIS_ERR_INVALID_ARG;
+  if (n_tokens > kStaticMaxTokens) {
+    snprintf(g_last_error, sizeof(g_last_error), "tardis_ffn_forward_static: n_tokens %lld exceeds the limit of %d",
+             (long long)n_tokens, kStaticMaxTokens);
+    return TARDIS_ERR_UNSUPPORTED;
+  }
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  H->last_stream = s;
+  const tardis_status_t st = launch_static_forward(H, x, y, n_tokens, s);
+  if (st == TARDIS_ERR_UNSUPPORTED)
+    snprintf(g_last_error, sizeof(g_last_error),
+             "tardis_ffn_forward_static: n_tokens * (4 d_model + d_ff / 8) exceeds the 4 MiB of built-in scratch (or d_model > 12288)");
+  if (st == TARDIS_OK) { H->last_path = 4; H->calls += 1; H->tokens += uint64_t(n_tokens); }
+  return st;
+}
+
 tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
   Handle* H = check(handle);
   if (!H || !out) return TARDIS_ERR_INVALID_ARG;

@@ -11,6 +11,7 @@ namespace tardis {
 constexpr uint64_t kMagic = 0x7A2D15F01DULL;
 constexpr int kGenericChunk = 256;   // tokens per pass of the generic kernels (scratch is sized for this)
 constexpr int kDecodeMaxTokens = 8;  // largest batch the fused decode kernel takes
+constexpr int kStaticMaxTokens = 64; // largest batch of the forward that keeps its scratch in the library image
 
 // device counter slots
 enum { CTR_FLAGGED_TOTAL = 0, CTR_FLAGGED_MAX = 1, CTR_ERROR = 2, CTR_RECHECKS = 3, CTR_TICKET = 4, CTR_COUNT = 8 };
@@ -64,6 +65,7 @@ void set_last_error(cudaError_t e, const char* where);
 tardis_status_t launch_fold(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);
 tardis_status_t launch_export_folded(Handle* H, void* Wf, float* bf, cudaStream_t s);
 tardis_status_t launch_generic_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
+tardis_status_t launch_static_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
 tardis_status_t decode_prepare(Handle* H, cudaStream_t s);                 // builds codes_mma, pmeta, scratch
 tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
 void decode_release(Handle* H);

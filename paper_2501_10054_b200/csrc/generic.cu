@@ -204,6 +204,74 @@ static tardis_status_t generic_typed(Handle* H, const T* x, T* y, int64_t n_tota
   return TARDIS_OK;
 }
 
+// ---- forward whose scratch is part of the library image -----------------------------------------------
+// Same kernels as above, but the fp32 accumulator and the flag bitmap live in one file-scope device array
+// instead of memory obtained from the allocator.  Every GPU that loads the library carries the array
+// until the process exits; all calls (of all handles) share it.
+constexpr size_t kStaticScratchBytes = size_t(4) << 20;   // 4 MiB
+constexpr int kStaticMaxDevices = 64;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch on `device` (which must be current).  In host code the array's name
+// is only a stand-in for the symbol, never a pointer a kernel may use: the address comes from the runtime,
+// once per device.
+static tardis_status_t static_scratch_address(int device, unsigned char** out) {
+  static unsigned char* cache[kStaticMaxDevices] = {};
+  if (device < 0 || device >= kStaticMaxDevices) return TARDIS_ERR_UNSUPPORTED;
+  if (!cache[device]) {
+    void* ptr = nullptr;
+    TARDIS_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    cache[device] = static_cast<unsigned char*>(ptr);
+  }
+  *out = cache[device];
+  return TARDIS_OK;
+}
+
+template <typename T, typename Acc>
+static tardis_status_t static_typed(Handle* H, const T* x, T* y, int n, float* yacc, uint32_t* bitmap, cudaStream_t s) {
+  const int d = H->d, h = H->h;
+  k_predictor_exact<T><<<h / 32, 1024, 0, s>>>(H->codes, static_cast<const T*>(H->scale), H->zero, H->b1, H->lo, H->hi,
+                                               x, n, d, h, H->G, bitmap, H->dbg_bitmap, H->dbg_scores);
+  k_flag_stats<<<n, 256, 0, s>>>(bitmap, h / 32, H->counters);
+  const size_t cnt = size_t(n) * d;
+  k_init_yacc<<<unsigned((cnt + 255) / 256), 256, 0, s>>>(yacc, H->bf, n, d);
+  int ksplit = n <= 8 ? 16 : 1;
+  int kchunk = ((d + ksplit - 1) / ksplit + 127) / 128 * 128;
+  ksplit = (d + kchunk - 1) / kchunk;
+  k_folded_product<T, Acc><<<dim3((d + 255) / 256, (n + 7) / 8, ksplit), 256, 0, s>>>(
+      static_cast<const T*>(H->C), x, yacc, n, d, kchunk);
+  k_fix<T, Acc><<<dim3(n, (h + 1023) / 1024), 256, size_t(d) * sizeof(float), s>>>(
+      static_cast<const T*>(H->W1), static_cast<const T*>(H->W2T), H->b1, H->a, H->c, x, bitmap, yacc, d, h, H->act);
+  k_store_y<T><<<unsigned((cnt + 255) / 256), 256, 0, s>>>(yacc, y, cnt);
+  H->launches += 6;
+  TARDIS_CUDA_TRY(cudaGetLastError());
+  return TARDIS_OK;
+}
+
+size_t static_forward_scratch_bytes(const Handle* H, int64_t n) {
+  const size_t acc = (size_t(n) * H->d * sizeof(float) + 255) / 256 * 256;
+  const size_t bm = (size_t(n) * (H->h / 32) * sizeof(uint32_t) + 255) / 256 * 256;
+  return acc + bm;
+}
+
+tardis_status_t launch_static_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s) {
+  if (size_t(H->d) * sizeof(float) > 48 * 1024) return TARDIS_ERR_UNSUPPORTED;
+  if (n > kStaticMaxTokens || static_forward_scratch_bytes(H, n) > kStaticScratchBytes) return TARDIS_ERR_UNSUPPORTED;
+  int cur = -1;
+  TARDIS_CUDA_TRY(cudaGetDevice(&cur));
+  if (cur != H->device) return TARDIS_ERR_INVALID_ARG;
+  unsigned char* base = nullptr;
+  tardis_status_t st = static_scratch_address(cur, &base);
+  if (st != TARDIS_OK) return st;
+  // Both regions are written in full by the first kernels that touch them (the bitmap by the predictor,
+  // the accumulator by its initialisation with b_f), so nothing of an earlier call's contents is read.
+  float* yacc = reinterpret_cast<float*>(base);
+  uint32_t* bitmap = reinterpret_cast<uint32_t*>(base + (size_t(n) * H->d * sizeof(float) + 255) / 256 * 256);
+  if (H->dtype == TARDIS_F32)
+    return static_typed<float, double>(H, static_cast<const float*>(x), static_cast<float*>(y), int(n), yacc, bitmap, s);
+  return static_typed<__nv_bfloat16, float>(H, static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), int(n), yacc, bitmap, s);
+}
+
 tardis_status_t launch_generic_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s) {
   if (size_t(H->d) * sizeof(float) > 48 * 1024) return TARDIS_ERR_UNSUPPORTED;
   if (H->dtype == TARDIS_F32)
