@@ -359,3 +359,233 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   for (int m = 0; m < VPT; ++m)
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[m][i] = 0.f;
+
+  // ---- speculative folded product: row chunks of C drawn from this column range's ticket ----
+  // stream_c(n) takes at most n chunks (two in flight per thread); the ticket for a chunk is drawn one
+  // step before the chunk is needed so that the atomic's latency is covered by the loads in flight.
+  auto stream_c = [&](int budget) {
+    constexpr int TK = LOADS / VPT;   // rows per chunk
+    unsigned int* ticket = p.ctl + CTL_TICKET + warp * 32;
+    auto issue = [&]() -> unsigned int {
+      unsigned int t = 0;
+      if (lane == 0) t = atomicAdd(ticket, 1u);
+      return t;
+    };
+    auto resolve = [&](unsigned int raw) -> int {
+      const unsigned int t = __shfl_sync(0xffffffffu, raw, 0);
+      return t < (unsigned int)p.ntk ? int(t) : -1;
+    };
+    auto load = [&](uint4 (&buf)[TK][VPT], int tk) {
+#pragma unroll
+      for (int r = 0; r < TK; ++r) {
+        const int k = tk * TK + r;
+#pragma unroll
+        for (int m = 0; m < VPT; ++m)
+          buf[r][m] = (k < d && cval[m]) ? ldg_stream(p.C + size_t(k) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
+      }
+    };
+    auto consume = [&](const uint4 (&buf)[TK][VPT], int tk) {
+#pragma unroll
+      for (int r = 0; r < TK; ++r) {
+        const int k = tk * TK + r;
+        const float sc = k < d ? __bfloat162float(xh[k]) : 0.f;
+#pragma unroll
+        for (int m = 0; m < VPT; ++m) fma8(acc[m], sc, buf[r][m]);
+      }
+    };
+    uint4 b0[TK][VPT], b1[TK][VPT];
+    int t0 = budget > 0 ? resolve(issue()) : -1;
+    int t1 = (t0 >= 0 && budget > 1) ? resolve(issue()) : -1;
+    budget -= 2;
+    if (t0 >= 0) load(b0, t0);
+    if (t1 >= 0) load(b1, t1);
+    bool more = t1 >= 0 && budget > 0;
+    while (t0 >= 0) {
+      unsigned int raw = more ? issue() : 0xffffffffu;
+      consume(b0, t0);
+      t0 = more ? resolve(raw) : -1;
+      --budget;
+      more = t0 >= 0 && budget > 0;
+      if (t0 >= 0) load(b0, t0);
+      if (t1 < 0) break;
+      raw = more ? issue() : 0xffffffffu;
+      consume(b1, t1);
+      t1 = more ? resolve(raw) : -1;
+      --budget;
+      more = t1 >= 0 && budget > 0;
+      if (t1 >= 0) load(b1, t1);
+    }
+  };
+
+  // CTAs of the second half of the grid (the ones that share an SM with a CTA of the first half) take a
+  // first share of the folded product before their predictor, so that the two CTAs of an SM are not in
+  // their memory-idle phases (scores, flags, compaction) at the same time.
+  if (blockIdx.x >= (gridDim.x >> 1) && p.pre_chunks > 0) stream_c(p.pre_chunks);
+
+  // ---- predictor: warp w takes chunk w of every unit; partial scores of a tile go to shared memory ----
+  {
+    double zacc[4] = {0.0, 0.0, 0.0, 0.0}, zt[2] = {0.0, 0.0};
+    const int kb_per_group = p.G / 64;                       // 1, 2 or 4
+    const int kbg_log2 = kb_per_group >> 1;                  // log2 of it
+    for (int u = 0; u < NU; ++u) {
+      const int b = u % p.nbuf;
+      const uint32_t par = uint32_t(u / p.nbuf) & 1u;
+      bool landed = mbar_wait(&full[b], par);
+      if (!landed) {                                 // record, give the copy one more bounded wait, skip the work
+        if (lane == 0) { atomicExch(&p.counters[CTR_ERROR], 1ull); misc[MS_ERR] = 1; }
+        landed = mbar_wait(&full[b], par);
+      }
+      const int tl = u / p.nranges, r = u - tl * p.nranges;
+      const int nch = min(p.cpr, p.nkc - r * p.cpr);
+      if (warp < nch && landed && !misc[MS_ERR]) {
+        const int kc = r * p.cpr + warp;
+        const uint8_t* blk = pbuf + size_t(b) * p.unit_bytes + size_t(warp) * p.pbs;
+        const uint4* cp = reinterpret_cast<const uint4*>(blk);
+        const uint2* mp = reinterpret_cast<const uint2*>(blk + 1024);
+        int ia[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int pair = 0; pair < 2; ++pair) {
+          const uint4 cw = cp[pair * 32 + lane];
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int kbl = pair * 2 + half;              // 64-channel block inside the 256-channel chunk
+            const int kb = kc * 4 + kbl;
+            const uint32_t A = half ? cw.z : cw.x, B = half ? cw.w : cw.y;
+            uint4 xb = make_uint4(0u, 0u, 0u, 0u);
+            if (g < 4) xb = *reinterpret_cast<const uint4*>(xq + size_t(g) * xq_stride + size_t(kb) * 64 + t4 * 16);
+            mma_u8s8(ia, A & 0x03030303u, B & 0x03030303u, A & 0x0C0C0C0Cu, B & 0x0C0C0C0Cu, xb.x, xb.y);
+            mma_u8s8(ia, A & 0x30303030u, B & 0x30303030u, A & 0xC0C0C0C0u, B & 0xC0C0C0C0u, xb.z, xb.w);
+            if (((kbl + 1) & (kb_per_group - 1)) == 0) {
+              const int gl = kbl >> kbg_log2;             // group inside the chunk
+              const uint2 mw = mp[gl * 8 + g];
+              const double s0 = bf16hi_to_double(mw.x), s1 = bf16hi_to_double(mw.y);
+              zacc[0] += s0 * int_to_double(ia[0]); zacc[1] += s0 * int_to_double(ia[1]);
+              zacc[2] += s1 * int_to_double(ia[2]); zacc[3] += s1 * int_to_double(ia[3]);
+              const double sx = sxd[min(kb >> kbg_log2, p.ngroups - 1)];
+              zt[0] += s0 * int_to_double(int(mw.x & 3u)) * sx;
+              zt[1] += s1 * int_to_double(int(mw.y & 3u)) * sx;
+              ia[0] = ia[1] = ia[2] = ia[3] = 0;
+            }
+          }
+        }
+      }
+      if (r == p.nranges - 1) {
+        // limbs: lane t4 = 0 holds limbs 0,1 ; t4 = 1 holds limbs 2,3 (columns 4..7 are unused for one token)
+        double v0 = 0.0, v1 = 0.0;
+        if (t4 == 0) { v0 = zacc[0] + 256.0 * zacc[1]; v1 = zacc[2] + 256.0 * zacc[3]; }
+        if (t4 == 1) { v0 = 65536.0 * (zacc[0] + 256.0 * zacc[1]); v1 = 65536.0 * (zacc[2] + 256.0 * zacc[3]); }
+        v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
+        v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+        if (t4 == 0) {
+          zpart[(tl * NW + warp) * 16 + g] = v0 * (1.0 / 64.0) - zt[0];
+          zpart[(tl * NW + warp) * 16 + g + 8] = v1 * (1.0 / 64.0) - zt[1];
+        }
+        zacc[0] = zacc[1] = zacc[2] = zacc[3] = 0.0; zt[0] = zt[1] = 0.0;
+      }
+      // hand the buffer back: the last warp to leave it starts the copy of the unit that reuses it
+      if (u + p.nbuf < NU) {
+        __threadfence_block();
+        __syncwarp();
+        if (lane == 0) {
+          const int old = atomicAdd(const_cast<int*>(&misc[MS_BUFCNT + b]), 1);
+          if (old == NW - 1) {
+            misc[MS_BUFCNT + b] = 0;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue_unit(u + p.nbuf);
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- scores, flags ----
+  const int nrow = plan.y * 16;
+  if (tid < nrow) {
+    const int tl = tid >> 4, r = tid & 15;
+    const int j = (plan.x + tl) * 16 + r;
+    double s = 0.0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) s += zpart[(tl * NW + w) * 16 + r];
+    const double zhat = double(tab[2 * TR + tid]) + ldexp(s, E);
+    const double lo = double(tab[tid]), hi = double(tab[TR + tid]);
+    int f = ((lo <= zhat) && (zhat < hi)) ? 0 : 1;
+    if (tok_nonfinite) f = 1;
+    else if (tau > 0.0 && (fabs(zhat - lo) <= tau || fabs(zhat - hi) <= tau)) {
+      const int q = atomicAdd(const_cast<int*>(&misc[MS_NRC]), 1);
+      if (q < MAXRC) rc[q] = tid;
+      else {                                        // list full: this thread re-evaluates its neuron alone
+        const int nwords = d / 16;
+        double a64 = 0.0;
+        for (int w = 0; w < nwords; ++w) {
+          const uint32_t word = p.codes[size_t(j) * nwords + w];
+          const int grp = (w * 16) / p.G;
+          const double zp = double(p.zero[size_t(j) * p.ngroups + grp]);
+          double inner = 0.0;
+          for (int q2 = 0; q2 < 16; ++q2) inner += (double((word >> (2 * q2)) & 3u) - zp) * double(__bfloat162float(xh[w * 16 + q2]));
+          a64 += double(__bfloat162float(p.scale[size_t(j) * p.ngroups + grp])) * inner;
+        }
+        const double z2 = a64 + double(tab[2 * TR + tid]);
+        f = ((lo <= z2) && (z2 < hi)) ? 0 : 1;
+        score[tid] = z2;
+        flagbits[tid] = f;
+        f |= 4;
+      }
+    }
+    if (!(f & 4)) {
+      flagbits[tid] = f;
+      score[tid] = tok_nonfinite ? __longlong_as_double(0x7ff8000000000000ll) : zhat;
+    }
+  }
+  __syncthreads();
+  // exact re-evaluation from the original codes (rare): one warp per listed neuron
+  {
+    const int nrc = min(int(misc[MS_NRC]), MAXRC);
+    const int nwords = d / 16;
+    for (int e = warp; e < nrc; e += NW) {
+      const int n = rc[e];
+      const int j = (plan.x + (n >> 4)) * 16 + (n & 15);
+      double a64 = 0.0;
+      for (int w = lane; w < nwords; w += 32) {
+        const uint32_t word = p.codes[size_t(j) * nwords + w];
+        const int grp = (w * 16) / p.G;
+        const double zp = double(p.zero[size_t(j) * p.ngroups + grp]);
+        double inner = 0.0;
+#pragma unroll
+        for (int q = 0; q < 16; ++q) inner += (double((word >> (2 * q)) & 3u) - zp) * double(__bfloat162float(xh[w * 16 + q]));
+        a64 += double(__bfloat162float(p.scale[size_t(j) * p.ngroups + grp])) * inner;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a64 += __shfl_xor_sync(0xffffffffu, a64, o);
+      if (lane == 0) {
+        const double zhat = a64 + double(tab[2 * TR + n]);
+        flagbits[n] = ((double(tab[n]) <= zhat) && (zhat < double(tab[TR + n]))) ? 0 : 1;
+        score[n] = zhat;
+      }
+    }
+    if (nrc > 0) {
+      if (tid == 0) atomicAdd(&p.counters[CTR_RECHECKS], (unsigned long long)nrc);
+      __syncthreads();
+    }
+  }
+  // ---- ascending flagged list: ballot + prefix over the (at most 8) warps that hold rows ----
+  {
+    const int f = (tid < nrow) ? (flagbits[tid] & 1) : 0;
+    const uint32_t bal = __ballot_sync(0xffffffffu, f != 0);
+    if (lane == 0) misc[MS_WCNT + warp] = __popc(bal);
+    __syncthreads();
+    int base = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { const int cnt = misc[MS_WCNT + w]; if (w < warp) base += cnt; total += cnt; }
+    if (f) fl_j[base + __popc(bal & ((1u << lane) - 1u))] = (plan.x + (tid >> 4)) * 16 + (tid & 15);
+    if (tid == 0) {
+      misc[MS_NFL] = total;
+      if (total) atomicAdd(&p.ctl[CTL_NFL], (unsigned int)total);   // read by the warp that finishes column range 0
+    }
+    // debug capture: 16-bit halves of the flag words, scores
+    if (p.dbg_bitmap && tid < nrow && (tid & 15) == 0)
+      reinterpret_cast<uint16_t*>(p.dbg_bitmap)[plan.x + (tid >> 4)] = uint16_t((bal >> (lane & 16)) & 0xffffu);
+    if (p.dbg_scores && tid < nrow) p.dbg_scores[(plan.x + (tid >> 4)) * 16 + (tid & 15)] = score[tid];
+  }
+  __syncthreads();
+  const int nfl = misc[MS_NFL];
