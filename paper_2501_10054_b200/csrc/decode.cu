@@ -589,3 +589,166 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   }
   __syncthreads();
   const int nfl = misc[MS_NFL];
+
+  constexpr int FB = FIXLOADS / VPT;   // flagged rows per batch
+  uint4 w[FB][VPT];
+
+  // ---- result fixing, first half: W1 rows -> z_j -> delta_j ----
+  if (nfl > 0) {
+    float xr[VPT][8];
+#pragma unroll
+    for (int m = 0; m < VPT; ++m) unpack8(xr[m], *reinterpret_cast<const uint4*>(xh + col[m]));
+    for (int e0 = 0; e0 < nfl; e0 += FB) {
+#pragma unroll
+      for (int r = 0; r < FB; ++r) {
+        const int j = (e0 + r < nfl) ? fl_j[e0 + r] : -1;
+#pragma unroll
+        for (int m = 0; m < VPT; ++m)
+          w[r][m] = (j >= 0 && cval[m]) ? ldg_stream(p.W1 + size_t(j) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
+      }
+      float part[FB];
+#pragma unroll
+      for (int r = 0; r < FB; ++r) {
+        part[r] = 0.f;
+#pragma unroll
+        for (int m = 0; m < VPT; ++m) part[r] += dot8(w[r][m], xr[m]);
+      }
+      // the W2T rows of the first batch go in flight while the last dot products meet
+      if (e0 + FB >= nfl) {
+#pragma unroll
+        for (int r = 0; r < FB; ++r) {
+          const int j = (r < nfl) ? fl_j[r] : -1;
+#pragma unroll
+          for (int m = 0; m < VPT; ++m)
+            w[r][m] = (j >= 0 && cval[m]) ? ldg_stream(p.W2T + size_t(j) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < FB; ++r) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part[r] += __shfl_xor_sync(0xffffffffu, part[r], o);
+        if (lane == 0) wpart[r * NW + warp] = part[r];
+      }
+      __syncthreads();
+      if (tid < FB && e0 + tid < nfl) {
+        const int row = fl_j[e0 + tid] - plan.x * 16;
+        float z = 0.f;
+#pragma unroll
+        for (int ww = 0; ww < NW; ++ww) z += wpart[tid * NW + ww];
+        z += tab[2 * TR + row];
+        fl_delta[e0 + tid] = gelu_f32(z, p.act) - tab[3 * TR + row] * z - tab[4 * TR + row];
+      }
+      __syncthreads();
+    }
+  }
+
+  // ---- result fixing, second half: W2T rows scaled by delta_j ----
+  for (int e0 = 0; e0 < nfl; e0 += FB) {
+    if (e0 > 0) {
+#pragma unroll
+      for (int r = 0; r < FB; ++r) {
+        const int j = (e0 + r < nfl) ? fl_j[e0 + r] : -1;
+#pragma unroll
+        for (int m = 0; m < VPT; ++m)
+          w[r][m] = (j >= 0 && cval[m]) ? ldg_stream(p.W2T + size_t(j) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < FB; ++r) {
+      const float dl = (e0 + r < nfl) ? fl_delta[e0 + r] : 0.f;
+#pragma unroll
+      for (int m = 0; m < VPT; ++m) fma8(acc[m], dl, w[r][m]);
+    }
+  }
+
+  // ---- the rest of the folded product ----
+  stream_c(0x7fffffff);
+
+  // ---- combine: add this warp's columns to one replica; the last warp on a column range finishes it ----
+  {
+    float* rep = p.yacc + size_t(blockIdx.x % NREP) * p.dacc;
+#pragma unroll
+    for (int m = 0; m < VPT; ++m)
+      if (cval[m]) {
+        red_add_v4(rep + col[m], acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
+        red_add_v4(rep + col[m] + 4, acc[m][4], acc[m][5], acc[m][6], acc[m][7]);
+      }
+  }
+  __threadfence();
+  __syncwarp();
+  unsigned int arrived = 0;
+  if (lane == 0) arrived = atomicAdd(&p.ctl[CTL_DONE + warp * 32], 1u);
+  arrived = __shfl_sync(0xffffffffu, arrived, 0);
+  if (arrived == gridDim.x - 1) {
+    __threadfence();
+#pragma unroll
+    for (int m = 0; m < VPT; ++m)
+      if (cval[m]) {
+        float4 s0 = *reinterpret_cast<const float4*>(p.bf + col[m]);
+        float4 s1 = *reinterpret_cast<const float4*>(p.bf + col[m] + 4);
+#pragma unroll 4
+        for (int rp = 0; rp < NREP; ++rp) {
+          float* q = p.yacc + size_t(rp) * p.dacc + col[m];
+          const float4 a0 = __ldcg(reinterpret_cast<const float4*>(q));
+          const float4 a1 = __ldcg(reinterpret_cast<const float4*>(q + 4));
+          s0.x += a0.x; s0.y += a0.y; s0.z += a0.z; s0.w += a0.w;
+          s1.x += a1.x; s1.y += a1.y; s1.z += a1.z; s1.w += a1.w;
+          *reinterpret_cast<float4*>(q) = make_float4(0.f, 0.f, 0.f, 0.f);
+          *reinterpret_cast<float4*>(q + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        __nv_bfloat162 o[4];
+        o[0] = __floats2bfloat162_rn(s0.x, s0.y);
+        o[1] = __floats2bfloat162_rn(s0.z, s0.w);
+        o[2] = __floats2bfloat162_rn(s1.x, s1.y);
+        o[3] = __floats2bfloat162_rn(s1.z, s1.w);
+        *reinterpret_cast<uint4*>(p.y + col[m]) = *reinterpret_cast<const uint4*>(o);
+      }
+    if (lane == 0) {
+      p.ctl[CTL_TICKET + warp * 32] = 0u;
+      p.ctl[CTL_DONE + warp * 32] = 0u;
+      if (warp == 0) {   // every CTA's warp 0 has arrived, so every CTA's flagged count is in
+        const unsigned int tot = atomicExch(&p.ctl[CTL_NFL], 0u);
+        atomicAdd(&p.counters[CTR_FLAGGED_TOTAL], (unsigned long long)tot);
+        atomicMax(&p.counters[CTR_FLAGGED_MAX], (unsigned long long)tot);
+      }
+    }
+  }
+}
+
+// ---- set-up kernels --------------------------------------------------------------------------------------
+// Predictor blocks: block (tile, kc) = 2 x 32 lanes x {A0,B0,A1,B1} code words + per-group {row g, row g+8} metadata.
+__global__ void k_pack_pblocks(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
+                               const uint8_t* __restrict__ zero, uint8_t* __restrict__ out, int d, int G,
+                               int nkc, int pbs) {
+  const int tile = blockIdx.x, kc = blockIdx.y;
+  uint8_t* blk = out + (size_t(tile) * nkc + kc) * pbs;
+  const int nwords = d / 16, ng = d / G;
+  for (int e = threadIdx.x; e < 256; e += blockDim.x) {        // 256 code words
+    const int pair = e >> 7, ln = (e >> 2) & 31, sub = e & 3;   // sub: 0 A(half0) 1 B(half0) 2 A(half1) 3 B(half1)
+    const int gg = ln >> 2, tt = ln & 3;
+    const int row = tile * 16 + gg + ((sub & 1) ? 8 : 0);
+    const int kbl = pair * 2 + (sub >> 1);
+    const int word = (kc * 4 + kbl) * 4 + tt;
+    reinterpret_cast<uint32_t*>(blk)[e] = (word < nwords) ? codes[size_t(row) * nwords + word] : 0u;
+  }
+  const int gpc = KC / G;
+  for (int e = threadIdx.x; e < gpc * 16; e += blockDim.x) {
+    const int gl = e >> 4, gg = (e >> 1) & 7, hi = e & 1;
+    const int row = tile * 16 + gg + (hi ? 8 : 0);
+    const int grp = kc * gpc + gl;
+    uint32_t w = 0u;
+    if (grp < ng) w = (uint32_t(__bfloat16_as_ushort(scale[size_t(row) * ng + grp])) << 16) | uint32_t(zero[size_t(row) * ng + grp] & 3u);
+    reinterpret_cast<uint32_t*>(blk + 1024)[e] = w;
+  }
+}
+
+__global__ void k_max_scale(const __nv_bfloat16* __restrict__ scale, size_t count, float* out) {
+  float m = 0.f;
+  for (size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x; e < count; e += size_t(gridDim.x) * blockDim.x)
+    m = fmaxf(m, fabsf(__bfloat162float(scale[e])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) atomicMax(reinterpret_cast<int*>(out), __float_as_int(m));
+}
+
+}  // namespace dec
