@@ -752,3 +752,136 @@ __global__ void k_max_scale(const __nv_bfloat16* __restrict__ scale, size_t coun
 }
 
 }  // namespace dec
+
+using namespace dec;
+
+tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
+  H->dscratch = nullptr;
+  H->codes_mma = nullptr;
+  const int d = H->d, h = H->h, G = H->G;
+  if (H->dtype != TARDIS_BF16) return TARDIS_OK;
+  if (!(G == 64 || G == 128 || G == 256)) return TARDIS_OK;         // generic kernels serve other group sizes
+  const int NT = h / 16;
+  const int nvec = d / 8;
+  const int cw = (nvec + NW - 1) / NW;
+  const int vpt = (cw + 31) / 32;
+  const int dpad = (d + KC - 1) / KC * KC;
+  if (vpt > 2 || d < 64 || dpad > XVR * NTH * 8) return TARDIS_OK;
+  int max_smem = 0, sm_smem = 0;
+  TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, H->device));
+  TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, H->device));
+
+  Scratch* S = new (std::nothrow) Scratch();
+  if (!S) return TARDIS_ERR_ALLOC;
+  memset(S, 0, sizeof(*S));
+  Params& p = S->base;
+  p.d = d; p.h = h; p.G = G; p.ngroups = H->ngroups; p.act = H->act;
+  p.dpad = dpad; p.dacc = (d + 31) / 32 * 32;
+  p.nkc = dpad / KC;
+  p.pbs = 1024 + 64 * (KC / G);
+  p.nranges = (p.nkc + NW - 1) / NW;
+  p.cpr = (p.nkc + p.nranges - 1) / p.nranges;
+  p.unit_bytes = p.cpr * p.pbs;
+  p.nvec = nvec; p.cw = cw;
+  const int tk_rows = LOADS / vpt;
+  p.ntk = (d + tk_rows - 1) / tk_rows;
+  p.pre_chunks = 2;
+  S->vpt = vpt;
+  // two CTAs per SM when their shared memory fits (each CTA also reserves 1 KB), else one
+  bool placed = false;
+  for (int per_sm = 2; per_sm >= 1 && !placed; --per_sm) {
+    const int grid = H->num_sms * per_sm;
+    const int tiles_max = (NT + grid - 1) / grid;
+    if (tiles_max > MAXTILES) continue;
+    const int units = tiles_max * p.nranges;
+    const size_t budget = per_sm == 2 ? size_t(sm_smem) / 2 - 1024 : size_t(max_smem);
+    const int nbuf_hi = units < MAXBUF ? units : MAXBUF;
+    const int nbuf_lo = units < 2 ? units : 2;
+    for (int nbuf = nbuf_hi; nbuf >= nbuf_lo && nbuf >= 1; --nbuf) {
+      const size_t need = SmemLayout(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes).total;
+      if (need <= budget && need <= size_t(max_smem)) {
+        S->grid = grid; p.tiles_max = tiles_max; p.nbuf = nbuf; S->smem_bytes = need;
+        placed = true;
+        break;
+      }
+    }
+  }
+  if (!placed) { delete S; return TARDIS_OK; }
+  const int grid = S->grid;
+  if (grid == H->num_sms) p.pre_chunks = 0;      // one CTA per SM: nothing to stagger
+
+  auto fail = [&](tardis_status_t st) { H->dscratch = S; decode_release(H); return st; };
+  size_t tally = 0;
+  const size_t pb_bytes = size_t(NT) * p.nkc * p.pbs;
+  const size_t yacc_bytes = sizeof(float) * NREP * p.dacc;
+  cudaError_t e = cudaMalloc(&S->pblocks, pb_bytes); tally += pb_bytes;
+  if (e == cudaSuccess) { e = cudaMalloc(&S->plan, sizeof(int2) * grid); tally += sizeof(int2) * grid; }
+  if (e == cudaSuccess) { e = cudaMalloc(&S->smax, 16); tally += 16; }
+  if (e == cudaSuccess) { e = cudaMalloc(&S->yacc, yacc_bytes); tally += yacc_bytes; }
+  if (e == cudaSuccess) { e = cudaMalloc(&S->ctl, sizeof(unsigned int) * CTL_WORDS); tally += sizeof(unsigned int) * CTL_WORDS; }
+  if (e != cudaSuccess) { set_last_error(e, "cudaMalloc"); cudaGetLastError(); return fail(TARDIS_ERR_ALLOC); }
+  S->bytes = tally;
+
+  // tiles spread evenly over the CTAs
+  std::vector<int2> plan(grid);
+  int tile_cum = 0;
+  for (int c = 0; c < grid; ++c) {
+    const int tc = NT / grid + (c < NT % grid ? 1 : 0);
+    plan[c] = make_int2(tile_cum, tc);
+    tile_cum += tc;
+  }
+  e = cudaMemcpyAsync(S->plan, plan.data(), sizeof(int2) * grid, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);   // plan.data() is a stack-owned host buffer
+  if (e == cudaSuccess) e = cudaMemsetAsync(S->smax, 0, 16, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(S->yacc, 0, yacc_bytes, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(S->ctl, 0, sizeof(unsigned int) * CTL_WORDS, s);
+  if (e != cudaSuccess) { set_last_error(e, "decode_prepare"); return fail(TARDIS_ERR_CUDA); }
+  k_pack_pblocks<<<dim3(NT, p.nkc), 128, 0, s>>>(H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero,
+                                                 S->pblocks, d, G, p.nkc, p.pbs);
+  k_max_scale<<<64, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->scale), size_t(h) * H->ngroups, S->smax);
+  e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+  if (e != cudaSuccess) { set_last_error(e, "decode_prepare launch"); return fail(TARDIS_ERR_CUDA); }
+
+  p.pblocks = S->pblocks; p.plan = S->plan; p.smax = S->smax; p.yacc = S->yacc; p.ctl = S->ctl;
+  p.W1 = static_cast<const __nv_bfloat16*>(H->W1); p.W2T = static_cast<const __nv_bfloat16*>(H->W2T);
+  p.C = static_cast<const __nv_bfloat16*>(H->C); p.bf = H->bf; p.lo = H->lo; p.hi = H->hi; p.a = H->a; p.c = H->c; p.b1 = H->b1;
+  p.codes = H->codes; p.scale = static_cast<const __nv_bfloat16*>(H->scale); p.zero = H->zero;
+  p.counters = H->counters;
+  H->dscratch = S;
+  H->dscratch_bytes = S->bytes;
+  H->bytes_scratch += S->bytes - pb_bytes;
+  H->bytes_predictor += pb_bytes;
+  H->codes_mma = reinterpret_cast<uint32_t*>(S->pblocks);
+  return TARDIS_OK;
+}
+
+tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s) {
+  Scratch* S = static_cast<Scratch*>(H->dscratch);
+  for (int t = 0; t < n; ++t) {
+    Params p = S->base;
+    p.x = static_cast<const __nv_bfloat16*>(x) + size_t(t) * H->d;
+    p.y = static_cast<__nv_bfloat16*>(y) + size_t(t) * H->d;
+    p.dbg_bitmap = H->dbg_bitmap ? H->dbg_bitmap + size_t(t) * (H->h / 32) : nullptr;
+    p.dbg_scores = H->dbg_scores ? H->dbg_scores + size_t(t) * H->h : nullptr;
+    if (S->vpt == 1) k_decode<1><<<S->grid, NTH, S->smem_bytes, s>>>(p);
+    else k_decode<2><<<S->grid, NTH, S->smem_bytes, s>>>(p);
+    H->launches += 1;
+  }
+  TARDIS_CUDA_TRY(cudaGetLastError());
+  return TARDIS_OK;
+}
+
+void decode_release(Handle* H) {
+  Scratch* S = static_cast<Scratch*>(H->dscratch);
+  if (!S) return;
+  void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl};
+  for (void* q : ptrs)
+    if (q) cudaFree(q);
+  delete S;
+  H->dscratch = nullptr;
+  H->codes_mma = nullptr;
+}
+
+}  // namespace tardis
