@@ -43,7 +43,7 @@ constexpr int MAXRC = 64;         // exact re-checks per CTA before the list ove
 constexpr int LOADS = 4;          // 128-bit loads per thread and folded-matrix chunk (rows x slots)
 constexpr int FIXLOADS = 8;       // 128-bit loads per thread and batch of flagged rows (rows x slots)
 constexpr int MAXBUF = 8;         // predictor unit buffers in shared memory
-constexpr int NREP = 8;           // replicas of the output accumulator
+constexpr int NREP = 4;           // replicas of the output accumulator
 constexpr int XVR = 2;            // 8-channel vectors of x per thread (padded d <= 8192)
 constexpr uint32_t SPIN_LIMIT = 1u << 21;   // spaced polls of a bounded mbarrier wait: a fraction of a second
 // control words (unsigned int) in global scratch; all zero between calls
@@ -214,6 +214,22 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     bulk_g2s(pbuf + size_t(b) * p.unit_bytes, p.pblocks + (size_t(plan.x + tl) * p.nkc + size_t(r) * p.cpr) * p.pbs, bytes, &full[b]);
   };
 
+  // x first: it heads the longest dependency chain of the kernel, so its loads go out before the
+  // predictor copies fill the memory queues
+  uint4 xw[XVR];
+#pragma unroll
+  for (int m = 0; m < XVR; ++m) {
+    const int v = tid + m * NTH;
+    xw[m] = make_uint4(0u, 0u, 0u, 0u);
+    if (v < p.nvec) xw[m] = *reinterpret_cast<const uint4*>(p.x + size_t(v) * 8);
+  }
+  // per-neuron tables of the CTA's rows
+  float tl0 = 0.f, tl1 = 0.f, tl2 = 0.f, tl3 = 0.f, tl4 = 0.f;
+  if (tid < plan.y * 16) {
+    const int j = plan.x * 16 + tid;
+    tl0 = p.lo[j]; tl1 = p.hi[j]; tl2 = p.b1[j]; tl3 = p.a[j]; tl4 = p.c[j];
+  }
+
   if (tid == 0) {
     for (int b = 0; b < p.nbuf; ++b) mbar_init(&full[b], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -223,23 +239,17 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   // predictor blocks first: nothing of them depends on x
   if (lane == 0 && warp < p.nbuf && warp < NU) issue_unit(warp);
 
-  // per-neuron tables of the CTA's rows (their latency also hides behind the x preparation)
   if (tid < plan.y * 16) {
-    const int j = plan.x * 16 + tid;
-    tab[tid] = p.lo[j]; tab[TR + tid] = p.hi[j]; tab[2 * TR + tid] = p.b1[j];
-    tab[3 * TR + tid] = p.a[j]; tab[4 * TR + tid] = p.c[j];
+    tab[tid] = tl0; tab[TR + tid] = tl1; tab[2 * TR + tid] = tl2; tab[3 * TR + tid] = tl3; tab[4 * TR + tid] = tl4;
   }
 
   // ---- x: registers, bf16 copy in shared memory, max |x| ----
-  uint4 xw[XVR];
   {
     float amax = 0.f;
     bool nonfinite = false;
 #pragma unroll
     for (int m = 0; m < XVR; ++m) {
       const int v = tid + m * NTH;
-      xw[m] = make_uint4(0u, 0u, 0u, 0u);
-      if (v < p.nvec) xw[m] = *reinterpret_cast<const uint4*>(p.x + size_t(v) * 8);
       if (v * 8 < p.dpad) *reinterpret_cast<uint4*>(xh + v * 8) = xw[m];
       float f[8];
       unpack8(f, xw[m]);
@@ -684,15 +694,21 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
 #pragma unroll
     for (int m = 0; m < VPT; ++m)
       if (cval[m]) {
-        float4 s0 = *reinterpret_cast<const float4*>(p.bf + col[m]);
-        float4 s1 = *reinterpret_cast<const float4*>(p.bf + col[m] + 4);
-#pragma unroll 4
+        float4 a0[NREP + 1], a1[NREP + 1];
+        a0[NREP] = *reinterpret_cast<const float4*>(p.bf + col[m]);
+        a1[NREP] = *reinterpret_cast<const float4*>(p.bf + col[m] + 4);
+#pragma unroll
         for (int rp = 0; rp < NREP; ++rp) {
+          const float* q = p.yacc + size_t(rp) * p.dacc + col[m];
+          a0[rp] = __ldcg(reinterpret_cast<const float4*>(q));
+          a1[rp] = __ldcg(reinterpret_cast<const float4*>(q + 4));
+        }
+        float4 s0 = a0[NREP], s1 = a1[NREP];
+#pragma unroll
+        for (int rp = 0; rp < NREP; ++rp) {
+          s0.x += a0[rp].x; s0.y += a0[rp].y; s0.z += a0[rp].z; s0.w += a0[rp].w;
+          s1.x += a1[rp].x; s1.y += a1[rp].y; s1.z += a1[rp].z; s1.w += a1[rp].w;
           float* q = p.yacc + size_t(rp) * p.dacc + col[m];
-          const float4 a0 = __ldcg(reinterpret_cast<const float4*>(q));
-          const float4 a1 = __ldcg(reinterpret_cast<const float4*>(q + 4));
-          s0.x += a0.x; s0.y += a0.y; s0.z += a0.z; s0.w += a0.w;
-          s1.x += a1.x; s1.y += a1.y; s1.z += a1.z; s1.w += a1.w;
           *reinterpret_cast<float4*>(q) = make_float4(0.f, 0.f, 0.f, 0.f);
           *reinterpret_cast<float4*>(q + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
         }
