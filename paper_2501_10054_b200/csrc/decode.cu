@@ -9,10 +9,12 @@
 //     prepared.  The codes are evaluated on the integer tensor cores: they are masked straight
 //     out of the packed words (no shifts: the field position is a power-of-4 weight that the
 //     pre-scaling of x undoes) and multiplied with a 4-limb signed base-256 fixed-point copy of x
-//     (mma.m16n8k32.u8.s8, s32 accumulators, exact); group sums are scaled and accumulated in
-//     fp64, so the score equals the mathematical one up to the (tracked) truncation of tiny x
-//     elements; a score that close to a range end is re-evaluated exactly from the original
-//     codes.  The 16 warps split the channel chunks of a tile; partial scores meet in shared memory.
+//     (mma.m16n8k32.u8.s8, s32 accumulators, exact).  The bf16 group scales of a neuron are held as
+//     16-bit integers over one power of two per neuron, so group sums are scaled and accumulated in
+//     64-bit integers (exact) and the score equals the mathematical one up to the (tracked)
+//     truncation of tiny x elements and one fp64 rounding; a score that close to a range end is
+//     re-evaluated in fp64 from the original codes.  The 16 warps split the channel chunks of a
+//     tile; partial scores meet in shared memory.
 //   * Flags are compacted by ballot + prefix sum into the CTA's ascending list.
 //   * Every thread owns 8 output columns (per slot).  All remaining weight traffic is coalesced
 //     128-bit read-only loads kept several deep per thread.  For the CTA's flagged neurons a
@@ -43,6 +45,7 @@ constexpr int MAXRC = 64;         // exact re-checks per CTA before the list ove
 constexpr int LOADS = 4;          // 128-bit loads per thread and folded-matrix chunk (rows x slots)
 constexpr int FIXLOADS = 8;       // 128-bit loads per thread and batch of flagged rows (rows x slots)
 constexpr int MAXBUF = 8;         // predictor unit buffers in shared memory
+constexpr int kBadRow = 0x40000000;   // row whose group scales do not fit the integer form: always re-evaluated
 constexpr int NREP = 4;           // replicas of the output accumulator
 constexpr int XVR = 2;            // 8-channel vectors of x per thread (padded d <= 8192)
 constexpr uint32_t SPIN_LIMIT = 1u << 21;   // spaced polls of a bounded mbarrier wait: a fraction of a second
@@ -59,6 +62,7 @@ struct Params {
   const float *bf, *lo, *hi, *a, *c, *b1;
   const uint32_t* codes; const __nv_bfloat16* scale; const uint8_t* zero;   // originals (exact re-check)
   const float* smax;       // largest group scale of the layer
+  const int* rowexp;       // per neuron: power of two its integer group scales are expressed in (kBadRow: none)
   const int2* plan;        // per CTA: first tile, tile count
   const __nv_bfloat16* x; __nv_bfloat16* y;
   float* yacc;             // [NREP][dacc] fp32
@@ -74,7 +78,7 @@ struct Params {
 };
 
 struct Scratch {           // handle-owned device memory of the fused path
-  uint8_t* pblocks; int2* plan; float* smax; float* yacc; unsigned int* ctl;
+  uint8_t* pblocks; int2* plan; float* smax; float* yacc; unsigned int* ctl; int* rowexp;
   Params base; size_t smem_bytes; size_t bytes; int grid; int vpt;
 };
 
@@ -123,16 +127,6 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 }
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-// Exact conversions done with integer operations and fp64 adds only: the conversion unit is narrow and
-// the predictor loop would otherwise queue on it.
-__device__ __forceinline__ double int_to_double(int v) {          // (2^52 + 2^31 + v) - (2^52 + 2^31)
-  return __hiloint2double(0x43300000, int(uint32_t(v) ^ 0x80000000u)) - 4503601774854144.0;
-}
-__device__ __forceinline__ double bf16hi_to_double(uint32_t w) {  // bf16 in the upper 16 bits of w
-  const uint32_t e = (w >> 23) & 0xffu;
-  if (e == 0u || e == 255u) return double(__uint_as_float(w & 0xffff0000u));   // zero, subnormal, inf, nan: rare
-  return __hiloint2double(int((w & 0x80000000u) | ((e + 896u) << 20) | ((w >> 3) & 0x000fe000u)), 0);
-}
 __device__ __forceinline__ void unpack8(float (&f)[8], const uint4& w) {
   f[0] = bf_lo(w.x); f[1] = bf_hi(w.x); f[2] = bf_lo(w.y); f[3] = bf_hi(w.y);
   f[4] = bf_lo(w.z); f[5] = bf_hi(w.z); f[6] = bf_lo(w.w); f[7] = bf_hi(w.w);
@@ -150,7 +144,7 @@ __device__ __forceinline__ float dot8(const uint4& w, const float (&xv)[8]) {
 
 // ---- shared-memory carve-up (host and device agree through this) -----------------------------------
 struct SmemLayout {
-  size_t pbuf, xq, xh, sxd, zpart, wpart, score, tab, fl_j, fl_delta, rc, flagbits, wred, bars, misc, total;
+  size_t pbuf, xq, xh, sxi, zpart, wpart, score, tab, fl_j, fl_delta, rc, flagbits, wred, bars, misc, total;
   __host__ __device__ SmemLayout(int dpad, int ngroups, int tiles_max, int nbuf, int unit_bytes) {
     size_t o = 0;
     auto take = [&](size_t bytes, size_t align) { o = (o + align - 1) / align * align; size_t r = o; o += bytes; return r; };
@@ -158,11 +152,11 @@ struct SmemLayout {
     pbuf = take(size_t(nbuf) * unit_bytes, 128);
     xq = take(size_t(4) * (dpad + 64), 128);
     xh = take(size_t(dpad) * 2, 16);
-    sxd = take(size_t(ngroups + 16) * sizeof(double), 8);
+    sxi = take(size_t(ngroups + 16) * sizeof(int), 8);
     zpart = take(rows * NW * sizeof(double), 8);
     wpart = take(size_t(FIXLOADS) * NW * sizeof(float), 4);
     score = take(rows * sizeof(double), 8);
-    tab = take(5 * rows * sizeof(float), 4);
+    tab = take(6 * rows * sizeof(float), 4);
     fl_j = take(rows * sizeof(int), 4);
     fl_delta = take(rows * sizeof(float), 4);
     rc = take(MAXRC * sizeof(int), 4);
@@ -183,11 +177,11 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   uint8_t* pbuf = smem + L.pbuf;
   uint8_t* xq = smem + L.xq;
   __nv_bfloat16* xh = reinterpret_cast<__nv_bfloat16*>(smem + L.xh);
-  double* sxd = reinterpret_cast<double*>(smem + L.sxd);
+  int* sxi = reinterpret_cast<int*>(smem + L.sxi);
   double* zpart = reinterpret_cast<double*>(smem + L.zpart);
   float* wpart = reinterpret_cast<float*>(smem + L.wpart);
   double* score = reinterpret_cast<double*>(smem + L.score);
-  float* tab = reinterpret_cast<float*>(smem + L.tab);   // [5][TR]: lo, hi, b1, a, c of the CTA's neurons
+  float* tab = reinterpret_cast<float*>(smem + L.tab);   // [6][TR]: lo, hi, b1, a, c, scale exponent (int bits) of the CTA's neurons
   int* fl_j = reinterpret_cast<int*>(smem + L.fl_j);
   float* fl_delta = reinterpret_cast<float*>(smem + L.fl_delta);
   int* rc = reinterpret_cast<int*>(smem + L.rc);
@@ -225,9 +219,10 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   }
   // per-neuron tables of the CTA's rows
   float tl0 = 0.f, tl1 = 0.f, tl2 = 0.f, tl3 = 0.f, tl4 = 0.f;
+  int tl5 = 0;
   if (tid < plan.y * 16) {
     const int j = plan.x * 16 + tid;
-    tl0 = p.lo[j]; tl1 = p.hi[j]; tl2 = p.b1[j]; tl3 = p.a[j]; tl4 = p.c[j];
+    tl0 = p.lo[j]; tl1 = p.hi[j]; tl2 = p.b1[j]; tl3 = p.a[j]; tl4 = p.c[j]; tl5 = p.rowexp[j];
   }
 
   if (tid == 0) {
@@ -240,7 +235,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   if (lane == 0 && warp < p.nbuf && warp < NU) issue_unit(warp);
 
   if (tid < plan.y * 16) {
-    tab[tid] = tl0; tab[TR + tid] = tl1; tab[2 * TR + tid] = tl2; tab[3 * TR + tid] = tl3; tab[4 * TR + tid] = tl4;
+    tab[tid] = tl0; tab[TR + tid] = tl1; tab[2 * TR + tid] = tl2; tab[3 * TR + tid] = tl3; tab[4 * TR + tid] = tl4; tab[5 * TR + tid] = __int_as_float(tl5);
   }
 
   // ---- x: registers, bf16 copy in shared memory, max |x| ----
@@ -339,7 +334,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       }
       // group sums of the integer x (exact)
       for (int o = 1; o < lpg; o <<= 1) sx += __shfl_xor_sync(0xffffffffu, sx, o);
-      if (active && (lane & (lpg - 1)) == 0) sxd[(v * 8) >> g_log2] = int_to_double(sx);
+      if (active && (lane & (lpg - 1)) == 0) sxi[(v * 8) >> g_log2] = sx;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) resid += __shfl_xor_sync(0xffffffffu, resid, o);
@@ -434,8 +429,8 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
 
   // ---- predictor: warp w takes chunk w of every unit; partial scores of a tile go to shared memory ----
   {
-    double zacc[4] = {0.0, 0.0, 0.0, 0.0}, zt[2] = {0.0, 0.0};
-    const int kb_per_group = p.G / 64;                       // 1, 2 or 4
+    long long zacc[4] = {0, 0, 0, 0}, zt[2] = {0, 0};
+    const int kb_per_group = p.G / 64;                       // 1 or 2
     const int kbg_log2 = kb_per_group >> 1;                  // log2 of it
     for (int u = 0; u < NU; ++u) {
       const int b = u % p.nbuf;
@@ -466,14 +461,15 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
             mma_u8s8(ia, A & 0x03030303u, B & 0x03030303u, A & 0x0C0C0C0Cu, B & 0x0C0C0C0Cu, xb.x, xb.y);
             mma_u8s8(ia, A & 0x30303030u, B & 0x30303030u, A & 0xC0C0C0C0u, B & 0xC0C0C0C0u, xb.z, xb.w);
             if (((kbl + 1) & (kb_per_group - 1)) == 0) {
+              // group done: sums (|.| < 2^22) times the integer scales (|.| < 2^15), all exact
               const int gl = kbl >> kbg_log2;             // group inside the chunk
               const uint2 mw = mp[gl * 8 + g];
-              const double s0 = bf16hi_to_double(mw.x), s1 = bf16hi_to_double(mw.y);
-              zacc[0] += s0 * int_to_double(ia[0]); zacc[1] += s0 * int_to_double(ia[1]);
-              zacc[2] += s1 * int_to_double(ia[2]); zacc[3] += s1 * int_to_double(ia[3]);
-              const double sx = sxd[min(kb >> kbg_log2, p.ngroups - 1)];
-              zt[0] += s0 * int_to_double(int(mw.x & 3u)) * sx;
-              zt[1] += s1 * int_to_double(int(mw.y & 3u)) * sx;
+              const int m0 = int(mw.x) >> 16, m1 = int(mw.y) >> 16;
+              zacc[0] += (long long)m0 * ia[0]; zacc[1] += (long long)m0 * ia[1];
+              zacc[2] += (long long)m1 * ia[2]; zacc[3] += (long long)m1 * ia[3];
+              const int sx = sxi[min(kb >> kbg_log2, p.ngroups - 1)];
+              zt[0] += (long long)(m0 * int(mw.x & 3u)) * sx;
+              zt[1] += (long long)(m1 * int(mw.y & 3u)) * sx;
               ia[0] = ia[1] = ia[2] = ia[3] = 0;
             }
           }
@@ -482,15 +478,15 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       if (r == p.nranges - 1) {
         // limbs: lane t4 = 0 holds limbs 0,1 ; t4 = 1 holds limbs 2,3 (columns 4..7 are unused for one token)
         double v0 = 0.0, v1 = 0.0;
-        if (t4 == 0) { v0 = zacc[0] + 256.0 * zacc[1]; v1 = zacc[2] + 256.0 * zacc[3]; }
-        if (t4 == 1) { v0 = 65536.0 * (zacc[0] + 256.0 * zacc[1]); v1 = 65536.0 * (zacc[2] + 256.0 * zacc[3]); }
+        if (t4 == 0) { v0 = double(zacc[0]) + 256.0 * double(zacc[1]); v1 = double(zacc[2]) + 256.0 * double(zacc[3]); }
+        if (t4 == 1) { v0 = 65536.0 * (double(zacc[0]) + 256.0 * double(zacc[1])); v1 = 65536.0 * (double(zacc[2]) + 256.0 * double(zacc[3])); }
         v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
         v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
         if (t4 == 0) {
-          zpart[(tl * NW + warp) * 16 + g] = v0 * (1.0 / 64.0) - zt[0];
-          zpart[(tl * NW + warp) * 16 + g + 8] = v1 * (1.0 / 64.0) - zt[1];
+          zpart[(tl * NW + warp) * 16 + g] = v0 * (1.0 / 64.0) - double(zt[0]);
+          zpart[(tl * NW + warp) * 16 + g + 8] = v1 * (1.0 / 64.0) - double(zt[1]);
         }
-        zacc[0] = zacc[1] = zacc[2] = zacc[3] = 0.0; zt[0] = zt[1] = 0.0;
+        zacc[0] = zacc[1] = zacc[2] = zacc[3] = 0; zt[0] = zt[1] = 0;
       }
       // hand the buffer back: the last warp to leave it starts the copy of the unit that reuses it
       if (u + p.nbuf < NU) {
@@ -517,11 +513,12 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     double s = 0.0;
 #pragma unroll
     for (int w = 0; w < NW; ++w) s += zpart[(tl * NW + w) * 16 + r];
-    const double zhat = double(tab[2 * TR + tid]) + ldexp(s, E);
+    const int rexp = __float_as_int(tab[5 * TR + tid]);
+    const double zhat = double(tab[2 * TR + tid]) + ldexp(s, E + (rexp == kBadRow ? 0 : rexp));
     const double lo = double(tab[tid]), hi = double(tab[TR + tid]);
     int f = ((lo <= zhat) && (zhat < hi)) ? 0 : 1;
     if (tok_nonfinite) f = 1;
-    else if (tau > 0.0 && (fabs(zhat - lo) <= tau || fabs(zhat - hi) <= tau)) {
+    else if (rexp == kBadRow || (tau > 0.0 && (fabs(zhat - lo) <= tau || fabs(zhat - hi) <= tau))) {
       const int q = atomicAdd(const_cast<int*>(&misc[MS_NRC]), 1);
       if (q < MAXRC) rc[q] = tid;
       else {                                        // list full: this thread re-evaluates its neuron alone
@@ -732,10 +729,35 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
 }
 
 // ---- set-up kernels --------------------------------------------------------------------------------------
-// Predictor blocks: block (tile, kc) = 2 x 32 lanes x {A0,B0,A1,B1} code words + per-group {row g, row g+8} metadata.
+// A bf16 scale is m 2^(e-134) with an integer |m| < 256 (e = biased exponent, at least 1).  Over the groups of
+// one neuron the exponents differ little, so every scale of the row is an integer of at most 15 bits times
+// 2^(emin-134); rowexp[j] = emin - 134, or kBadRow when the spread is too wide (or a scale is inf / nan).
+__device__ __forceinline__ void bf16_parts(__nv_bfloat16 v, int* m, int* e) {
+  const uint32_t b = __bfloat16_as_ushort(v);
+  const int ex = int((b >> 7) & 0xffu), man = int(b & 0x7fu);
+  *e = ex ? ex : 1;
+  *m = (ex ? (128 | man) : man) * ((b & 0x8000u) ? -1 : 1);
+}
+__global__ void k_row_exponent(const __nv_bfloat16* __restrict__ scale, int h, int ng, int* __restrict__ rowexp) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= h) return;
+  int emin = 1 << 20, emax = 0;
+  bool bad = false;
+  for (int g = 0; g < ng; ++g) {
+    int m, e;
+    bf16_parts(scale[size_t(j) * ng + g], &m, &e);
+    if (e == 255) bad = true;
+    if (m != 0) { emin = min(emin, e); emax = max(emax, e); }
+  }
+  if (emax == 0) emin = emax = 1;                    // all scales zero
+  rowexp[j] = (bad || emax - emin > 7) ? kBadRow : emin - 134;
+}
+
+// Predictor blocks: block (tile, kc) = 2 x 32 lanes x {A0,B0,A1,B1} code words + per-group {row g, row g+8}
+// words (integer scale << 16 | zero-point).
 __global__ void k_pack_pblocks(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
-                               const uint8_t* __restrict__ zero, uint8_t* __restrict__ out, int d, int G,
-                               int nkc, int pbs) {
+                               const uint8_t* __restrict__ zero, const int* __restrict__ rowexp,
+                               uint8_t* __restrict__ out, int d, int G, int nkc, int pbs) {
   const int tile = blockIdx.x, kc = blockIdx.y;
   uint8_t* blk = out + (size_t(tile) * nkc + kc) * pbs;
   const int nwords = d / 16, ng = d / G;
@@ -753,7 +775,13 @@ __global__ void k_pack_pblocks(const uint32_t* __restrict__ codes, const __nv_bf
     const int row = tile * 16 + gg + (hi ? 8 : 0);
     const int grp = kc * gpc + gl;
     uint32_t w = 0u;
-    if (grp < ng) w = (uint32_t(__bfloat16_as_ushort(scale[size_t(row) * ng + grp])) << 16) | uint32_t(zero[size_t(row) * ng + grp] & 3u);
+    const int re = rowexp[row];
+    if (grp < ng && re != kBadRow) {
+      int m, ex;
+      bf16_parts(scale[size_t(row) * ng + grp], &m, &ex);
+      const int M = m * (1 << (m != 0 ? ex - (re + 134) : 0));
+      w = (uint32_t(M & 0xffff) << 16) | uint32_t(zero[size_t(row) * ng + grp] & 3u);
+    }
     reinterpret_cast<uint32_t*>(blk + 1024)[e] = w;
   }
 }
@@ -776,7 +804,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   H->codes_mma = nullptr;
   const int d = H->d, h = H->h, G = H->G;
   if (H->dtype != TARDIS_BF16) return TARDIS_OK;
-  if (!(G == 64 || G == 128 || G == 256)) return TARDIS_OK;         // generic kernels serve other group sizes
+  if (!(G == 64 || G == 128)) return TARDIS_OK;                     // generic kernels serve other group sizes
   const int NT = h / 16;
   const int nvec = d / 8;
   const int cw = (nvec + NW - 1) / NW;
@@ -833,6 +861,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   cudaError_t e = cudaMalloc(&S->pblocks, pb_bytes); tally += pb_bytes;
   if (e == cudaSuccess) { e = cudaMalloc(&S->plan, sizeof(int2) * grid); tally += sizeof(int2) * grid; }
   if (e == cudaSuccess) { e = cudaMalloc(&S->smax, 16); tally += 16; }
+  if (e == cudaSuccess) { e = cudaMalloc(&S->rowexp, sizeof(int) * h); tally += sizeof(int) * h; }
   if (e == cudaSuccess) { e = cudaMalloc(&S->yacc, yacc_bytes); tally += yacc_bytes; }
   if (e == cudaSuccess) { e = cudaMalloc(&S->ctl, sizeof(unsigned int) * CTL_WORDS); tally += sizeof(unsigned int) * CTL_WORDS; }
   if (e != cudaSuccess) { set_last_error(e, "cudaMalloc"); cudaGetLastError(); return fail(TARDIS_ERR_ALLOC); }
@@ -852,7 +881,8 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   if (e == cudaSuccess) e = cudaMemsetAsync(S->yacc, 0, yacc_bytes, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(S->ctl, 0, sizeof(unsigned int) * CTL_WORDS, s);
   if (e != cudaSuccess) { set_last_error(e, "decode_prepare"); return fail(TARDIS_ERR_CUDA); }
-  k_pack_pblocks<<<dim3(NT, p.nkc), 128, 0, s>>>(H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero,
+  k_row_exponent<<<(h + 255) / 256, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->scale), h, H->ngroups, S->rowexp);
+  k_pack_pblocks<<<dim3(NT, p.nkc), 128, 0, s>>>(H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, S->rowexp,
                                                  S->pblocks, d, G, p.nkc, p.pbs);
   k_max_scale<<<64, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->scale), size_t(h) * H->ngroups, S->smax);
   e = cudaGetLastError();
@@ -860,7 +890,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
   if (e != cudaSuccess) { set_last_error(e, "decode_prepare launch"); return fail(TARDIS_ERR_CUDA); }
 
-  p.pblocks = S->pblocks; p.plan = S->plan; p.smax = S->smax; p.yacc = S->yacc; p.ctl = S->ctl;
+  p.pblocks = S->pblocks; p.plan = S->plan; p.smax = S->smax; p.rowexp = S->rowexp; p.yacc = S->yacc; p.ctl = S->ctl;
   p.W1 = static_cast<const __nv_bfloat16*>(H->W1); p.W2T = static_cast<const __nv_bfloat16*>(H->W2T);
   p.C = static_cast<const __nv_bfloat16*>(H->C); p.bf = H->bf; p.lo = H->lo; p.hi = H->hi; p.a = H->a; p.c = H->c; p.b1 = H->b1;
   p.codes = H->codes; p.scale = static_cast<const __nv_bfloat16*>(H->scale); p.zero = H->zero;
@@ -892,7 +922,7 @@ tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, 
 void decode_release(Handle* H) {
   Scratch* S = static_cast<Scratch*>(H->dscratch);
   if (!S) return;
-  void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl};
+  void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl, S->rowexp};
   for (void* q : ptrs)
     if (q) cudaFree(q);
   delete S;
