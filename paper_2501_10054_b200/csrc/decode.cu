@@ -122,6 +122,14 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
                : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// The same with a zero accumulator going in: MMAs of one warp that do not depend on each other pipeline
+// four times better than a chain through one accumulator, so each MMA of a group starts its own sum.
+__device__ __forceinline__ void mma_u8s8_z(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                           uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+               : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
   asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
@@ -430,8 +438,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   // ---- predictor: warp w takes chunk w of every unit; partial scores of a tile go to shared memory ----
   {
     long long zacc[4] = {0, 0, 0, 0}, zt[2] = {0, 0};
-    const int kb_per_group = p.G / 64;                       // 1 or 2
-    const int kbg_log2 = kb_per_group >> 1;                  // log2 of it
+    const int gpc = KC / p.G;                                // groups per chunk: 4 or 2
     for (int u = 0; u < NU; ++u) {
       const int b = u % p.nbuf;
       const uint32_t par = uint32_t(u / p.nbuf) & 1u;
@@ -447,33 +454,45 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         const uint8_t* blk = pbuf + size_t(b) * p.unit_bytes + size_t(warp) * p.pbs;
         const uint4* cp = reinterpret_cast<const uint4*>(blk);
         const uint2* mp = reinterpret_cast<const uint2*>(blk + 1024);
-        int ia[4] = {0, 0, 0, 0};
+        // group g2 of the chunk done: sums (|.| < 2^22) times the integer scales (|.| < 2^15), all exact
+        auto scale_group = [&](const int (&ia)[4], int gl) {
+          const uint2 mw = mp[gl * 8 + g];
+          const int m0 = int(mw.x) >> 16, m1 = int(mw.y) >> 16;
+          zacc[0] += (long long)m0 * ia[0]; zacc[1] += (long long)m0 * ia[1];
+          zacc[2] += (long long)m1 * ia[2]; zacc[3] += (long long)m1 * ia[3];
+          const int sx = sxi[min(kc * gpc + gl, p.ngroups - 1)];
+          zt[0] += (long long)(m0 * int(mw.x & 3u)) * sx;
+          zt[1] += (long long)(m1 * int(mw.y & 3u)) * sx;
+        };
+
 #pragma unroll
-        for (int pair = 0; pair < 2; ++pair) {
+        for (int pair = 0; pair < 2; ++pair) {            // 128 channels: four independent MMAs
           const uint4 cw = cp[pair * 32 + lane];
+          const int kb = kc * 4 + pair * 2;
+          uint4 xb0 = make_uint4(0u, 0u, 0u, 0u), xb1 = xb0;
+          if (g < 4) {
+            xb0 = *reinterpret_cast<const uint4*>(xq + size_t(g) * xq_stride + size_t(kb) * 64 + t4 * 16);
+            xb1 = *reinterpret_cast<const uint4*>(xq + size_t(g) * xq_stride + size_t(kb + 1) * 64 + t4 * 16);
+          }
+          int q0[4], q1[4], q2[4], q3[4];
+          mma_u8s8_z(q0, cw.x & 0x03030303u, cw.y & 0x03030303u, cw.x & 0x0C0C0C0Cu, cw.y & 0x0C0C0C0Cu, xb0.x, xb0.y);
+          mma_u8s8_z(q1, cw.x & 0x30303030u, cw.y & 0x30303030u, cw.x & 0xC0C0C0C0u, cw.y & 0xC0C0C0C0u, xb0.z, xb0.w);
+          mma_u8s8_z(q2, cw.z & 0x03030303u, cw.w & 0x03030303u, cw.z & 0x0C0C0C0Cu, cw.w & 0x0C0C0C0Cu, xb1.x, xb1.y);
+          mma_u8s8_z(q3, cw.z & 0x30303030u, cw.w & 0x30303030u, cw.z & 0xC0C0C0C0u, cw.w & 0xC0C0C0C0u, xb1.z, xb1.w);
+          if (p.G == 64) {
+            int ga[4], gb[4];
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int kbl = pair * 2 + half;              // 64-channel block inside the 256-channel chunk
-            const int kb = kc * 4 + kbl;
-            const uint32_t A = half ? cw.z : cw.x, B = half ? cw.w : cw.y;
-            uint4 xb = make_uint4(0u, 0u, 0u, 0u);
-            if (g < 4) xb = *reinterpret_cast<const uint4*>(xq + size_t(g) * xq_stride + size_t(kb) * 64 + t4 * 16);
-            mma_u8s8(ia, A & 0x03030303u, B & 0x03030303u, A & 0x0C0C0C0Cu, B & 0x0C0C0C0Cu, xb.x, xb.y);
-            mma_u8s8(ia, A & 0x30303030u, B & 0x30303030u, A & 0xC0C0C0C0u, B & 0xC0C0C0C0u, xb.z, xb.w);
-            if (((kbl + 1) & (kb_per_group - 1)) == 0) {
-              // group done: sums (|.| < 2^22) times the integer scales (|.| < 2^15), all exact
-              const int gl = kbl >> kbg_log2;             // group inside the chunk
-              const uint2 mw = mp[gl * 8 + g];
-              const int m0 = int(mw.x) >> 16, m1 = int(mw.y) >> 16;
-              zacc[0] += (long long)m0 * ia[0]; zacc[1] += (long long)m0 * ia[1];
-              zacc[2] += (long long)m1 * ia[2]; zacc[3] += (long long)m1 * ia[3];
-              const int sx = sxi[min(kb >> kbg_log2, p.ngroups - 1)];
-              zt[0] += (long long)(m0 * int(mw.x & 3u)) * sx;
-              zt[1] += (long long)(m1 * int(mw.y & 3u)) * sx;
-              ia[0] = ia[1] = ia[2] = ia[3] = 0;
-            }
+            for (int i = 0; i < 4; ++i) { ga[i] = q0[i] + q1[i]; gb[i] = q2[i] + q3[i]; }
+            scale_group(ga, pair * 2);
+            scale_group(gb, pair * 2 + 1);
+          } else {                                        // G == 128
+            int ga[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) ga[i] = (q0[i] + q1[i]) + (q2[i] + q3[i]);
+            scale_group(ga, pair);
           }
         }
+
       }
       if (r == p.nranges - 1) {
         // limbs: lane t4 = 0 holds limbs 0,1 ; t4 = 1 holds limbs 2,3 (columns 4..7 are unused for one token)
