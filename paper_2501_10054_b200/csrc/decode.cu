@@ -42,7 +42,6 @@ constexpr int NTH = NW * 32;      // threads per CTA
 constexpr int KC = 256;           // channels per predictor block
 constexpr int MAXTILES = 16;      // predictor tiles (of 16 neurons) per CTA
 constexpr int MAXRC = 64;         // exact re-checks per CTA before the list overflows (rest handled in place)
-constexpr int LOADS = 4;          // 128-bit loads per thread and folded-matrix chunk (rows x slots)
 constexpr int FIXLOADS = 8;       // 128-bit loads per thread and batch of flagged rows (rows x slots)
 constexpr int MAXBUF = 8;         // predictor unit buffers in shared memory
 constexpr int kBadRow = 0x40000000;   // row whose group scales do not fit the integer form: always re-evaluated
@@ -50,15 +49,16 @@ constexpr int NREP = 4;           // replicas of the output accumulator
 constexpr int XVR = 2;            // 8-channel vectors of x per thread (padded d <= 8192)
 constexpr uint32_t SPIN_LIMIT = 1u << 21;   // spaced polls of a bounded mbarrier wait: a fraction of a second
 // control words (unsigned int) in global scratch; all zero between calls
-constexpr int CTL_TICKET = 0;     // [NW] stride 32: next folded-matrix row chunk of a warp's column range
-constexpr int CTL_DONE = 512;     // [NW] stride 32: warps that have added their columns
+constexpr int CTL_TICKET = 0;     // [NW] stride 32: next folded-matrix unit of a warp index
+constexpr int CTL_DONE = 512;     // CTAs that have added all their contributions
 constexpr int CTL_NFL = 1024;     // flagged neurons of the token so far
 constexpr int CTL_WORDS = 1056;
 
 struct Params {
   const uint8_t* pblocks;  // [tile][kchunk] predictor blocks
   int pbs, nkc, G;
-  const __nv_bfloat16 *W1, *W2T, *C;
+  const __nv_bfloat16 *W1, *W2T;
+  const uint4* Cp;         // folded matrix in tensor-core fragment order (see k_pack_folded)
   const float *bf, *lo, *hi, *a, *c, *b1;
   const uint32_t* codes; const __nv_bfloat16* scale; const uint8_t* zero;   // originals (exact re-check)
   const float* smax;       // largest group scale of the layer
@@ -73,12 +73,13 @@ struct Params {
   int nbuf, unit_bytes;    // unit buffers in shared memory and their size
   int tiles_max;
   int nvec, cw;            // 8-column vectors in a row; vectors per warp
-  int ntk;                 // row chunks of the folded matrix (LOADS / VPT rows each)
+  int nunits;              // folded-matrix units in all
+  int ntk;                 // folded-matrix units (16 outputs x 256 channels) per warp index
   int pre_chunks;          // chunks a second-half CTA takes before its predictor
 };
 
 struct Scratch {           // handle-owned device memory of the fused path
-  uint8_t* pblocks; int2* plan; float* smax; float* yacc; unsigned int* ctl; int* rowexp;
+  uint8_t* pblocks; int2* plan; float* smax; float* yacc; unsigned int* ctl; int* rowexp; uint4* Cp;
   Params base; size_t smem_bytes; size_t bytes; int grid; int vpt;
 };
 
@@ -130,6 +131,15 @@ __device__ __forceinline__ void mma_u8s8_z(int (&c)[4], uint32_t a0, uint32_t a1
                : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
 }
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void red_add_f32(float* addr, float v) {
+  asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
+}
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
   asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
@@ -162,7 +172,7 @@ struct SmemLayout {
     xh = take(size_t(dpad) * 2, 16);
     sxi = take(size_t(ngroups + 16) * sizeof(int), 8);
     zpart = take(rows * NW * sizeof(double), 8);
-    wpart = take(size_t(FIXLOADS) * NW * sizeof(float), 4);
+    wpart = take(size_t(16) * NW * sizeof(float), 4);
     score = take(rows * sizeof(double), 8);
     tab = take(6 * rows * sizeof(float), 4);
     fl_j = take(rows * sizeof(int), 4);
@@ -175,7 +185,7 @@ struct SmemLayout {
     total = o;
   }
 };
-enum { MS_NFL = 0, MS_NRC = 1, MS_ERR = 2, MS_WCNT = 8, MS_BUFCNT = 32 };
+enum { MS_NFL = 0, MS_NRC = 1, MS_ERR = 2, MS_LAST = 3, MS_WCNT = 8, MS_BUFCNT = 32 };
 
 // ---- the kernel ---------------------------------------------------------------------------------------
 template <int VPT>
@@ -273,9 +283,9 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   bool tok_nonfinite = false;
 #pragma unroll
   for (int w = 0; w < NW; ++w) { amax_all = fmaxf(amax_all, wred[w]); tok_nonfinite |= wred[NW + w] != 0.f; }
-  // exponent E: |x| 2^-E < 2^24 for every element
+  // exponent E: |x| 2^-E < 2^22 for every element
   int E = 0;
-  if (amax_all > 0.f && !tok_nonfinite) E = max(int((__float_as_uint(amax_all) >> 23) & 0xff) - 127 - 23, -100);
+  if (amax_all > 0.f && !tok_nonfinite) E = max(int((__float_as_uint(amax_all) >> 23) & 0xff) - 127 - 21, -100);
 
   // ---- fixed-point limbs of x in tensor-core operand order; group sums; truncation residual ----
   // A thread holds 8 channels = half of a 16-channel unit; the two halves meet through one shuffle.
@@ -297,8 +307,9 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         const float s = (active && !tok_nonfinite) ? f[c] * inv : 0.f;
-        const int X = __float2int_rz(s);
-        resid += fabsf(s - float(X));
+        const float t = s + 12582912.f;                         // 1.5 * 2^23: rounds s to an integer (|s| < 2^22)
+        const int X = __float_as_int(t) - 0x4B400000;
+        resid += fabsf(s - (t - 12582912.f));
         sx += X;
         // signed base-256 digits of X 4^(3-f): adding 0x80 to the three low bytes and flipping
         // those bits back leaves byte l = digit l as a signed 8-bit value
@@ -349,7 +360,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     if (lane == 0) wred[2 * NW + warp] = resid;
   }
   __syncthreads();
-  // tolerance of the fast score: every dropped fraction (< 1 unit of 2^E) times |code - zero| <= 3 times the scale
+  // tolerance of the fast score: every rounding residual (<= 1/2 unit of 2^E) times |code - zero| <= 3 times the scale
   double tau;
   {
     float rs = 0.f;
@@ -367,66 +378,69 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     cval[m] = vl < p.cw && vec < p.nvec;
     col[m] = cval[m] ? vec * 8 : 0;
   }
-  float acc[VPT][8];
-#pragma unroll
-  for (int m = 0; m < VPT; ++m)
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc[m][i] = 0.f;
 
-  // ---- speculative folded product: row chunks of C drawn from this column range's ticket ----
-  // stream_c(n) takes at most n chunks (two in flight per thread); the ticket for a chunk is drawn one
-  // step before the chunk is needed so that the atomic's latency is covered by the loads in flight.
+  // ---- speculative folded product on the tensor cores ----
+  // The folded matrix is stored in units of 16 outputs x 256 channels (8 KB, contiguous, already in
+  // A-fragment order).  A warp draws units from the ticket of its warp index, streams a unit as four
+  // blocks of four 128-bit loads per lane (one block ahead of the one being multiplied), multiplies it
+  // with x (the B operand: column 0 = x, other columns zero) in two independent accumulators, and adds
+  // the 16 partial outputs to the accumulator replica of its CTA.  stream_c(n) takes at most n units.
+  float* const rep = p.yacc + size_t(blockIdx.x % NREP) * p.dacc;
   auto stream_c = [&](int budget) {
-    constexpr int TK = LOADS / VPT;   // rows per chunk
     unsigned int* ticket = p.ctl + CTL_TICKET + warp * 32;
-    auto issue = [&]() -> unsigned int {
+    auto issue = [&]() -> unsigned int {        // lane 0 draws; the value is looked at one unit later
       unsigned int t = 0;
       if (lane == 0) t = atomicAdd(ticket, 1u);
       return t;
     };
     auto resolve = [&](unsigned int raw) -> int {
       const unsigned int t = __shfl_sync(0xffffffffu, raw, 0);
-      return t < (unsigned int)p.ntk ? int(t) : -1;
+      return t < (unsigned int)p.ntk && int(t * NW + warp) < p.nunits ? int(t * NW + warp) : -1;
     };
-    auto load = [&](uint4 (&buf)[TK][VPT], int tk) {
+    auto load = [&](uint4 (&buf)[4], int u, int bi) {
+      const uint4* src = p.Cp + (size_t(u) * 16 + bi * 4) * 32 + lane;
 #pragma unroll
-      for (int r = 0; r < TK; ++r) {
-        const int k = tk * TK + r;
-#pragma unroll
-        for (int m = 0; m < VPT; ++m)
-          buf[r][m] = (k < d && cval[m]) ? ldg_stream(p.C + size_t(k) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
+      for (int m = 0; m < 4; ++m) buf[m] = ldg_stream(src + m * 32);
+    };
+    auto multiply = [&](float (&c)[2][4], const uint4 (&buf)[4], int u, int bi) {
+      uint4 x0 = make_uint4(0u, 0u, 0u, 0u), x1 = x0;
+      if (g == 0) {
+        const uint4* xp = reinterpret_cast<const uint4*>(xh + (u % p.nkc) * KC + bi * 64 + t4 * 16);
+        x0 = xp[0]; x1 = xp[1];
       }
+      mma_bf16(c[0], buf[0].x, buf[0].y, buf[0].z, buf[0].w, x0.x, x0.y);
+      mma_bf16(c[1], buf[1].x, buf[1].y, buf[1].z, buf[1].w, x0.z, x0.w);
+      mma_bf16(c[0], buf[2].x, buf[2].y, buf[2].z, buf[2].w, x1.x, x1.y);
+      mma_bf16(c[1], buf[3].x, buf[3].y, buf[3].z, buf[3].w, x1.z, x1.w);
     };
-    auto consume = [&](const uint4 (&buf)[TK][VPT], int tk) {
+    uint4 ba[4], bb[4];
+    int u = budget > 0 ? resolve(issue()) : -1;
+    --budget;
+    bool more = u >= 0 && budget > 0;
+    unsigned int raw = more ? issue() : 0xffffffffu;
+    if (u >= 0) load(ba, u, 0);
+    while (u >= 0) {
+      float c[2][4];
 #pragma unroll
-      for (int r = 0; r < TK; ++r) {
-        const int k = tk * TK + r;
-        const float sc = k < d ? __bfloat162float(xh[k]) : 0.f;
-#pragma unroll
-        for (int m = 0; m < VPT; ++m) fma8(acc[m], sc, buf[r][m]);
-      }
-    };
-    uint4 b0[TK][VPT], b1[TK][VPT];
-    int t0 = budget > 0 ? resolve(issue()) : -1;
-    int t1 = (t0 >= 0 && budget > 1) ? resolve(issue()) : -1;
-    budget -= 2;
-    if (t0 >= 0) load(b0, t0);
-    if (t1 >= 0) load(b1, t1);
-    bool more = t1 >= 0 && budget > 0;
-    while (t0 >= 0) {
-      unsigned int raw = more ? issue() : 0xffffffffu;
-      consume(b0, t0);
-      t0 = more ? resolve(raw) : -1;
+      for (int m = 0; m < 2; ++m) c[m][0] = c[m][1] = c[m][2] = c[m][3] = 0.f;
+      load(bb, u, 1);
+      multiply(c, ba, u, 0);
+      load(ba, u, 2);
+      multiply(c, bb, u, 1);
+      load(bb, u, 3);
+      multiply(c, ba, u, 2);
+      const int un = more ? resolve(raw) : -1;        // the next unit: its first block goes in flight now
       --budget;
-      more = t0 >= 0 && budget > 0;
-      if (t0 >= 0) load(b0, t0);
-      if (t1 < 0) break;
+      more = un >= 0 && budget > 0;
       raw = more ? issue() : 0xffffffffu;
-      consume(b1, t1);
-      t1 = more ? resolve(raw) : -1;
-      --budget;
-      more = t1 >= 0 && budget > 0;
-      if (t1 >= 0) load(b1, t1);
+      if (un >= 0) load(ba, un, 0);
+      multiply(c, bb, u, 3);
+      if (t4 == 0) {
+        const int i0 = (u / p.nkc) * 16 + g;
+        red_add_f32(rep + i0, c[0][0] + c[1][0]);
+        red_add_f32(rep + i0 + 8, c[0][2] + c[1][2]);
+      }
+      u = un;
     }
   };
 
@@ -616,47 +630,43 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   __syncthreads();
   const int nfl = misc[MS_NFL];
 
-  constexpr int FB = FIXLOADS / VPT;   // flagged rows per batch
-  uint4 w[FB][VPT];
-
-  // ---- result fixing, first half: W1 rows -> z_j -> delta_j ----
-  if (nfl > 0) {
-    float xr[VPT][8];
+  // ---- result fixing, first half: W1 rows -> z_j -> delta_j, on the tensor cores ----
+  // 16 flagged rows form the A operand (row g from the list entry g, row g + 8 from entry g + 8), x the B
+  // operand (column 0).  A lane reads 8 consecutive channels of its two rows per step; the same 8
+  // channels of x sit in the matching operand slots, so the order of channels inside an MMA does not
+  // matter.  The 16 warps split the channel range; their partial z_j meet in shared memory.
+  {
+    const int kw = ((p.dpad / NW) + 31) / 32 * 32;          // channels per warp
+    for (int e0 = 0; e0 < nfl; e0 += 16) {
+      const int ja = (e0 + g < nfl) ? fl_j[e0 + g] : -1;
+      const int jb = (e0 + 8 + g < nfl) ? fl_j[e0 + 8 + g] : -1;
+      const __nv_bfloat16* pa = p.W1 + size_t(ja < 0 ? 0 : ja) * d;
+      const __nv_bfloat16* pb = p.W1 + size_t(jb < 0 ? 0 : jb) * d;
+      float z0[4] = {0.f, 0.f, 0.f, 0.f}, z1[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int k0 = warp * kw; k0 < (warp + 1) * kw; k0 += 128) {
+        uint4 wa[4], wb[4];
 #pragma unroll
-    for (int m = 0; m < VPT; ++m) unpack8(xr[m], *reinterpret_cast<const uint4*>(xh + col[m]));
-    for (int e0 = 0; e0 < nfl; e0 += FB) {
+        for (int q = 0; q < 4; ++q) {
+          const int k = k0 + q * 32 + t4 * 8;
+          const bool in = k < d && k < (warp + 1) * kw;
+          wa[q] = (in && ja >= 0) ? ldg_stream(pa + k) : make_uint4(0u, 0u, 0u, 0u);
+          wb[q] = (in && jb >= 0) ? ldg_stream(pb + k) : make_uint4(0u, 0u, 0u, 0u);
+        }
 #pragma unroll
-      for (int r = 0; r < FB; ++r) {
-        const int j = (e0 + r < nfl) ? fl_j[e0 + r] : -1;
-#pragma unroll
-        for (int m = 0; m < VPT; ++m)
-          w[r][m] = (j >= 0 && cval[m]) ? ldg_stream(p.W1 + size_t(j) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
-      }
-      float part[FB];
-#pragma unroll
-      for (int r = 0; r < FB; ++r) {
-        part[r] = 0.f;
-#pragma unroll
-        for (int m = 0; m < VPT; ++m) part[r] += dot8(w[r][m], xr[m]);
-      }
-      // the W2T rows of the first batch go in flight while the last dot products meet
-      if (e0 + FB >= nfl) {
-#pragma unroll
-        for (int r = 0; r < FB; ++r) {
-          const int j = (r < nfl) ? fl_j[r] : -1;
-#pragma unroll
-          for (int m = 0; m < VPT; ++m)
-            w[r][m] = (j >= 0 && cval[m]) ? ldg_stream(p.W2T + size_t(j) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
+        for (int q = 0; q < 4; ++q) {
+          const int k = k0 + q * 32 + t4 * 8;
+          uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+          if (g == 0 && k < p.dpad) xv = *reinterpret_cast<const uint4*>(xh + k);
+          mma_bf16(z0, wa[q].x, wb[q].x, wa[q].y, wb[q].y, xv.x, xv.y);
+          mma_bf16(z1, wa[q].z, wb[q].z, wa[q].w, wb[q].w, xv.z, xv.w);
         }
       }
-#pragma unroll
-      for (int r = 0; r < FB; ++r) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) part[r] += __shfl_xor_sync(0xffffffffu, part[r], o);
-        if (lane == 0) wpart[r * NW + warp] = part[r];
+      if (t4 == 0) {
+        wpart[g * NW + warp] = z0[0] + z1[0];
+        wpart[(g + 8) * NW + warp] = z0[2] + z1[2];
       }
       __syncthreads();
-      if (tid < FB && e0 + tid < nfl) {
+      if (tid < 16 && e0 + tid < nfl) {
         const int row = fl_j[e0 + tid] - plan.x * 16;
         float z = 0.f;
 #pragma unroll
@@ -668,9 +678,17 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     }
   }
 
+  constexpr int FB = FIXLOADS / VPT;   // flagged rows per batch of the second half
+  uint4 w[FB][VPT];
+  float acc[VPT][8];
+#pragma unroll
+  for (int m = 0; m < VPT; ++m)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[m][i] = 0.f;
+
   // ---- result fixing, second half: W2T rows scaled by delta_j ----
   for (int e0 = 0; e0 < nfl; e0 += FB) {
-    if (e0 > 0) {
+    {
 #pragma unroll
       for (int r = 0; r < FB; ++r) {
         const int j = (e0 + r < nfl) ? fl_j[e0 + r] : -1;
@@ -691,8 +709,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   stream_c(0x7fffffff);
 
   // ---- combine: add this warp's columns to one replica; the last warp on a column range finishes it ----
-  {
-    float* rep = p.yacc + size_t(blockIdx.x % NREP) * p.dacc;
+  if (nfl > 0) {
 #pragma unroll
     for (int m = 0; m < VPT; ++m)
       if (cval[m]) {
@@ -700,12 +717,13 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         red_add_v4(rep + col[m] + 4, acc[m][4], acc[m][5], acc[m][6], acc[m][7]);
       }
   }
+  // every warp of every CTA may have added to any column, so the columns are complete when the last CTA
+  // is: the CTAs count themselves, and the last one turns the accumulator into y
   __threadfence();
-  __syncwarp();
-  unsigned int arrived = 0;
-  if (lane == 0) arrived = atomicAdd(&p.ctl[CTL_DONE + warp * 32], 1u);
-  arrived = __shfl_sync(0xffffffffu, arrived, 0);
-  if (arrived == gridDim.x - 1) {
+  __syncthreads();
+  if (tid == 0) misc[MS_LAST] = int(atomicAdd(&p.ctl[CTL_DONE], 1u));
+  __syncthreads();
+  if (misc[MS_LAST] == int(gridDim.x) - 1) {
     __threadfence();
 #pragma unroll
     for (int m = 0; m < VPT; ++m)
@@ -737,8 +755,8 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       }
     if (lane == 0) {
       p.ctl[CTL_TICKET + warp * 32] = 0u;
-      p.ctl[CTL_DONE + warp * 32] = 0u;
-      if (warp == 0) {   // every CTA's warp 0 has arrived, so every CTA's flagged count is in
+      if (warp == 0) {   // every CTA has arrived, so every CTA's flagged count is in
+        p.ctl[CTL_DONE] = 0u;
         const unsigned int tot = atomicExch(&p.ctl[CTL_NFL], 0u);
         atomicAdd(&p.counters[CTR_FLAGGED_TOTAL], (unsigned long long)tot);
         atomicMax(&p.counters[CTR_FLAGGED_MAX], (unsigned long long)tot);
@@ -805,6 +823,28 @@ __global__ void k_pack_pblocks(const uint32_t* __restrict__ codes, const __nv_bf
   }
 }
 
+// Folded matrix in A-fragment order of mma.m16n8k16 (bf16).  Unit (it, kc) = outputs 16 it .. 16 it + 15
+// times channels 256 kc .. 256 kc + 255 = 4 blocks x 4 MMAs x 32 lanes x 16 bytes, contiguous; units are
+// ordered it-major.  Register r of lane (g, t4) in MMA m of block bi holds W_f[16 it + g + 8 (r & 1)]
+// [256 kc + 64 bi + 16 t4 + 4 m + 2 (r >> 1) + {0, 1}]: a lane's B operands for a block are then 16
+// consecutive channels of x.  C is the fold's output, C[k][i] = W_f[i][k]; channels beyond d are zero.
+__global__ void k_pack_folded(const __nv_bfloat16* __restrict__ C, uint4* __restrict__ out, int d, int nkc) {
+  const int u = blockIdx.x, it = u / nkc, kc = u - it * nkc;
+  for (int e = threadIdx.x; e < 16 * 32; e += blockDim.x) {
+    const int bm = e >> 5, ln = e & 31, bi = bm >> 2, m = bm & 3, gg = ln >> 2, tt = ln & 3;
+    uint32_t r[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int row = it * 16 + gg + ((q & 1) ? 8 : 0);
+      const int k = kc * KC + bi * 64 + tt * 16 + m * 4 + ((q >> 1) ? 2 : 0);
+      const uint32_t lo = (k < d) ? __bfloat16_as_ushort(C[size_t(k) * d + row]) : 0u;
+      const uint32_t hi = (k + 1 < d) ? __bfloat16_as_ushort(C[size_t(k + 1) * d + row]) : 0u;
+      r[q] = lo | (hi << 16);
+    }
+    out[size_t(u) * 512 + e] = make_uint4(r[0], r[1], r[2], r[3]);
+  }
+}
+
 __global__ void k_max_scale(const __nv_bfloat16* __restrict__ scale, size_t count, float* out) {
   float m = 0.f;
   for (size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x; e < count; e += size_t(gridDim.x) * blockDim.x)
@@ -829,7 +869,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   const int cw = (nvec + NW - 1) / NW;
   const int vpt = (cw + 31) / 32;
   const int dpad = (d + KC - 1) / KC * KC;
-  if (vpt > 2 || d < 64 || dpad > XVR * NTH * 8) return TARDIS_OK;
+  if (vpt > 2 || d < 64 || d % 16 || dpad > XVR * NTH * 8) return TARDIS_OK;
   int max_smem = 0, sm_smem = 0;
   TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, H->device));
   TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, H->device));
@@ -846,8 +886,8 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   p.cpr = (p.nkc + p.nranges - 1) / p.nranges;
   p.unit_bytes = p.cpr * p.pbs;
   p.nvec = nvec; p.cw = cw;
-  const int tk_rows = LOADS / vpt;
-  p.ntk = (d + tk_rows - 1) / tk_rows;
+  p.nunits = (d / 16) * p.nkc;
+  p.ntk = (p.nunits + NW - 1) / NW;
   p.pre_chunks = 2;
   S->vpt = vpt;
   // two CTAs per SM when their shared memory fits (each CTA also reserves 1 KB), else one
@@ -881,6 +921,8 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   if (e == cudaSuccess) { e = cudaMalloc(&S->plan, sizeof(int2) * grid); tally += sizeof(int2) * grid; }
   if (e == cudaSuccess) { e = cudaMalloc(&S->smax, 16); tally += 16; }
   if (e == cudaSuccess) { e = cudaMalloc(&S->rowexp, sizeof(int) * h); tally += sizeof(int) * h; }
+  const size_t cp_bytes = size_t(p.nunits) * 8192;
+  if (e == cudaSuccess) { e = cudaMalloc(&S->Cp, cp_bytes); tally += cp_bytes; }
   if (e == cudaSuccess) { e = cudaMalloc(&S->yacc, yacc_bytes); tally += yacc_bytes; }
   if (e == cudaSuccess) { e = cudaMalloc(&S->ctl, sizeof(unsigned int) * CTL_WORDS); tally += sizeof(unsigned int) * CTL_WORDS; }
   if (e != cudaSuccess) { set_last_error(e, "cudaMalloc"); cudaGetLastError(); return fail(TARDIS_ERR_ALLOC); }
@@ -903,6 +945,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   k_row_exponent<<<(h + 255) / 256, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->scale), h, H->ngroups, S->rowexp);
   k_pack_pblocks<<<dim3(NT, p.nkc), 128, 0, s>>>(H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, S->rowexp,
                                                  S->pblocks, d, G, p.nkc, p.pbs);
+  k_pack_folded<<<p.nunits, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->C), S->Cp, d, p.nkc);
   k_max_scale<<<64, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->scale), size_t(h) * H->ngroups, S->smax);
   e = cudaGetLastError();
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
@@ -911,13 +954,14 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
 
   p.pblocks = S->pblocks; p.plan = S->plan; p.smax = S->smax; p.rowexp = S->rowexp; p.yacc = S->yacc; p.ctl = S->ctl;
   p.W1 = static_cast<const __nv_bfloat16*>(H->W1); p.W2T = static_cast<const __nv_bfloat16*>(H->W2T);
-  p.C = static_cast<const __nv_bfloat16*>(H->C); p.bf = H->bf; p.lo = H->lo; p.hi = H->hi; p.a = H->a; p.c = H->c; p.b1 = H->b1;
+  p.Cp = S->Cp; p.bf = H->bf; p.lo = H->lo; p.hi = H->hi; p.a = H->a; p.c = H->c; p.b1 = H->b1;
   p.codes = H->codes; p.scale = static_cast<const __nv_bfloat16*>(H->scale); p.zero = H->zero;
   p.counters = H->counters;
   H->dscratch = S;
   H->dscratch_bytes = S->bytes;
-  H->bytes_scratch += S->bytes - pb_bytes;
+  H->bytes_scratch += S->bytes - pb_bytes - cp_bytes;
   H->bytes_predictor += pb_bytes;
+  H->bytes_folded += cp_bytes;
   H->codes_mma = reinterpret_cast<uint32_t*>(S->pblocks);
   return TARDIS_OK;
 }
@@ -941,7 +985,7 @@ tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, 
 void decode_release(Handle* H) {
   Scratch* S = static_cast<Scratch*>(H->dscratch);
   if (!S) return;
-  void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl, S->rowexp};
+  void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl, S->rowexp, S->Cp};
   for (void* q : ptrs)
     if (q) cudaFree(q);
   delete S;
