@@ -49,10 +49,10 @@ constexpr int NREP = 4;           // replicas of the output accumulator
 constexpr int XVR = 2;            // 8-channel vectors of x per thread (padded d <= 8192)
 constexpr uint32_t SPIN_LIMIT = 1u << 21;   // spaced polls of a bounded mbarrier wait: a fraction of a second
 // control words (unsigned int) in global scratch; all zero between calls
-constexpr int CTL_TICKET = 0;     // [NW] stride 32: next folded-matrix unit of a warp index
-constexpr int CTL_DONE = 512;     // CTAs that have added all their contributions
-constexpr int CTL_NFL = 1024;     // flagged neurons of the token so far
-constexpr int CTL_WORDS = 1056;
+constexpr int CTL_TICKET = 0;     // [32] stride 32: next output tile of a channel chunk of the folded matrix
+constexpr int CTL_DONE = 1024;    // CTAs that have added all their contributions
+constexpr int CTL_NFL = 1056;     // flagged neurons of the token so far
+constexpr int CTL_WORDS = 1088;
 
 struct Params {
   const uint8_t* pblocks;  // [tile][kchunk] predictor blocks
@@ -74,7 +74,7 @@ struct Params {
   int tiles_max;
   int nvec, cw;            // 8-column vectors in a row; vectors per warp
   int nunits;              // folded-matrix units in all
-  int ntk;                 // folded-matrix units (16 outputs x 256 channels) per warp index
+  int ntk;                 // output tiles of the folded matrix (16 outputs each)
   int pre_chunks;          // chunks a second-half CTA takes before its predictor
 };
 
@@ -169,7 +169,7 @@ struct SmemLayout {
     const size_t rows = size_t(tiles_max) * 16;
     pbuf = take(size_t(nbuf) * unit_bytes, 128);
     xq = take(size_t(4) * (dpad + 64), 128);
-    xh = take(size_t(dpad) * 2, 16);
+    xh = take(size_t(dpad + 16) * 2, 16);     // + 16 zeros: the B operand of lanes that feed the unused columns
     sxi = take(size_t(ngroups + 16) * sizeof(int), 8);
     zpart = take(rows * NW * sizeof(double), 8);
     wpart = take(size_t(16) * NW * sizeof(float), 4);
@@ -248,6 +248,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < 48) misc[tid] = 0;
+  if (tid < 8) reinterpret_cast<uint32_t*>(xh + p.dpad)[tid] = 0u;
   __syncthreads();
   // predictor blocks first: nothing of them depends on x
   if (lane == 0 && warp < p.nbuf && warp < NU) issue_unit(warp);
@@ -381,13 +382,14 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
 
   // ---- speculative folded product on the tensor cores ----
   // The folded matrix is stored in units of 16 outputs x 256 channels (8 KB, contiguous, already in
-  // A-fragment order).  A warp draws units from the ticket of its warp index, streams a unit as four
-  // blocks of four 128-bit loads per lane (one block ahead of the one being multiplied), multiplies it
-  // with x (the B operand: column 0 = x, other columns zero) in two independent accumulators, and adds
-  // the 16 partial outputs to the accumulator replica of its CTA.  stream_c(n) takes at most n units.
+  // A-fragment order).  Warp w works on channel chunk w (and w + 16, ...) and draws the output tiles from
+  // the ticket of its warp index; it streams a unit as four blocks of four 128-bit loads per lane (one
+  // block ahead of the one being multiplied), multiplies it with x (the B operand: column 0 = x, other
+  // columns zero) in two independent accumulators, and adds the 16 partial outputs to the accumulator
+  // replica of its CTA.  stream_c(n) takes at most n tickets.
   float* const rep = p.yacc + size_t(blockIdx.x % NREP) * p.dacc;
   auto stream_c = [&](int budget) {
-    unsigned int* ticket = p.ctl + CTL_TICKET + warp * 32;
+    unsigned int* ticket = p.ctl + CTL_TICKET;
     auto issue = [&]() -> unsigned int {        // lane 0 draws; the value is looked at one unit later
       unsigned int t = 0;
       if (lane == 0) t = atomicAdd(ticket, 1u);
@@ -395,52 +397,55 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     };
     auto resolve = [&](unsigned int raw) -> int {
       const unsigned int t = __shfl_sync(0xffffffffu, raw, 0);
-      return t < (unsigned int)p.ntk && int(t * NW + warp) < p.nunits ? int(t * NW + warp) : -1;
+      return t < (unsigned int)p.ntk ? int(t) : -1;
     };
-    auto load = [&](uint4 (&buf)[4], int u, int bi) {
-      const uint4* src = p.Cp + (size_t(u) * 16 + bi * 4) * 32 + lane;
+    for (int kc = warp; kc < p.nkc; kc += NW) {
+      ticket = p.ctl + CTL_TICKET + kc * 32;
+      // lanes of column 0 read x, the others the zeros behind it
+      const uint4* xp = reinterpret_cast<const uint4*>(g == 0 ? xh + kc * KC + t4 * 16 : xh + p.dpad);
+      const int xstep = g == 0 ? 8 : 0;                 // uint4 per 64-channel block
+      const uint4* cbase = p.Cp + size_t(kc) * 512 + lane;
+      const size_t tstride = size_t(p.nkc) * 512;       // uint4 per output tile
+      auto load = [&](uint4 (&buf)[4], int it, int bi) {
+        const uint4* src = cbase + size_t(it) * tstride + bi * 128;
 #pragma unroll
-      for (int m = 0; m < 4; ++m) buf[m] = ldg_stream(src + m * 32);
-    };
-    auto multiply = [&](float (&c)[2][4], const uint4 (&buf)[4], int u, int bi) {
-      uint4 x0 = make_uint4(0u, 0u, 0u, 0u), x1 = x0;
-      if (g == 0) {
-        const uint4* xp = reinterpret_cast<const uint4*>(xh + (u % p.nkc) * KC + bi * 64 + t4 * 16);
-        x0 = xp[0]; x1 = xp[1];
-      }
-      mma_bf16(c[0], buf[0].x, buf[0].y, buf[0].z, buf[0].w, x0.x, x0.y);
-      mma_bf16(c[1], buf[1].x, buf[1].y, buf[1].z, buf[1].w, x0.z, x0.w);
-      mma_bf16(c[0], buf[2].x, buf[2].y, buf[2].z, buf[2].w, x1.x, x1.y);
-      mma_bf16(c[1], buf[3].x, buf[3].y, buf[3].z, buf[3].w, x1.z, x1.w);
-    };
-    uint4 ba[4], bb[4];
-    int u = budget > 0 ? resolve(issue()) : -1;
-    --budget;
-    bool more = u >= 0 && budget > 0;
-    unsigned int raw = more ? issue() : 0xffffffffu;
-    if (u >= 0) load(ba, u, 0);
-    while (u >= 0) {
-      float c[2][4];
-#pragma unroll
-      for (int m = 0; m < 2; ++m) c[m][0] = c[m][1] = c[m][2] = c[m][3] = 0.f;
-      load(bb, u, 1);
-      multiply(c, ba, u, 0);
-      load(ba, u, 2);
-      multiply(c, bb, u, 1);
-      load(bb, u, 3);
-      multiply(c, ba, u, 2);
-      const int un = more ? resolve(raw) : -1;        // the next unit: its first block goes in flight now
+        for (int m = 0; m < 4; ++m) buf[m] = ldg_stream(src + m * 32);
+      };
+      auto multiply = [&](float (&c)[2][4], const uint4 (&buf)[4], int bi) {
+        const uint4 x0 = xp[bi * xstep], x1 = xp[bi * xstep + 1];
+        mma_bf16(c[0], buf[0].x, buf[0].y, buf[0].z, buf[0].w, x0.x, x0.y);
+        mma_bf16(c[1], buf[1].x, buf[1].y, buf[1].z, buf[1].w, x0.z, x0.w);
+        mma_bf16(c[0], buf[2].x, buf[2].y, buf[2].z, buf[2].w, x1.x, x1.y);
+        mma_bf16(c[1], buf[3].x, buf[3].y, buf[3].z, buf[3].w, x1.z, x1.w);
+      };
+      uint4 ba[4], bb[4];
+      int it = budget > 0 ? resolve(issue()) : -1;
       --budget;
-      more = un >= 0 && budget > 0;
-      raw = more ? issue() : 0xffffffffu;
-      if (un >= 0) load(ba, un, 0);
-      multiply(c, bb, u, 3);
-      if (t4 == 0) {
-        const int i0 = (u / p.nkc) * 16 + g;
-        red_add_f32(rep + i0, c[0][0] + c[1][0]);
-        red_add_f32(rep + i0 + 8, c[0][2] + c[1][2]);
+      bool more = it >= 0 && budget > 0;
+      unsigned int raw = more ? issue() : 0xffffffffu;
+      if (it >= 0) load(ba, it, 0);
+      while (it >= 0) {
+        float c[2][4];
+#pragma unroll
+        for (int m = 0; m < 2; ++m) c[m][0] = c[m][1] = c[m][2] = c[m][3] = 0.f;
+        load(bb, it, 1);
+        multiply(c, ba, 0);
+        load(ba, it, 2);
+        multiply(c, bb, 1);
+        load(bb, it, 3);
+        multiply(c, ba, 2);
+        const int nx = more ? resolve(raw) : -1;        // the next tile: its first block goes in flight now
+        --budget;
+        more = nx >= 0 && budget > 0;
+        raw = more ? issue() : 0xffffffffu;
+        if (nx >= 0) load(ba, nx, 0);
+        multiply(c, bb, 3);
+        if (t4 == 0) {
+          red_add_f32(rep + it * 16 + g, c[0][0] + c[1][0]);
+          red_add_f32(rep + it * 16 + g + 8, c[0][2] + c[1][2]);
+        }
+        it = nx;
       }
-      u = un;
     }
   };
 
@@ -453,15 +458,14 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   {
     long long zacc[4] = {0, 0, 0, 0}, zt[2] = {0, 0};
     const int gpc = KC / p.G;                                // groups per chunk: 4 or 2
+    int b = 0, tl = 0, r = 0;                                // buffer, tile and chunk range of unit u
+    uint32_t par = 0u;                                       // phase of the buffer's barrier
     for (int u = 0; u < NU; ++u) {
-      const int b = u % p.nbuf;
-      const uint32_t par = uint32_t(u / p.nbuf) & 1u;
       bool landed = mbar_wait(&full[b], par);
       if (!landed) {                                 // record, give the copy one more bounded wait, skip the work
         if (lane == 0) { atomicExch(&p.counters[CTR_ERROR], 1ull); misc[MS_ERR] = 1; }
         landed = mbar_wait(&full[b], par);
       }
-      const int tl = u / p.nranges, r = u - tl * p.nranges;
       const int nch = min(p.cpr, p.nkc - r * p.cpr);
       if (warp < nch && landed && !misc[MS_ERR]) {
         const int kc = r * p.cpr + warp;
@@ -511,8 +515,13 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       if (r == p.nranges - 1) {
         // limbs: lane t4 = 0 holds limbs 0,1 ; t4 = 1 holds limbs 2,3 (columns 4..7 are unused for one token)
         double v0 = 0.0, v1 = 0.0;
-        if (t4 == 0) { v0 = double(zacc[0]) + 256.0 * double(zacc[1]); v1 = double(zacc[2]) + 256.0 * double(zacc[3]); }
-        if (t4 == 1) { v0 = 65536.0 * (double(zacc[0]) + 256.0 * double(zacc[1])); v1 = 65536.0 * (double(zacc[2]) + 256.0 * double(zacc[3])); }
+        // |sums| < 2^47: adding them to the bit pattern of 2^52 + 2^51 and taking that constant off again converts exactly
+        const double d0 = __longlong_as_double(zacc[0] + 0x4338000000000000LL) - 6755399441055744.0;
+        const double d1 = __longlong_as_double(zacc[1] + 0x4338000000000000LL) - 6755399441055744.0;
+        const double d2 = __longlong_as_double(zacc[2] + 0x4338000000000000LL) - 6755399441055744.0;
+        const double d3 = __longlong_as_double(zacc[3] + 0x4338000000000000LL) - 6755399441055744.0;
+        if (t4 == 0) { v0 = d0 + 256.0 * d1; v1 = d2 + 256.0 * d3; }
+        if (t4 == 1) { v0 = 65536.0 * (d0 + 256.0 * d1); v1 = 65536.0 * (d2 + 256.0 * d3); }
         v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
         v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
         if (t4 == 0) {
@@ -522,7 +531,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         zacc[0] = zacc[1] = zacc[2] = zacc[3] = 0; zt[0] = zt[1] = 0;
       }
       // hand the buffer back: the last warp to leave it starts the copy of the unit that reuses it
-      if (u + p.nbuf < NU) {
+      if (u + p.nbuf < NU) {                             // (never with every unit resident from the start)
         __threadfence_block();
         __syncwarp();
         if (lane == 0) {
@@ -534,6 +543,8 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
           }
         }
       }
+      if (++b == p.nbuf) { b = 0; par ^= 1u; }
+      if (++r == p.nranges) { r = 0; ++tl; }
     }
   }
   __syncthreads();
@@ -754,7 +765,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         *reinterpret_cast<uint4*>(p.y + col[m]) = *reinterpret_cast<const uint4*>(o);
       }
     if (lane == 0) {
-      p.ctl[CTL_TICKET + warp * 32] = 0u;
+      for (int kc = warp; kc < p.nkc; kc += NW) p.ctl[CTL_TICKET + kc * 32] = 0u;
       if (warp == 0) {   // every CTA has arrived, so every CTA's flagged count is in
         p.ctl[CTL_DONE] = 0u;
         const unsigned int tot = atomicExch(&p.ctl[CTL_NFL], 0u);
@@ -869,7 +880,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   const int cw = (nvec + NW - 1) / NW;
   const int vpt = (cw + 31) / 32;
   const int dpad = (d + KC - 1) / KC * KC;
-  if (vpt > 2 || d < 64 || d % 16 || dpad > XVR * NTH * 8) return TARDIS_OK;
+  if (vpt > 2 || d < 64 || d % 16 || dpad > XVR * NTH * 8 || dpad / KC > 32) return TARDIS_OK;
   int max_smem = 0, sm_smem = 0;
   TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, H->device));
   TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, H->device));
@@ -887,7 +898,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   p.unit_bytes = p.cpr * p.pbs;
   p.nvec = nvec; p.cw = cw;
   p.nunits = (d / 16) * p.nkc;
-  p.ntk = (p.nunits + NW - 1) / NW;
+  p.ntk = d / 16;
   p.pre_chunks = 2;
   S->vpt = vpt;
   // two CTAs per SM when their shared memory fits (each CTA also reserves 1 KB), else one
