@@ -75,7 +75,6 @@ struct Params {
   int nvec, cw;            // 8-column vectors in a row; vectors per warp
   int nunits;              // folded-matrix units in all
   int ntk;                 // output tiles of the folded matrix (16 outputs each)
-  int pre_chunks;          // chunks a second-half CTA takes before its predictor
 };
 
 struct Scratch {           // handle-owned device memory of the fused path
@@ -226,15 +225,9 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     bulk_g2s(pbuf + size_t(b) * p.unit_bytes, p.pblocks + (size_t(plan.x + tl) * p.nkc + size_t(r) * p.cpr) * p.pbs, bytes, &full[b]);
   };
 
-  // x first: it heads the longest dependency chain of the kernel, so its loads go out before the
-  // predictor copies fill the memory queues
-  uint4 xw[XVR];
-#pragma unroll
-  for (int m = 0; m < XVR; ++m) {
-    const int v = tid + m * NTH;
-    xw[m] = make_uint4(0u, 0u, 0u, 0u);
-    if (v < p.nvec) xw[m] = *reinterpret_cast<const uint4*>(p.x + size_t(v) * 8);
-  }
+  // Programmatic dependent launch: the next launch in the stream may start its own prologue (everything
+  // up to its griddepcontrol.wait reads only the layer's constant state) while this one is still running.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // per-neuron tables of the CTA's rows
   float tl0 = 0.f, tl1 = 0.f, tl2 = 0.f, tl3 = 0.f, tl4 = 0.f;
   int tl5 = 0;
@@ -252,6 +245,17 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   __syncthreads();
   // predictor blocks first: nothing of them depends on x
   if (lane == 0 && warp < p.nbuf && warp < NU) issue_unit(warp);
+
+  // From here on the kernel touches what earlier work in the stream may still be writing (x, the
+  // scratch shared by the calls of one handle): wait until that work has completed and is visible.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  uint4 xw[XVR];
+#pragma unroll
+  for (int m = 0; m < XVR; ++m) {
+    const int v = tid + m * NTH;
+    xw[m] = make_uint4(0u, 0u, 0u, 0u);
+    if (v < p.nvec) xw[m] = *reinterpret_cast<const uint4*>(p.x + size_t(v) * 8);
+  }
 
   if (tid < plan.y * 16) {
     tab[tid] = tl0; tab[TR + tid] = tl1; tab[2 * TR + tid] = tl2; tab[3 * TR + tid] = tl3; tab[4 * TR + tid] = tl4; tab[5 * TR + tid] = __int_as_float(tl5);
@@ -386,9 +390,9 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   // the ticket of its warp index; it streams a unit as four blocks of four 128-bit loads per lane (one
   // block ahead of the one being multiplied), multiplies it with x (the B operand: column 0 = x, other
   // columns zero) in two independent accumulators, and adds the 16 partial outputs to the accumulator
-  // replica of its CTA.  stream_c(n) takes at most n tickets.
+  // replica of its CTA.
   float* const rep = p.yacc + size_t(blockIdx.x % NREP) * p.dacc;
-  auto stream_c = [&](int budget) {
+  auto stream_c = [&]() {
     unsigned int* ticket = p.ctl + CTL_TICKET;
     auto issue = [&]() -> unsigned int {        // lane 0 draws; the value is looked at one unit later
       unsigned int t = 0;
@@ -419,9 +423,8 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         mma_bf16(c[1], buf[3].x, buf[3].y, buf[3].z, buf[3].w, x1.z, x1.w);
       };
       uint4 ba[4], bb[4];
-      int it = budget > 0 ? resolve(issue()) : -1;
-      --budget;
-      bool more = it >= 0 && budget > 0;
+      int it = resolve(issue());
+      bool more = it >= 0;
       unsigned int raw = more ? issue() : 0xffffffffu;
       if (it >= 0) load(ba, it, 0);
       while (it >= 0) {
@@ -435,8 +438,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         load(bb, it, 3);
         multiply(c, ba, 2);
         const int nx = more ? resolve(raw) : -1;        // the next tile: its first block goes in flight now
-        --budget;
-        more = nx >= 0 && budget > 0;
+        more = nx >= 0;
         raw = more ? issue() : 0xffffffffu;
         if (nx >= 0) load(ba, nx, 0);
         multiply(c, bb, 3);
@@ -448,11 +450,6 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       }
     }
   };
-
-  // CTAs of the second half of the grid (the ones that share an SM with a CTA of the first half) take a
-  // first share of the folded product before their predictor, so that the two CTAs of an SM are not in
-  // their memory-idle phases (scores, flags, compaction) at the same time.
-  if (blockIdx.x >= (gridDim.x >> 1) && p.pre_chunks > 0) stream_c(p.pre_chunks);
 
   // ---- predictor: warp w takes chunk w of every unit; partial scores of a tile go to shared memory ----
   {
@@ -717,7 +714,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   }
 
   // ---- the rest of the folded product ----
-  stream_c(0x7fffffff);
+  stream_c();
 
   // ---- combine: add this warp's columns to one replica; the last warp on a column range finishes it ----
   if (nfl > 0) {
@@ -899,7 +896,6 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   p.nvec = nvec; p.cw = cw;
   p.nunits = (d / 16) * p.nkc;
   p.ntk = d / 16;
-  p.pre_chunks = 2;
   S->vpt = vpt;
   // two CTAs per SM when their shared memory fits (each CTA also reserves 1 KB), else one
   bool placed = false;
@@ -922,7 +918,6 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   }
   if (!placed) { delete S; return TARDIS_OK; }
   const int grid = S->grid;
-  if (grid == H->num_sms) p.pre_chunks = 0;      // one CTA per SM: nothing to stagger
 
   auto fail = [&](tardis_status_t st) { H->dscratch = S; decode_release(H); return st; };
   size_t tally = 0;
@@ -985,11 +980,16 @@ tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, 
     p.y = static_cast<__nv_bfloat16*>(y) + size_t(t) * H->d;
     p.dbg_bitmap = H->dbg_bitmap ? H->dbg_bitmap + size_t(t) * (H->h / 32) : nullptr;
     p.dbg_scores = H->dbg_scores ? H->dbg_scores + size_t(t) * H->h : nullptr;
-    if (S->vpt == 1) k_decode<1><<<S->grid, NTH, S->smem_bytes, s>>>(p);
-    else k_decode<2><<<S->grid, NTH, S->smem_bytes, s>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S->grid); cfg.blockDim = dim3(NTH); cfg.dynamicSmemBytes = S->smem_bytes; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (S->vpt == 1) TARDIS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode<1>, p));
+    else TARDIS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode<2>, p));
     H->launches += 1;
   }
-  TARDIS_CUDA_TRY(cudaGetLastError());
   return TARDIS_OK;
 }
 
