@@ -310,12 +310,15 @@ def main():
                 "traffic": None, "peak_source": peak_src, "kernel": "k_decode" if B <= 8 else "generic",
                 "algorithmic_bytes_per_launch": alg, "avg_launch_us": dur_s * 1e6,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
-    prof = os.path.join(ROOT, "profiles", "k_decode_traffic.json")
-    if os.path.exists(prof):
-        try:
-            roofline["traffic"] = json.load(open(prof)).get(args.workload)
-        except Exception:
-            pass
+    # DRAM bytes per launch from the committed ncu summary of this kernel (null when there is none)
+    prof = os.path.join(ROOT, "profiles", "k_decode_%s.txt" % args.workload)
+    if B == 1 and os.path.exists(prof):
+        for line in open(prof):
+            if line.startswith("dram_bytes_per_launch:"):
+                try:
+                    roofline["traffic"] = float(line.split(":")[1].split()[0])
+                except Exception:
+                    pass
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),

@@ -16,18 +16,20 @@
 //     re-evaluated in fp64 from the original codes.  The 16 warps split the channel chunks of a
 //     tile; partial scores meet in shared memory.
 //   * Flags are compacted by ballot + prefix sum into the CTA's ascending list.
-//   * Every thread owns 8 output columns (per slot).  All remaining weight traffic is coalesced
-//     128-bit read-only loads kept several deep per thread.  For the CTA's flagged neurons a
-//     thread reads its slice of the W1 row (partial dot products meet through warp shuffles and
-//     shared memory to give the exact z_j), then its slice of the W2T row, scaled by
-//     delta_j = GELU(z_j) - a_j z_j - c_j, into its column accumulators.
-//   * The folded matrix C = W_f^T is handed out dynamically: each warp (owning a fixed column
-//     range in every CTA) draws row chunks from a global ticket of its column range, so CTAs
-//     with few flagged neurons take more of the folded product and all finish together.
-//   * Warps add their columns into one of several replicas of an fp32 accumulator (vector
-//     reductions; the replicas keep the number of reductions per address small); the last warp
-//     to arrive on a column range sums the replicas, adds b_f, rounds to bf16, and re-zeroes
-//     the scratch.
+//   * Result fixing, first half: the W1 rows of the CTA's flagged neurons are the A operand of bf16
+//     MMAs (16 flagged rows at a time, 128-bit read-only loads), x the B operand; the 16 warps split
+//     the channels and their partial z_j meet in shared memory, giving
+//     delta_j = GELU(z_j) - a_j z_j - c_j.  Second half: every thread owns 8 output columns (per
+//     slot) and adds delta_j times its slice of the W2T rows into fp32 column accumulators.
+//   * The speculative folded product runs on the bf16 tensor cores too: the fold leaves W_f in
+//     A-fragment order (units of 16 outputs x 256 channels, 8 KB, contiguous).  Warp w works on
+//     channel chunk w and draws output tiles from a global ticket of that chunk, so CTAs with few
+//     flagged neurons take more of the folded product and all finish together.
+//   * All partial outputs are added (red.global) into one of a few replicas of an fp32 accumulator
+//     (the replicas keep the number of reductions per address small).  CTAs count themselves when
+//     done; the last one sums the replicas, adds b_f, rounds to bf16, and re-zeroes the scratch.
+//   * The launch uses programmatic dependent launch: everything up to griddepcontrol.wait (tables,
+//     predictor copies) reads constant state only and overlaps the tail of the previous launch.
 #include <stdio.h>
 
 #include <vector>
