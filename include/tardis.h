@@ -147,6 +147,15 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
 tardis_status_t tardis_ffn_forward_static(tardis_handle_t handle, const void* x, void* y,
                                           int64_t n_tokens, tardis_stream_t stream);
 
+/* The dense product every batched step of the path is made of, on its own: C = A B^T with bf16 operands
+ * and fp32 accumulation on the tensor cores (the batched speculative product X W_f^T of Section 5.4, the
+ * fold W2 (diag(a) W1) of Section 5.2 and the batched pre-activations X W1^T all have this shape).
+ * A: device bf16 [M, K] row-major with leading dimension lda; B: device bf16 [N, K] row-major (ldb);
+ * C: device float [M, N] (ldc), fully overwritten.  K, lda, ldb multiples of 8; A, B 16-byte aligned.
+ * Asynchronous on `stream`.  Errors: INVALID_ARG, UNSUPPORTED (driver without tensor-map support), CUDA. */
+tardis_status_t tardis_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t lda,
+                                 const void* B, int32_t ldb, float* C, int32_t ldc, tardis_stream_t stream);
+
 /* Synchronises the stream of the handle's most recent call, then fills *out
  * (host memory).  Returns TIMEOUT / CORRUPT when the device error word says so. */
 tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out);

@@ -20,7 +20,7 @@ TARDIS_OK = 0
 TARDIS_F32, TARDIS_BF16 = 0, 1
 TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF = 0, 1
 
-EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_stats",
+EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy",
            "tardis_status_string", "tardis_last_error"]
 
@@ -73,7 +73,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_export_folded.argtypes = [vp, vp, vp, vp]
     lib.tardis_set_path.argtypes = [vp, i32]
     lib.tardis_destroy.argtypes = [vp]
-    for name in EXPORTS[:8]:
+    lib.tardis_gemm_bf16.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, i32, vp]
+    for name in EXPORTS[:9]:
         getattr(lib, name).restype = ctypes.c_int
     lib.tardis_status_string.argtypes = [ctypes.c_int]
     lib.tardis_status_string.restype = ctypes.c_char_p
@@ -143,6 +144,18 @@ def tardis_ffn_forward_static(handle: int, x: torch.Tensor, y: torch.Tensor, n_t
         raise TardisError(st, "tardis_ffn_forward_static: %s" % lib.tardis_last_error().decode())
     _check(st, "tardis_ffn_forward_static")
     return y
+
+
+def tardis_gemm_bf16(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, stream=None):
+    """C[M, N] (float32) = A[M, K] B[N, K]^T for bfloat16 row-major A, B (last stride 1)."""
+    lib = load_library()
+    M, K = A.shape
+    N = B.shape[0]
+    if A.stride(1) != 1 or B.stride(1) != 1 or C.stride(1) != 1 or not (A.is_cuda and B.is_cuda and C.is_cuda):
+        raise TardisError(1, "tensors must be CUDA tensors with unit inner stride")
+    _check(lib.tardis_gemm_bf16(M, N, K, A.data_ptr(), A.stride(0), B.data_ptr(), B.stride(0), C.data_ptr(), C.stride(0),
+                                _stream(stream)), "tardis_gemm_bf16")
+    return C
 
 
 def tardis_stats(handle: int) -> dict:

@@ -5,6 +5,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "gemm.cuh"
 
 namespace tardis {
 
@@ -151,6 +152,16 @@ tardis_status_t tardis_ffn_forward_static(tardis_handle_t handle, const void* x,
              "tardis_ffn_forward_static: n_tokens * (4 d_model + d_ff / 8) exceeds the 4 MiB of built-in scratch (or d_model > 12288)");
   if (st == TARDIS_OK) { H->last_path = 4; H->calls += 1; H->tokens += uint64_t(n_tokens); }
   return st;
+}
+
+tardis_status_t tardis_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t lda, const void* B, int32_t ldb,
+                                 float* C, int32_t ldc, tardis_stream_t stream) {
+  if (!A || !B || !C || M <= 0 || N <= 0 || K <= 0 || ldc < N) return TARDIS_ERR_INVALID_ARG;
+  GemmArgs g = {};
+  g.M = M; g.N = N; g.K1 = K; g.K2 = 0;
+  g.A1 = A; g.B1 = B; g.lda1 = lda; g.ldb1 = ldb;
+  g.epilogue = GEMM_EPI_F32; g.out_f32 = C; g.ldo = ldc;
+  return launch_gemm(g, reinterpret_cast<cudaStream_t>(stream));
 }
 
 tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
