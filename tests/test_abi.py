@@ -21,7 +21,7 @@ def lib():
 def test_header_symbols_exported(lib):
     hdr = open(os.path.join(ROOT, "include", "tardis.h")).read()
     hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    names = set(re.findall(r"\b(tardis_[a-z_]+)\s*\(", hdr))
+    names = set(re.findall(r"\b(tardis_[a-z0-9_]+)\s*\(", hdr))
     assert {"tardis_fold", "tardis_ffn_forward", "tardis_stats"} <= names
     for n in names:
         assert hasattr(lib, n), n
