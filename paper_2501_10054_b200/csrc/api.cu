@@ -39,6 +39,7 @@ static tardis_status_t dev_alloc(T** p, size_t count, size_t* tally) {
 
 static void free_all(Handle* H) {
   decode_release(H);
+  batched_release(H);
   void* ptrs[] = {H->W1, H->W2T, H->C, H->bf, H->lo, H->hi, H->a, H->c, H->b1, H->codes, H->scale,
                   H->zero, H->yacc, H->bitmap, H->counters};
   for (void* p : ptrs)
@@ -105,6 +106,7 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
 
   st = launch_fold(H, desc, s);
   if (st == TARDIS_OK && H->dtype == TARDIS_BF16) st = decode_prepare(H, s);
+  if (st == TARDIS_OK && H->dtype == TARDIS_BF16) st = batched_prepare(H, desc, s);
   if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
   *out = reinterpret_cast<tardis_handle_t>(H);
   return TARDIS_OK;
@@ -121,9 +123,13 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   H->last_stream = s;
   tardis_status_t st;
   const bool fused = H->path_override == 0 && H->codes_mma != nullptr && n_tokens <= kDecodeMaxTokens;
+  const bool batched = H->path_override == 0 && !fused && H->bstate != nullptr;
   if (fused) {
     st = launch_decode_forward(H, x, y, int(n_tokens), s);
     H->last_path = 2;
+  } else if (batched) {
+    st = launch_batched_forward(H, x, y, n_tokens, s);
+    H->last_path = 3;
   } else {
     st = launch_generic_forward(H, x, y, n_tokens, s);
     H->last_path = 1;

@@ -39,6 +39,7 @@ struct Handle {
   unsigned long long* counters;  // [CTR_COUNT]
   void* dscratch;        // fused decode scratch (see decode.cu)
   size_t dscratch_bytes;
+  void* bstate;          // batched / prefill state and scratch (see batched.cu); null when not built
   // debug capture (caller-owned)
   uint32_t* dbg_bitmap;
   double* dbg_scores;
@@ -69,6 +70,10 @@ tardis_status_t launch_static_forward(Handle* H, const void* x, void* y, int64_t
 tardis_status_t decode_prepare(Handle* H, cudaStream_t s);                 // builds codes_mma, pmeta, scratch
 tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
 void decode_release(Handle* H);
+tardis_status_t batched_prepare(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);   // bf16 only
+tardis_status_t launch_batched_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
+void batched_release(Handle* H);
+tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);  // bf16 fold on the tensor cores
 
 // ---- small device helpers ----
 template <typename T> __device__ __forceinline__ float to_f32(T v);

@@ -79,8 +79,10 @@ def assert_parity(layer, s, x, y_gpu, F_gpu, S_gpu, full_fold=True, folded=None,
     assert not mism.any(), "%s: %d flag mismatches outside the 1e-6 band (band holds %d)" % (label, mism.sum(), band.sum())
     if S_gpu is not None and score_tol is not None:
         fin = np.isfinite(ref["zhat"])
-        err = np.abs(S_gpu - ref["zhat"])[fin]
-        assert err.size == 0 or err.max() <= score_tol, "%s: score error %.3e" % (label, err.max())
+        tol = np.broadcast_to(np.asarray(score_tol, dtype=float).reshape(-1, 1) if np.ndim(score_tol) else score_tol, fin.shape)
+        err = np.abs(S_gpu - ref["zhat"])
+        bad = fin & (err > tol)
+        assert not bad.any(), "%s: score error %.3e" % (label, err[bad].max())
     rel = O.rel_error(y_gpu.double().cpu().numpy(), ref["y"])
     tol = TOL[layer.cfg.dtype]
     assert np.nanmax(rel) <= tol, "%s: max relative error %.3e > %.1e" % (label, np.nanmax(rel), tol)

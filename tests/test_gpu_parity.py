@@ -25,9 +25,14 @@ def _run(cfg, n, calls=None, seed=0, path=0, full_fold=True):
     try:
         T.tardis_set_path(h, path)
         y, F, S = Hp.gpu_forward(h, L, x, calls)
-        # generic kernels: exact fp64 score; fused kernel: exact up to the tracked truncation of tiny x elements
-        info = Hp.assert_parity(L, s, x, y, F, S, full_fold=full_fold, label=cfg.name,
-                                score_tol=1e-9 if path == 1 or cfg.dtype == "f32" else 5e-7)
+        # generic kernels: exact fp64 score; fused decode kernel (calls of up to 8 tokens): exact up to the tracked
+        # rounding of tiny x elements; batched path: fp32 tensor-core scores (flags are settled exactly near the
+        # range ends, the captured score is the fast one)
+        if path == 1 or cfg.dtype == "f32":
+            tol = 1e-9
+        else:
+            tol = np.concatenate([np.full(b, 5e-7 if b <= 8 else 3e-4) for b in (calls or [n])])
+        info = Hp.assert_parity(L, s, x, y, F, S, full_fold=full_fold, label=cfg.name, score_tol=tol)
         st = T.tardis_stats(h)
         assert st["tokens"] == n and st["device_error"] == 0
         assert st["flagged_total"] == int(F.sum())
