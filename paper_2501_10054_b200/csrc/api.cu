@@ -104,9 +104,16 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   A(&H->counters, size_t(CTR_COUNT), &H->bytes_scratch);
   if (st != TARDIS_OK) { free_all(H); return st; }
 
-  st = launch_fold(H, desc, s);
-  if (st == TARDIS_OK && H->dtype == TARDIS_BF16) st = decode_prepare(H, s);
-  if (st == TARDIS_OK && H->dtype == TARDIS_BF16) st = batched_prepare(H, desc, s);
+  const bool bf16 = H->dtype == TARDIS_BF16;
+  if (bf16) st = batched_prepare(H);                          // allocations; its buffers double as fold temporaries
+  const bool tensor_fold = st == TARDIS_OK && bf16 && H->bstate != nullptr;
+  if (st == TARDIS_OK) st = launch_fold(H, desc, s, tensor_fold);
+  if (st == TARDIS_OK && tensor_fold) {
+    st = launch_fold_tensor(H, desc, s);
+    if (st == TARDIS_ERR_UNSUPPORTED) st = launch_fold_product(H, s);   // no tensor-map support: plain kernel
+  }
+  if (st == TARDIS_OK && bf16) st = decode_prepare(H, s);
+  if (st == TARDIS_OK && bf16) st = batched_finish(H, desc, s);
   if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
   *out = reinterpret_cast<tardis_handle_t>(H);
   return TARDIS_OK;

@@ -231,7 +231,7 @@ template <typename T> __global__ void k_transpose_b(const T* __restrict__ in, T*
   }
 }
 
-tardis_status_t batched_prepare(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s) {
+tardis_status_t batched_prepare(Handle* H) {
   H->bstate = nullptr;
   if (H->dtype != TARDIS_BF16) return TARDIS_OK;
   const int d = H->d, h = H->h;
@@ -255,6 +255,83 @@ tardis_status_t batched_prepare(Handle* H, const tardis_fold_desc_t* desc, cudaS
     if (e != cudaSuccess) { set_last_error(e, "cudaMalloc"); cudaGetLastError(); batched_release(H); return TARDIS_ERR_ALLOC; }
     (r.scratch ? S->bytes_scratch : S->bytes_state) += r.bytes;
   }
+  H->bytes_folded += size_t(d) * d * 2;
+  H->bytes_w2t += hd * 2;                       // second copy of W2 (original orientation)
+  H->bytes_predictor += 2 * hd * 2 + size_t(h) * 4;
+  H->bytes_scratch += S->bytes_scratch;
+  return TARDIS_OK;
+}
+
+// a_j W1[j][k] in fp32, transposed to [k][j] and split into bf16 hi + lo (16 significant bits together)
+__global__ void k_scale_transpose_split(const __nv_bfloat16* __restrict__ W1, const float* __restrict__ a,
+                                        __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo, int h, int d) {
+  __shared__ float tile[32][33];
+  const int k0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int j = j0 + r, k = k0 + threadIdx.x;
+    if (j < h && k < d) tile[r][threadIdx.x] = a[j] * __bfloat162float(W1[size_t(j) * d + k]);
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int k = k0 + r, j = j0 + threadIdx.x;
+    if (j < h && k < d) {
+      const float v = tile[threadIdx.x][r];
+      const __nv_bfloat16 hv = __float2bfloat16_rn(v);
+      hi[size_t(k) * h + j] = hv;
+      lo[size_t(k) * h + j] = __float2bfloat16_rn(v - __bfloat162float(hv));
+    }
+  }
+}
+
+// rows [i0, i0 + rows) of W_f (fp32) rounded once to bf16 and stored as C[k][i]
+__global__ void k_store_folded(const float* __restrict__ Wf32, __nv_bfloat16* __restrict__ C, int i0, int rows, int d) {
+  __shared__ float tile[32][33];
+  const int k0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int ii = r0 + r, k = k0 + threadIdx.x;
+    if (ii < rows && k < d) tile[r][threadIdx.x] = Wf32[size_t(ii) * d + k];
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int k = k0 + r, ii = r0 + threadIdx.x;
+    if (ii < rows && k < d) C[size_t(k) * d + i0 + ii] = __float2bfloat16_rn(tile[threadIdx.x][r]);
+  }
+}
+
+// Constant folding (Section 5.2) on the tensor cores: W_f = W2 (diag(a) W1), with diag(a) W1 formed in fp32 and
+// carried as two bf16 matrices so that the product keeps 16 significant bits of it; fp32 accumulation over
+// all neurons, one rounding to bf16.  Uses the batched path's buffers as temporaries (they are filled later).
+tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s) {
+  State* S = static_cast<State*>(H->bstate);
+  if (!S || H->dtype != TARDIS_BF16) return TARDIS_ERR_UNSUPPORTED;
+  const int d = H->d, h = H->h;
+  dim3 tb(32, 8);
+  k_scale_transpose_split<<<dim3((d + 31) / 32, (h + 31) / 32), tb, 0, s>>>(static_cast<const __nv_bfloat16*>(H->W1), H->a,
+                                                                            S->What_hi, S->What_lo, h, d);
+  const size_t cap = size_t(kChunk) * h;                     // floats in the score buffer
+  int rows_per = int(cap / d);
+  rows_per = rows_per / 128 * 128;
+  if (rows_per < 128) return TARDIS_ERR_UNSUPPORTED;
+  for (int i0 = 0; i0 < d; i0 += rows_per) {
+    const int rows = d - i0 < rows_per ? d - i0 : rows_per;
+    GemmArgs g = {};
+    g.M = rows; g.N = d; g.K1 = h; g.K2 = h;
+    g.A1 = static_cast<const __nv_bfloat16*>(desc->W2) + size_t(i0) * h; g.lda1 = h; g.B1 = S->What_hi; g.ldb1 = h;
+    g.A2 = g.A1; g.lda2 = h; g.B2 = S->What_lo; g.ldb2 = h;
+    g.epilogue = GEMM_EPI_F32; g.out_f32 = S->zhat; g.ldo = d; g.error_word = &H->counters[CTR_ERROR];
+    const tardis_status_t st = launch_gemm(g, s);
+    if (st != TARDIS_OK) return st;
+    k_store_folded<<<dim3((d + 31) / 32, (rows + 31) / 32), tb, 0, s>>>(S->zhat, static_cast<__nv_bfloat16*>(H->C), i0, rows, d);
+  }
+  TARDIS_CUDA_TRY(cudaGetLastError());
+  return TARDIS_OK;
+}
+
+tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s) {
+  State* S = static_cast<State*>(H->bstate);
+  if (!S) return TARDIS_OK;
+  const int d = H->d, h = H->h;
+  const size_t hd = size_t(h) * d;
   dim3 tb(32, 8);
   // W_f[i][k] row-major (the GEMMs want the channel index contiguous in both operands): transpose of C
   k_transpose_b<__nv_bfloat16><<<dim3((d + 31) / 32, (d + 31) / 32), tb, 0, s>>>(static_cast<const __nv_bfloat16*>(H->C), S->Wf, d, d);
@@ -262,10 +339,6 @@ tardis_status_t batched_prepare(Handle* H, const tardis_fold_desc_t* desc, cudaS
   k_dequant_split<<<h, 256, 0, s>>>(H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, S->What_hi, S->What_lo,
                                     S->smaxrow, d, H->G);
   TARDIS_CUDA_TRY(cudaGetLastError());
-  H->bytes_folded += size_t(d) * d * 2;
-  H->bytes_w2t += hd * 2;                       // second copy of W2 (original orientation)
-  H->bytes_predictor += 2 * hd * 2 + size_t(h) * 4;
-  H->bytes_scratch += S->bytes_scratch;
   return TARDIS_OK;
 }
 

@@ -63,14 +63,16 @@ void set_last_error(cudaError_t e, const char* where);
   } while (0)
 
 // ---- kernels' host launchers (each returns after enqueueing on `s`) ----
-tardis_status_t launch_fold(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);
+tardis_status_t launch_fold(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s, bool skip_product = false);
+tardis_status_t launch_fold_product(Handle* H, cudaStream_t s);   // the SIMT product alone
 tardis_status_t launch_export_folded(Handle* H, void* Wf, float* bf, cudaStream_t s);
 tardis_status_t launch_generic_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
 tardis_status_t launch_static_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
 tardis_status_t decode_prepare(Handle* H, cudaStream_t s);                 // builds codes_mma, pmeta, scratch
 tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
 void decode_release(Handle* H);
-tardis_status_t batched_prepare(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);   // bf16 only
+tardis_status_t batched_prepare(Handle* H);                                                   // bf16 only: allocations
+tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);    // fills the batched state
 tardis_status_t launch_batched_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
 void batched_release(Handle* H);
 tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);  // bf16 fold on the tensor cores

@@ -100,11 +100,13 @@ __global__ void __launch_bounds__(256) k_fold_bias(const T* __restrict__ W2T, co
 }
 
 template <typename T>
-static tardis_status_t fold_typed(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s) {
+static tardis_status_t fold_typed(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s, bool skip_product) {
   const int d = H->d, h = H->h;
   dim3 tb(32, 8);
   k_transpose<T><<<dim3((h + 31) / 32, (d + 31) / 32), tb, 0, s>>>(static_cast<const T*>(desc->W2), static_cast<T*>(H->W2T), d, h);
-  if (sizeof(T) == 4) {
+  if (skip_product) {
+    // the caller forms the product on the tensor cores
+  } else if (sizeof(T) == 4) {
     constexpr int TM = 4;
     dim3 g((d + 16 * TM - 1) / (16 * TM), (d + 16 * TM - 1) / (16 * TM));
     k_fold_gemm<T, double, TM><<<g, dim3(16, 16), 0, s>>>(static_cast<const T*>(H->W1), static_cast<const T*>(H->W2T), H->a,
@@ -120,7 +122,7 @@ static tardis_status_t fold_typed(Handle* H, const tardis_fold_desc_t* desc, cud
   return TARDIS_OK;
 }
 
-tardis_status_t launch_fold(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s) {
+tardis_status_t launch_fold(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s, bool skip_product) {
   const size_t h = H->h, d = H->d, ng = H->ngroups;
   const cudaMemcpyKind D2D = cudaMemcpyDeviceToDevice;
   TARDIS_CUDA_TRY(cudaMemcpyAsync(H->W1, desc->W1, h * d * H->esize, D2D, s));
@@ -134,8 +136,20 @@ tardis_status_t launch_fold(Handle* H, const tardis_fold_desc_t* desc, cudaStrea
   TARDIS_CUDA_TRY(cudaMemcpyAsync(H->scale, desc->pred_scale, h * ng * H->esize, D2D, s));
   TARDIS_CUDA_TRY(cudaMemcpyAsync(H->zero, desc->pred_zero, h * ng, D2D, s));
   TARDIS_CUDA_TRY(cudaMemsetAsync(H->counters, 0, CTR_COUNT * sizeof(unsigned long long), s));
-  if (H->dtype == TARDIS_F32) return fold_typed<float>(H, desc, s);
-  return fold_typed<__nv_bfloat16>(H, desc, s);
+  if (H->dtype == TARDIS_F32) return fold_typed<float>(H, desc, s, skip_product);
+  return fold_typed<__nv_bfloat16>(H, desc, s, skip_product);
+}
+
+tardis_status_t launch_fold_product(Handle* H, cudaStream_t s) {
+  const int d = H->d, h = H->h;
+  if (H->dtype != TARDIS_BF16) return TARDIS_ERR_UNSUPPORTED;
+  constexpr int TM = 8;
+  dim3 g((d + 16 * TM - 1) / (16 * TM), (d + 16 * TM - 1) / (16 * TM));
+  k_fold_gemm<__nv_bfloat16, float, TM><<<g, dim3(16, 16), 0, s>>>(static_cast<const __nv_bfloat16*>(H->W1),
+                                                                   static_cast<const __nv_bfloat16*>(H->W2T), H->a,
+                                                                   static_cast<__nv_bfloat16*>(H->C), d, h);
+  TARDIS_CUDA_TRY(cudaGetLastError());
+  return TARDIS_OK;
 }
 
 tardis_status_t launch_export_folded(Handle* H, void* Wf, float* bf, cudaStream_t s) {

@@ -1,0 +1,79 @@
+"""Parity at the full sizes of the five benchmark configurations, in the launch shapes bench.py times
+(batch-1 decode, batched decode, prefill chunks).  The GPU runs every token; the oracle checks a seeded
+sample of them one by one through the direct definition of the partially linear FFN (no d x d fold
+needed), which equals the folded path by the pinned identities."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2501_10054_b200 as T
+import workloads as W
+from oracle import tardis_oracle as O
+from tests import helpers as Hp
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(cfg, batches, sample_per_call, seed=0, fold_rows=8):
+    dev = torch.device("cuda", 0)
+    L = W.make_layer(cfg, seed, device=dev)
+    s = L.numpy64()
+    n = sum(batches)
+    x = W.make_tokens(cfg, n, seed, device=dev)
+    h = T.fold_layer(L)
+    rng = np.random.default_rng(seed)
+    try:
+        # fold: sampled rows of W_f against the oracle (one bf16 rounding of an fp32-accumulated product)
+        d = cfg.d_model
+        Wf = torch.empty(d, d, dtype=x.dtype, device=dev)
+        bf = torch.empty(d, dtype=torch.float32, device=dev)
+        T.tardis_export_folded(h, Wf, bf)
+        torch.cuda.synchronize()
+        rows = np.sort(rng.choice(d, size=fold_rows, replace=False))
+        ref_rows = O.fold_rows(rows, s["W1"], s["W2"], s["a"])
+        got_rows = Wf[torch.as_tensor(rows, device=dev)].double().cpu().numpy()
+        scale = np.abs(ref_rows).max()
+        assert np.abs(got_rows - ref_rows).max() <= 2.0 ** -8 * scale
+        y, F, S = Hp.gpu_forward(h, L, x, batches)
+        st = T.tardis_stats(h)
+        assert st["device_error"] == 0 and st["tokens"] == n
+        assert st["flagged_total"] == int(F.sum())
+        # sampled tokens of every call
+        idx, t0 = [], 0
+        for b in batches:
+            k = min(b, sample_per_call)
+            idx += list(t0 + np.sort(rng.choice(b, size=k, replace=False)))
+            t0 += b
+        idx = np.asarray(idx)
+        xs = x[torch.as_tensor(idx, device=dev)]
+        info = Hp.assert_parity(L, s, xs, y[torch.as_tensor(idx, device=dev)], F[idx], None, full_fold=False,
+                                score_tol=None, label=cfg.name)
+        return info, float(F.mean())
+    finally:
+        T.tardis_destroy(h)
+        del L
+        torch.cuda.empty_cache()
+
+
+def test_decode_7b_batch1_and_batch64():
+    info, frac = _check(W.CONFIGS["decode_7b"], [1] * 6 + [64], sample_per_call=4)
+    assert 0.07 < frac < 0.13
+
+
+@pytest.mark.parametrize("q", [0, 2])
+def test_falcon_shape_decode_batches(q):
+    import dataclasses
+    qlo, qhi = W.FALCON_QUANTILES[q]
+    cfg = dataclasses.replace(W.CONFIGS["falcon_7b"], q_lo=qlo, q_hi=qhi)
+    info, frac = _check(cfg, [1, 1, 4, 16, 64], sample_per_call=3)
+    assert 0.02 < frac < 0.45
+
+
+def test_prefill_layer_2048_tokens():
+    info, frac = _check(W.CONFIGS["prefill_7b"], [2048], sample_per_call=12, seed=3)
+    assert 0.07 < frac < 0.13
+
+
+def test_large_8k_decode_and_prefill():
+    info, frac = _check(W.CONFIGS["large_8k"], [1, 1, 32, 1500], sample_per_call=3, fold_rows=4)
+    assert 0.07 < frac < 0.13
