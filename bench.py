@@ -341,8 +341,47 @@ def main():
         if NT % 64 == 0 and B != 64:
             s0 = [T.tardis_stats(hd) for hd in handles]
             ms64 = timed(make_step(64, x_all, y_all), max(3, args.steps // 4), 3)
+            u64 = h * (1 - (1 - flagged / h) ** 64)
+            alg64 = algorithmic_bytes(cfg, 64, u64)
+            gbs64 = alg64 / (ms64 * 1e-3 / (NT // 64)) / 1e9
             out["batch64"] = {"value": world * NT / (ms64 * 1e-3), "unit": UNIT, "ms_per_step": ms64,
-                              "path": T.tardis_stats(handles[0])["last_path"]}
+                              "path": T.tardis_stats(handles[0])["last_path"],
+                              "roofline": {"bound": "hbm", "achieved": gbs64, "peak": peak, "unit": "GB/s", "frac": gbs64 / peak,
+                                           "algorithmic_bytes_per_call": alg64}}
+
+        # prefill chunk of one layer through the batched path, and its folded GEMM alone against the bf16 peak
+        npre = 8192
+        xp = W.make_tokens(cfg, npre, seed=rank + 77, device=dev)
+        yp = torch.empty_like(xp)
+
+        def prefill_step():
+            st = fwd(handles[0], xp.data_ptr(), yp.data_ptr(), npre, sptr)
+            if st:
+                raise RuntimeError("tardis_ffn_forward status %d" % st)
+
+        msp = timed(prefill_step, 5, 3)
+        Wf = torch.empty(d, d, dtype=xp.dtype, device=dev)
+        T.tardis_export_folded(handles[0], Wf, None)
+        Cout = torch.empty(npre, d, dtype=torch.float32, device=dev)
+        msg = timed(lambda: T.tardis_gemm_bf16(xp, Wf, Cout), 10, 3)
+        tf = 2.0 * npre * d * d / (msg * 1e-3) / 1e12
+        tpeak = float(peaks.get("bf16_tflops", 1590.0))
+        out["prefill_context"] = {"tokens": npre, "value": world * npre / (msp * 1e-3), "unit": UNIT, "ms_per_chunk": msp,
+                                  "flops_per_token": 8 * d * h + 2 * d * d,
+                                  "wf_gemm": {"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak,
+                                              "ms": msg, "peak_source": "measured burst" if "bf16_tflops" in peaks else "fallback"}}
+        del xp, yp, Cout, Wf
+        # the offline fold of one layer (tensor-core product + predictor / folded-matrix packing)
+        Lf = W.make_layer(cfg, seed=rank * 1000 + 999, device=dev)
+        torch.cuda.synchronize()
+        ef0, ef1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ef0.record()
+        hf = T.fold_layer(Lf)
+        ef1.record()
+        torch.cuda.synchronize()
+        out["fold_ms_per_layer"] = ef0.elapsed_time(ef1)
+        T.tardis_destroy(hf)
+        del Lf
 
         def dense_step():
             for i in range(NT // B):
