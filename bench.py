@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--graph", type=int, default=0, help="replay one step as a CUDA graph")
     ap.add_argument("--no-context", action="store_true", help="skip the dense-FFN / batch-64 / oracle context legs")
     ap.add_argument("--cpu-sample-tokens", type=int, default=16)
+    ap.add_argument("--mode", default="decode", choices=["decode", "prefill"],
+                    help="prefill: time one prefill chunk of one layer through the batched path (a context run, not the headline)")
+    ap.add_argument("--prefill-tokens", type=int, default=8192)
     return ap.parse_args()
 
 
@@ -188,6 +191,9 @@ def main():
     lib = T.load_library()
 
     cfg = W.CONFIGS[args.workload]
+    if args.mode == "prefill":
+        run_prefill(args, cfg, T, W, torch, dev, rank, world)
+        return
     d, h, B, NT = cfg.d_model, cfg.d_ff, args.batch, args.tokens
     assert NT % B == 0
     # ---- set-up: independent layers (weak scaling: every rank has its own layers and tokens) ----
@@ -410,6 +416,47 @@ def main():
         T.tardis_destroy(hd)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_prefill(args, cfg, T, W, torch, dev, rank, world):
+    """One layer, one chunk of --prefill-tokens tokens per step through the batched path (tcgen05 GEMMs)."""
+    d, h, n = cfg.d_model, cfg.d_ff, args.prefill_tokens
+    L = W.make_layer(cfg, seed=rank * 1000, device=dev)
+    hd = T.fold_layer(L)
+    x = W.make_tokens(cfg, n, seed=rank + 77, device=dev)
+    y = torch.empty_like(x)
+    for _ in range(max(3, args.warmup)):
+        T.tardis_ffn_forward(hd, x, y)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps = max(1, args.steps)
+    e0.record()
+    for _ in range(steps):
+        T.tardis_ffn_forward(hd, x, y)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    st = T.tardis_stats(hd)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    tpeak = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    flops = float(n) * (8 * d * h + 2 * d * d)
+    tf = flops / (ms * 1e-3) / 1e12
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": world * n / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": "%s prefill chunk, d_model=%d d_ff=%d, %d tokens/step (one layer)" % (cfg.name, d, h, n),
+                       "flagged_frac": st["flagged_total"] / max(1, st["tokens"]) / h, "l2": "inputs larger than L2"},
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None,
+                         "peak_source": "measured sustained" if "bf16_tflops_sustained" in peaks else "fallback",
+                         "kernel": "k_gemm (4 products per chunk: scores hi+lo, folded, pre-activations, output)",
+                         "flops_per_step": flops}}))
+    T.tardis_destroy(hd)
 
 
 class _Null:
