@@ -118,48 +118,35 @@ __device__ double exact_score_single(const uint32_t* __restrict__ codes, const _
   return acc;
 }
 
-// One thread per (token, word of 32 neurons): flags from the fast scores; scores too close to a range end
-// are queued for exact re-evaluation (their bit is settled there).
+// One thread per (token, neuron), one warp per flag word: flags from the fast scores; scores too close to a
+// range end are queued for exact re-evaluation (their bit is settled there).
 __global__ void k_flags(const float* __restrict__ zhat, const float* __restrict__ lo, const float* __restrict__ hi,
                         const float* __restrict__ smaxrow, const float* __restrict__ x1, int n, int h,
                         uint32_t* __restrict__ bitmap, uint2* __restrict__ rlist, unsigned int* __restrict__ rcount,
                         const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
                         const uint8_t* __restrict__ zero, const float* __restrict__ b1,
                         const __nv_bfloat16* __restrict__ x, int d, int G) {
-  const int words = h / 32;
-  const size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (e >= size_t(n) * words) return;
-  const int t = int(e / words), w = int(e % words);
+  const size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x;     // n * h is a multiple of the block size
+  if (e >= size_t(n) * h) return;
+  const int t = int(e / h), j = int(e - size_t(t) * h);
   const float xn = x1[t];
-  uint32_t word = 0u;
-  if (!(xn <= 3.0e38f)) {
-    word = 0xffffffffu;                                      // non-finite token
-  } else {
-    const float4* z4 = reinterpret_cast<const float4*>(zhat + size_t(t) * h + w * 32);
-    for (int q = 0; q < 8; ++q) {
-      const float4 z = z4[q];
-      const float zs[4] = {z.x, z.y, z.z, z.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int j = w * 32 + q * 4 + i;
-        const float l = lo[j], u = hi[j];
-        const float tau = kEps * 3.f * smaxrow[j] * xn + 1e-30f;
-        const bool inside = (l <= zs[i]) && (zs[i] < u);
-        if (!inside) word |= 1u << (q * 4 + i);
-        if (fabsf(zs[i] - l) <= tau || fabsf(zs[i] - u) <= tau) {
-          const unsigned int slot = atomicAdd(&rcount[0], 1u);
-          if (slot < (unsigned int)kMaxRecheck) rlist[slot] = make_uint2((unsigned int)t, (unsigned int)j);
-          else {                                             // queue full: settle this one here (slow, but exact)
-            const double ze = exact_score_single(codes, scale, zero, x + size_t(t) * d, j, d, G) + double(b1[j]);
-            const bool in2 = (double(l) <= ze) && (ze < double(u));
-            if (in2) word &= ~(1u << (q * 4 + i)); else word |= 1u << (q * 4 + i);
-            atomicAdd(&rcount[1], 1u);
-          }
-        }
+  bool flag = true;                                                    // non-finite token: every neuron flagged
+  if (xn <= 3.0e38f) {
+    const float z = zhat[e], l = lo[j], u = hi[j];
+    const float tau = kEps * 3.f * smaxrow[j] * xn + 1e-30f;
+    flag = !((l <= z) && (z < u));
+    if (fabsf(z - l) <= tau || fabsf(z - u) <= tau) {
+      const unsigned int slot = atomicAdd(&rcount[0], 1u);
+      if (slot < (unsigned int)kMaxRecheck) rlist[slot] = make_uint2((unsigned int)t, (unsigned int)j);
+      else {                                                           // queue full: settle this one here (slow, but exact)
+        const double ze = exact_score_single(codes, scale, zero, x + size_t(t) * d, j, d, G) + double(b1[j]);
+        flag = !((double(l) <= ze) && (ze < double(u)));
+        atomicAdd(&rcount[1], 1u);
       }
     }
   }
-  bitmap[e] = word;
+  const uint32_t word = __ballot_sync(0xffffffffu, flag);
+  if ((threadIdx.x & 31) == 0) bitmap[e >> 5] = word;
 }
 
 // One warp per queued pair: exact fp64 score from the packed codes decides the flag.
@@ -370,8 +357,8 @@ tardis_status_t launch_batched_forward(Handle* H, const void* xv, void* yv, int6
     g.epilogue = GEMM_EPI_F32; g.out_f32 = S->zhat; g.ldo = h; g.bias = H->b1; g.error_word = &H->counters[CTR_ERROR];
     tardis_status_t st = launch_gemm(g, s);
     if (st != TARDIS_OK) return st;
-    const size_t nw = size_t(n) * (h / 32);
-    k_flags<<<unsigned((nw + 127) / 128), 128, 0, s>>>(S->zhat, H->lo, H->hi, S->smaxrow, S->x1, n, h, S->bitmap, S->rlist, S->rcount,
+    const size_t ne = size_t(n) * h;
+    k_flags<<<unsigned((ne + 255) / 256), 256, 0, s>>>(S->zhat, H->lo, H->hi, S->smaxrow, S->x1, n, h, S->bitmap, S->rlist, S->rcount,
                                                        H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, H->b1, xc, d, H->G);
     k_recheck<<<H->num_sms * 4, 256, 0, s>>>(S->rlist, S->rcount, H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, H->b1,
                                              H->lo, H->hi, xc, d, h, H->G, S->bitmap, S->zhat, H->counters);

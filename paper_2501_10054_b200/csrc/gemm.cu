@@ -213,24 +213,42 @@ k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtenso
             } else {
               for (int i = 0; i < nv; ++i) o[i] = v[i] + (p.bias ? p.bias[n + i] : 0.f);
             }
-          } else if (p.epilogue == GEMM_EPI_ADD_BF16) {
-            const float* ad = p.addend + size_t(m) * p.ldo + n;
-            __nv_bfloat16* o = p.out_bf16 + size_t(m) * p.ldo + n;
-#pragma unroll 8
-            for (int i = 0; i < 32; ++i)
-              if (i < nv) o[i] = __float2bfloat16_rn(v[i] + ad[i]);
-          } else {   // GEMM_EPI_DELTA: one flag word covers this thread's 32 columns
-            const uint32_t word = p.bitmap[size_t(m) * (p.N / 32) + (n >> 5)];
-            __nv_bfloat16* o = p.out_bf16 + size_t(m) * p.ldo + n;
-#pragma unroll 8
-            for (int i = 0; i < 32; ++i) {
-              if (i >= nv) break;
-              float dl = 0.f;
-              if ((word >> i) & 1u) {
-                const float z = v[i] + (p.bias ? p.bias[n + i] : 0.f);
-                dl = gelu_f32(z, p.act) - p.a[n + i] * z - p.c[n + i];
+          } else {
+            // bf16 outputs: this thread's 32 values become four 16-byte stores
+            if (p.epilogue == GEMM_EPI_ADD_BF16) {
+              const float* ad = p.addend + size_t(m) * p.ldo + n;
+              if (nv == 32 && (p.ldo & 3) == 0) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                  const float4 t = *reinterpret_cast<const float4*>(ad + i);
+                  v[i] += t.x; v[i + 1] += t.y; v[i + 2] += t.z; v[i + 3] += t.w;
+                }
+              } else {
+                for (int i = 0; i < nv; ++i) v[i] += ad[i];
               }
-              o[i] = __float2bfloat16_rn(dl);
+            } else {   // GEMM_EPI_DELTA: one flag word covers this thread's 32 columns
+              const uint32_t word = p.bitmap[size_t(m) * (p.N / 32) + (n >> 5)];
+#pragma unroll 8
+              for (int i = 0; i < 32; ++i) {
+                float dl = 0.f;
+                if (((word >> i) & 1u) && i < nv) {
+                  const float z = v[i] + (p.bias ? p.bias[n + i] : 0.f);
+                  dl = gelu_f32(z, p.act) - p.a[n + i] * z - p.c[n + i];
+                }
+                v[i] = dl;
+              }
+            }
+            __nv_bfloat16* o = p.out_bf16 + size_t(m) * p.ldo + n;
+            if (nv == 32 && (p.ldo & 7) == 0) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 8) {
+                __nv_bfloat162 h[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) h[q] = __floats2bfloat162_rn(v[i + 2 * q], v[i + 2 * q + 1]);
+                *reinterpret_cast<uint4*>(o + i) = *reinterpret_cast<const uint4*>(h);
+              }
+            } else {
+              for (int i = 0; i < nv; ++i) o[i] = __float2bfloat16_rn(v[i]);
             }
           }
         }
