@@ -189,6 +189,17 @@ __global__ void k_flag_counts(const uint32_t* __restrict__ bitmap, int words, un
   }
 }
 
+__global__ void k_round_store(const float* __restrict__ yacc, __nv_bfloat16* __restrict__ y, size_t count) {
+  const size_t e = (size_t(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
+  if (e + 3 < count) {
+    const float4 v = *reinterpret_cast<const float4*>(yacc + e);
+    __nv_bfloat162 o[2] = {__floats2bfloat162_rn(v.x, v.y), __floats2bfloat162_rn(v.z, v.w)};
+    *reinterpret_cast<uint2*>(y + e) = *reinterpret_cast<const uint2*>(o);
+  } else {
+    for (size_t i = e; i < count; ++i) y[i] = __float2bfloat16_rn(yacc[i]);
+  }
+}
+
 __global__ void k_capture(const uint32_t* __restrict__ bitmap, const float* __restrict__ zhat, const float* __restrict__ x1,
                           int n, int h, uint32_t* __restrict__ dbg_bitmap, double* __restrict__ dbg_scores) {
   const size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -369,10 +380,15 @@ tardis_status_t launch_batched_forward(Handle* H, const void* xv, void* yv, int6
                                                             H->dbg_bitmap ? H->dbg_bitmap + size_t(t0) * (h / 32) : nullptr,
                                                             H->dbg_scores ? H->dbg_scores + size_t(t0) * h : nullptr);
     }
+    // A batch of one tile of tokens is bound by weight traffic and its products over d outputs have few
+    // tiles: those split their channel range over several CTAs, which add into the fp32 accumulator.
+    const int splits = (n <= 128 && d <= 8192) ? 4 : 1;
     // 2. speculative folded product
     GemmArgs f = {};
     f.M = n; f.N = d; f.K1 = d; f.A1 = xc; f.lda1 = d; f.B1 = S->Wf; f.ldb1 = d;
     f.epilogue = GEMM_EPI_F32; f.out_f32 = S->yacc; f.ldo = d; f.bias = H->bf; f.error_word = &H->counters[CTR_ERROR];
+    f.splits = splits;
+    if (splits > 1) TARDIS_CUDA_TRY(cudaMemsetAsync(S->yacc, 0, size_t(n) * d * sizeof(float), s));
     st = launch_gemm(f, s);
     if (st != TARDIS_OK) return st;
     // 3. result fixing: exact pre-activations of every neuron, masked correction, output product
@@ -383,10 +399,18 @@ tardis_status_t launch_batched_forward(Handle* H, const void* xv, void* yv, int6
     st = launch_gemm(z, s);
     if (st != TARDIS_OK) return st;
     GemmArgs o = {};
-    o.M = n; o.N = d; o.K1 = h; o.A1 = S->delta; o.lda1 = h; o.B1 = S->W2; o.ldb1 = h;
-    o.epilogue = GEMM_EPI_ADD_BF16; o.out_bf16 = y + size_t(t0) * d; o.ldo = d; o.addend = S->yacc; o.error_word = &H->counters[CTR_ERROR];
+    o.M = n; o.N = d; o.K1 = h; o.A1 = S->delta; o.lda1 = h; o.B1 = S->W2; o.ldb1 = h; o.ldo = d; o.error_word = &H->counters[CTR_ERROR];
+    if (splits > 1) {
+      o.epilogue = GEMM_EPI_F32; o.out_f32 = S->yacc; o.splits = splits;
+    } else {
+      o.epilogue = GEMM_EPI_ADD_BF16; o.out_bf16 = y + size_t(t0) * d; o.addend = S->yacc;
+    }
     st = launch_gemm(o, s);
     if (st != TARDIS_OK) return st;
+    if (splits > 1) {
+      const size_t cnt = size_t(n) * d;
+      k_round_store<<<unsigned((cnt / 4 + 255) / 256 + 1), 256, 0, s>>>(S->yacc, y + size_t(t0) * d, cnt);
+    }
     H->launches += 9 + ((H->dbg_bitmap || H->dbg_scores) ? 1 : 0);
   }
   TARDIS_CUDA_TRY(cudaGetLastError());

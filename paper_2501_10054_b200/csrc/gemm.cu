@@ -100,7 +100,7 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N) {
 
 struct KParams {
   int M, N, kb1, kb2;          // k blocks (of 64) of the two operand pairs
-  int epilogue, ldo, act;
+  int epilogue, ldo, act, splits;
   float* out_f32; __nv_bfloat16* out_bf16;
   const float *bias, *addend, *a, *c;
   const uint32_t* bitmap;
@@ -128,7 +128,11 @@ k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtenso
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  const int nkb = p.kb1 + p.kb2;
+  // this CTA's share of the k blocks (all of them unless the launch splits the channel range)
+  const int nkb_all = p.kb1 + p.kb2;
+  const int per = (nkb_all + p.splits - 1) / p.splits;
+  const int kb_lo = blockIdx.z * per;
+  const int nkb = max(0, min(nkb_all, kb_lo + per) - kb_lo);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -153,8 +157,9 @@ k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtenso
         uint8_t* sa = smem + s * C::STAGE_BYTES;
         uint8_t* sb = sa + BM * BK * 2;
         mbar_expect_tx(&full[s], C::STAGE_BYTES);
-        const bool second = kb >= p.kb1;
-        const int kx = (second ? kb - p.kb1 : kb) * BK;
+        const int kg = kb_lo + kb;                   // k block in the whole channel range
+        const bool second = kg >= p.kb1;
+        const int kx = (second ? kg - p.kb1 : kg) * BK;
         tma_load_2d(sa, second ? &tmA2 : &tmA1, kx, m0, &full[s]);
         tma_load_2d(sb, second ? &tmB2 : &tmB1, kx, n0, &full[s]);
       }
@@ -201,7 +206,22 @@ k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtenso
         const int n = n0 + ch * 32;
         const int nv = min(32, p.N - n);
         if (m < p.M && nv > 0) {                      // (no early exit: the next tcgen05.ld needs the whole warp)
-          if (p.epilogue == GEMM_EPI_F32) {
+          if (p.epilogue == GEMM_EPI_F32 && p.splits > 1) {
+            float* o = p.out_f32 + size_t(m) * p.ldo + n;
+            const bool with_bias = p.bias && blockIdx.z == 0;
+            if (nkb > 0 || with_bias) {
+              if (nv == 32 && (p.ldo & 3) == 0) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                  float4 t = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                  if (with_bias) { t.x += p.bias[n + i]; t.y += p.bias[n + i + 1]; t.z += p.bias[n + i + 2]; t.w += p.bias[n + i + 3]; }
+                  asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + i), "f"(t.x), "f"(t.y), "f"(t.z), "f"(t.w) : "memory");
+                }
+              } else {
+                for (int i = 0; i < nv; ++i) atomicAdd(o + i, v[i] + (with_bias ? p.bias[n + i] : 0.f));
+              }
+            }
+          } else if (p.epilogue == GEMM_EPI_F32) {
             float* o = p.out_f32 + size_t(m) * p.ldo + n;
             if (nv == 32 && (p.ldo & 3) == 0) {
 #pragma unroll
@@ -303,11 +323,11 @@ static tardis_status_t launch_bn(const GemmArgs& g, cudaStream_t s) {
     return TARDIS_ERR_INVALID_ARG;
   KParams p;
   p.M = g.M; p.N = g.N; p.kb1 = (g.K1 + BK - 1) / BK; p.kb2 = g.K2 > 0 ? (g.K2 + BK - 1) / BK : 0;
-  p.epilogue = g.epilogue; p.ldo = g.ldo; p.act = g.act;
+  p.epilogue = g.epilogue; p.ldo = g.ldo; p.act = g.act; p.splits = g.splits > 1 ? g.splits : 1;
   p.out_f32 = g.out_f32; p.out_bf16 = static_cast<__nv_bfloat16*>(g.out_bf16);
   p.bias = g.bias; p.addend = g.addend; p.a = g.a; p.c = g.c; p.bitmap = g.bitmap; p.error_word = g.error_word;
   TARDIS_CUDA_TRY(cudaFuncSetAttribute(k_gemm<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM));
-  dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM);
+  dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, p.splits);
   k_gemm<BN><<<grid, NTHREADS, Cfg<BN>::SMEM, s>>>(a1, b1, a2, b2, p);
   TARDIS_CUDA_TRY(cudaGetLastError());
   return TARDIS_OK;
@@ -323,8 +343,9 @@ tardis_status_t launch_gemm(const GemmArgs& g, cudaStream_t s) {
   if (bad(g.A1, g.lda1, g.K1) || bad(g.B1, g.ldb1, g.K1)) return TARDIS_ERR_INVALID_ARG;
   if (g.K2 > 0 && (bad(g.A2, g.lda2, g.K2) || bad(g.B2, g.ldb2, g.K2))) return TARDIS_ERR_INVALID_ARG;
   if (g.epilogue == GEMM_EPI_DELTA && (g.N % 32)) return TARDIS_ERR_INVALID_ARG;
+  if (g.splits > 1 && g.epilogue != GEMM_EPI_F32) return TARDIS_ERR_INVALID_ARG;
   // wide tiles when they still fill the machine, narrow ones for skinny problems
-  const long tiles256 = long((g.N + 255) / 256) * ((g.M + BM - 1) / BM);
+  const long tiles256 = long((g.N + 255) / 256) * ((g.M + BM - 1) / BM) * (g.splits > 1 ? g.splits : 1);
   if (tiles256 >= 120) return launch_bn<256>(g, s);
   return launch_bn<128>(g, s);
 }

@@ -21,6 +21,8 @@ struct GemmArgs {
   const void *A1, *B1, *A2, *B2;    // device bf16; leading dimensions lda1 ... in elements (multiples of 8)
   int lda1, ldb1, lda2, ldb2;
   int epilogue;                     // GemmEpilogue
+  int splits;                       // > 1 (GEMM_EPI_F32 only): the channel range is split over that many CTAs per tile, which
+                                    // ADD their parts to out_f32 (the caller zeroes it first); the bias is added once
   float* out_f32; void* out_bf16;   // row-major, leading dimension ldo
   int ldo;
   const float* bias;                // [N] or null
