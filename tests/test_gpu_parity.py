@@ -146,3 +146,27 @@ def test_run_to_run_flags_identical():
     assert (F1 == F2).all() and np.abs(S1 - S2).max() <= 1e-4
     assert (y1.float() - y2.float()).abs().max() <= 2e-2 * y1.float().abs().max()
     T.tardis_destroy(h)
+
+
+def test_batched_path_chunk_boundary_nan_token_and_empty_ranges():
+    """More tokens than one scratch chunk (1024) in a single call, a token holding a NaN in the middle of it,
+    and the result compared token by token with the oracle on a seeded sample."""
+    cfg = W.LayerConfig("chunks", 256, 1024, n_calib=512)
+    L = _layer(cfg)
+    s = L.numpy64()
+    n = 1030
+    x = W.make_tokens(cfg, n, 4).cuda()
+    x[1027, 5] = float("nan")
+    h = T.fold_layer(L)
+    try:
+        y, F, S = Hp.gpu_forward(h, L, x, [n])
+        assert T.tardis_stats(h)["last_path"] == 3
+        assert F[1027].all() and torch.isnan(y[1027]).all()
+        keep = np.array([0, 1, 511, 1023, 1024, 1026, 1028, 1029])
+        assert not torch.isnan(y[torch.as_tensor(keep).cuda()]).any()
+        Hp.assert_parity(L, s, x[torch.as_tensor(keep).cuda()], y[torch.as_tensor(keep).cuda()], F[keep], S[keep],
+                         score_tol=3e-4, label="chunks")
+        st = T.tardis_stats(h)
+        assert st["flagged_total"] == int(F.sum()) and st["device_error"] == 0
+    finally:
+        T.tardis_destroy(h)
