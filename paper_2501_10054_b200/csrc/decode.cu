@@ -40,6 +40,7 @@ namespace tardis {
 namespace dec {
 
 constexpr int NW = 16;            // warps per CTA
+constexpr int NWP = 8;            // of them, warps that run the predictor -> flags -> fixing chain; the others only stream the folded matrix
 constexpr int NTH = NW * 32;      // threads per CTA
 constexpr int KC = 256;           // channels per predictor block
 constexpr int MAXTILES = 16;      // predictor tiles (of 16 neurons) per CTA
@@ -74,7 +75,7 @@ struct Params {
   int nranges, cpr;        // a tile's chunks are taken in nranges units of cpr chunks (cpr <= NW)
   int nbuf, unit_bytes;    // unit buffers in shared memory and their size
   int tiles_max;
-  int nvec, cw;            // 8-column vectors in a row; vectors per warp
+  int nvec, npass;         // 8-column vectors in a row; passes of the chain warps over them
   int nunits;              // folded-matrix units in all
   int ntk;                 // output tiles of the folded matrix (16 outputs each)
 };
@@ -186,7 +187,9 @@ struct SmemLayout {
     total = o;
   }
 };
-enum { MS_NFL = 0, MS_NRC = 1, MS_ERR = 2, MS_LAST = 3, MS_WCNT = 8, MS_BUFCNT = 32 };
+enum { MS_NFL = 0, MS_NRC = 1, MS_ERR = 2, MS_LAST = 3, MS_SDONE = 4, MS_WCNT = 8, MS_BUFCNT = 32 };
+// Named barrier of the chain warps (the streaming warps have left the CTA by then).
+__device__ __forceinline__ void chain_sync() { asm volatile("bar.sync 2, %0;" ::"n"(NWP * 32) : "memory"); }
 
 // ---- the kernel ---------------------------------------------------------------------------------------
 template <int VPT>
@@ -294,6 +297,73 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   int E = 0;
   if (amax_all > 0.f && !tok_nonfinite) E = max(int((__float_as_uint(amax_all) >> 23) & 0xff) - 127 - 21, -100);
 
+  // ---- speculative folded product on the tensor cores ----
+  // The folded matrix is stored in units of 16 outputs x 256 channels (8 KB, contiguous, already in
+  // A-fragment order).  A warp works on channel chunks first, first + step, ... and draws the output tiles from
+  // the global ticket of the chunk; it streams a unit as four blocks of four 128-bit loads per lane (one
+  // block ahead of the one being multiplied), multiplies it with x (the B operand: column 0 = x, other
+  // columns zero) in two independent accumulators, and adds the 16 partial outputs to the accumulator
+  // replica of its CTA.
+  float* const rep = p.yacc + size_t(blockIdx.x % NREP) * p.dacc;
+  auto stream_c = [&](int first, int step) {
+    unsigned int* ticket = p.ctl + CTL_TICKET;
+    auto issue = [&]() -> unsigned int {        // lane 0 draws; the value is looked at one unit later
+      unsigned int t = 0;
+      if (lane == 0) t = atomicAdd(ticket, 1u);
+      return t;
+    };
+    auto resolve = [&](unsigned int raw) -> int {
+      const unsigned int t = __shfl_sync(0xffffffffu, raw, 0);
+      return t < (unsigned int)p.ntk ? int(t) : -1;
+    };
+    for (int kc = first; kc < p.nkc; kc += step) {
+      ticket = p.ctl + CTL_TICKET + kc * 32;
+      // lanes of column 0 read x, the others the zeros behind it
+      const uint4* xp = reinterpret_cast<const uint4*>(g == 0 ? xh + kc * KC + t4 * 16 : xh + p.dpad);
+      const int xstep = g == 0 ? 8 : 0;                 // uint4 per 64-channel block
+      const uint4* cbase = p.Cp + size_t(kc) * 512 + lane;
+      const size_t tstride = size_t(p.nkc) * 512;       // uint4 per output tile
+      auto load = [&](uint4 (&buf)[4], int it, int bi) {
+        const uint4* src = cbase + size_t(it) * tstride + bi * 128;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) buf[m] = ldg_stream(src + m * 32);
+      };
+      auto multiply = [&](float (&c)[2][4], const uint4 (&buf)[4], int bi) {
+        const uint4 x0 = xp[bi * xstep], x1 = xp[bi * xstep + 1];
+        mma_bf16(c[0], buf[0].x, buf[0].y, buf[0].z, buf[0].w, x0.x, x0.y);
+        mma_bf16(c[1], buf[1].x, buf[1].y, buf[1].z, buf[1].w, x0.z, x0.w);
+        mma_bf16(c[0], buf[2].x, buf[2].y, buf[2].z, buf[2].w, x1.x, x1.y);
+        mma_bf16(c[1], buf[3].x, buf[3].y, buf[3].z, buf[3].w, x1.z, x1.w);
+      };
+      uint4 ba[4], bb[4];
+      int it = resolve(issue());
+      bool more = it >= 0;
+      unsigned int raw = more ? issue() : 0xffffffffu;
+      if (it >= 0) load(ba, it, 0);
+      while (it >= 0) {
+        float c[2][4];
+#pragma unroll
+        for (int m = 0; m < 2; ++m) c[m][0] = c[m][1] = c[m][2] = c[m][3] = 0.f;
+        load(bb, it, 1);
+        multiply(c, ba, 0);
+        load(ba, it, 2);
+        multiply(c, bb, 1);
+        load(bb, it, 3);
+        multiply(c, ba, 2);
+        const int nx = more ? resolve(raw) : -1;        // the next tile: its first block goes in flight now
+        more = nx >= 0;
+        raw = more ? issue() : 0xffffffffu;
+        if (nx >= 0) load(ba, nx, 0);
+        multiply(c, bb, 3);
+        if (t4 == 0) {
+          red_add_f32(rep + it * 16 + g, c[0][0] + c[1][0]);
+          red_add_f32(rep + it * 16 + g + 8, c[0][2] + c[1][2]);
+        }
+        it = nx;
+      }
+    }
+  };
+
   // ---- fixed-point limbs of x in tensor-core operand order; group sums; truncation residual ----
   // A thread holds 8 channels = half of a 16-channel unit; the two halves meet through one shuffle.
   {
@@ -366,7 +436,19 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     for (int o = 16; o > 0; o >>= 1) resid += __shfl_xor_sync(0xffffffffu, resid, o);
     if (lane == 0) wred[2 * NW + warp] = resid;
   }
-  __syncthreads();
+  // ---- roles ----
+  // The limbs are complete once all 16 warps have passed here.  The streaming warps only announce their part
+  // (bar.arrive) and go on to the folded product, which needs nothing but x; when the tickets run out they
+  // report to the CTA's counter and leave.  The chain warps wait for everybody's limbs (bar.sync).
+  if (warp >= NWP) {
+    asm volatile("bar.arrive 1, %0;" ::"n"(NTH) : "memory");
+    stream_c(warp - NWP, NW - NWP);
+    __threadfence();                               // the additions of this warp are visible before it reports
+    __syncwarp();
+    if (lane == 0) atomicAdd(const_cast<int*>(&misc[MS_SDONE]), 1);
+    return;
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(NTH) : "memory");
   // tolerance of the fast score: every rounding residual (<= 1/2 unit of 2^E) times |code - zero| <= 3 times the scale
   double tau;
   {
@@ -376,84 +458,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     tau = double(rs) * 1.001 * 3.0 * double(*p.smax) * ldexp(1.0, E);
   }
 
-  // ---- this thread's columns ----
-  int col[VPT];
-  bool cval[VPT];
-#pragma unroll
-  for (int m = 0; m < VPT; ++m) {
-    const int vl = m * 32 + lane, vec = warp * p.cw + vl;
-    cval[m] = vl < p.cw && vec < p.nvec;
-    col[m] = cval[m] ? vec * 8 : 0;
-  }
-
-  // ---- speculative folded product on the tensor cores ----
-  // The folded matrix is stored in units of 16 outputs x 256 channels (8 KB, contiguous, already in
-  // A-fragment order).  Warp w works on channel chunk w (and w + 16, ...) and draws the output tiles from
-  // the ticket of its warp index; it streams a unit as four blocks of four 128-bit loads per lane (one
-  // block ahead of the one being multiplied), multiplies it with x (the B operand: column 0 = x, other
-  // columns zero) in two independent accumulators, and adds the 16 partial outputs to the accumulator
-  // replica of its CTA.
-  float* const rep = p.yacc + size_t(blockIdx.x % NREP) * p.dacc;
-  auto stream_c = [&]() {
-    unsigned int* ticket = p.ctl + CTL_TICKET;
-    auto issue = [&]() -> unsigned int {        // lane 0 draws; the value is looked at one unit later
-      unsigned int t = 0;
-      if (lane == 0) t = atomicAdd(ticket, 1u);
-      return t;
-    };
-    auto resolve = [&](unsigned int raw) -> int {
-      const unsigned int t = __shfl_sync(0xffffffffu, raw, 0);
-      return t < (unsigned int)p.ntk ? int(t) : -1;
-    };
-    for (int kc = warp; kc < p.nkc; kc += NW) {
-      ticket = p.ctl + CTL_TICKET + kc * 32;
-      // lanes of column 0 read x, the others the zeros behind it
-      const uint4* xp = reinterpret_cast<const uint4*>(g == 0 ? xh + kc * KC + t4 * 16 : xh + p.dpad);
-      const int xstep = g == 0 ? 8 : 0;                 // uint4 per 64-channel block
-      const uint4* cbase = p.Cp + size_t(kc) * 512 + lane;
-      const size_t tstride = size_t(p.nkc) * 512;       // uint4 per output tile
-      auto load = [&](uint4 (&buf)[4], int it, int bi) {
-        const uint4* src = cbase + size_t(it) * tstride + bi * 128;
-#pragma unroll
-        for (int m = 0; m < 4; ++m) buf[m] = ldg_stream(src + m * 32);
-      };
-      auto multiply = [&](float (&c)[2][4], const uint4 (&buf)[4], int bi) {
-        const uint4 x0 = xp[bi * xstep], x1 = xp[bi * xstep + 1];
-        mma_bf16(c[0], buf[0].x, buf[0].y, buf[0].z, buf[0].w, x0.x, x0.y);
-        mma_bf16(c[1], buf[1].x, buf[1].y, buf[1].z, buf[1].w, x0.z, x0.w);
-        mma_bf16(c[0], buf[2].x, buf[2].y, buf[2].z, buf[2].w, x1.x, x1.y);
-        mma_bf16(c[1], buf[3].x, buf[3].y, buf[3].z, buf[3].w, x1.z, x1.w);
-      };
-      uint4 ba[4], bb[4];
-      int it = resolve(issue());
-      bool more = it >= 0;
-      unsigned int raw = more ? issue() : 0xffffffffu;
-      if (it >= 0) load(ba, it, 0);
-      while (it >= 0) {
-        float c[2][4];
-#pragma unroll
-        for (int m = 0; m < 2; ++m) c[m][0] = c[m][1] = c[m][2] = c[m][3] = 0.f;
-        load(bb, it, 1);
-        multiply(c, ba, 0);
-        load(ba, it, 2);
-        multiply(c, bb, 1);
-        load(bb, it, 3);
-        multiply(c, ba, 2);
-        const int nx = more ? resolve(raw) : -1;        // the next tile: its first block goes in flight now
-        more = nx >= 0;
-        raw = more ? issue() : 0xffffffffu;
-        if (nx >= 0) load(ba, nx, 0);
-        multiply(c, bb, 3);
-        if (t4 == 0) {
-          red_add_f32(rep + it * 16 + g, c[0][0] + c[1][0]);
-          red_add_f32(rep + it * 16 + g + 8, c[0][2] + c[1][2]);
-        }
-        it = nx;
-      }
-    }
-  };
-
-  // ---- predictor: warp w takes chunk w of every unit; partial scores of a tile go to shared memory ----
+  // ---- predictor: chain warp w takes chunks w, w + 8, ... of every unit; partial scores of a tile go to shared memory ----
   {
     long long zacc[4] = {0, 0, 0, 0}, zt[2] = {0, 0};
     const int gpc = KC / p.G;                                // groups per chunk: 4 or 2
@@ -466,9 +471,10 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         landed = mbar_wait(&full[b], par);
       }
       const int nch = min(p.cpr, p.nkc - r * p.cpr);
-      if (warp < nch && landed && !misc[MS_ERR]) {
-        const int kc = r * p.cpr + warp;
-        const uint8_t* blk = pbuf + size_t(b) * p.unit_bytes + size_t(warp) * p.pbs;
+      const bool usable = landed && !misc[MS_ERR];
+      for (int cc = warp; cc < nch && usable; cc += NWP) {
+        const int kc = r * p.cpr + cc;
+        const uint8_t* blk = pbuf + size_t(b) * p.unit_bytes + size_t(cc) * p.pbs;
         const uint4* cp = reinterpret_cast<const uint4*>(blk);
         const uint2* mp = reinterpret_cast<const uint2*>(blk + 1024);
         // group g2 of the chunk done: sums (|.| < 2^22) times the integer scales (|.| < 2^15), all exact
@@ -524,8 +530,8 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
         v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
         if (t4 == 0) {
-          zpart[(tl * NW + warp) * 16 + g] = v0 * (1.0 / 64.0) - double(zt[0]);
-          zpart[(tl * NW + warp) * 16 + g + 8] = v1 * (1.0 / 64.0) - double(zt[1]);
+          zpart[(tl * NWP + warp) * 16 + g] = v0 * (1.0 / 64.0) - double(zt[0]);
+          zpart[(tl * NWP + warp) * 16 + g + 8] = v1 * (1.0 / 64.0) - double(zt[1]);
         }
         zacc[0] = zacc[1] = zacc[2] = zacc[3] = 0; zt[0] = zt[1] = 0;
       }
@@ -535,7 +541,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         __syncwarp();
         if (lane == 0) {
           const int old = atomicAdd(const_cast<int*>(&misc[MS_BUFCNT + b]), 1);
-          if (old == NW - 1) {
+          if (old == NWP - 1) {
             misc[MS_BUFCNT + b] = 0;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             issue_unit(u + p.nbuf);
@@ -546,7 +552,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       if (++r == p.nranges) { r = 0; ++tl; }
     }
   }
-  __syncthreads();
+  chain_sync();
 
   // ---- scores, flags ----
   const int nrow = plan.y * 16;
@@ -555,7 +561,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     const int j = (plan.x + tl) * 16 + r;
     double s = 0.0;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) s += zpart[(tl * NW + w) * 16 + r];
+    for (int w = 0; w < NWP; ++w) s += zpart[(tl * NWP + w) * 16 + r];
     const int rexp = __float_as_int(tab[5 * TR + tid]);
     const double zhat = double(tab[2 * TR + tid]) + ldexp(s, E + (rexp == kBadRow ? 0 : rexp));
     const double lo = double(tab[tid]), hi = double(tab[TR + tid]);
@@ -587,12 +593,12 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       score[tid] = tok_nonfinite ? __longlong_as_double(0x7ff8000000000000ll) : zhat;
     }
   }
-  __syncthreads();
+  chain_sync();
   // exact re-evaluation from the original codes (rare): one warp per listed neuron
   {
     const int nrc = min(int(misc[MS_NRC]), MAXRC);
     const int nwords = d / 16;
-    for (int e = warp; e < nrc; e += NW) {
+    for (int e = warp; e < nrc; e += NWP) {
       const int n = rc[e];
       const int j = (plan.x + (n >> 4)) * 16 + (n & 15);
       double a64 = 0.0;
@@ -615,7 +621,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     }
     if (nrc > 0) {
       if (tid == 0) atomicAdd(&p.counters[CTR_RECHECKS], (unsigned long long)nrc);
-      __syncthreads();
+      chain_sync();
     }
   }
   // ---- ascending flagged list: ballot + prefix over the (at most 8) warps that hold rows ----
@@ -623,10 +629,10 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     const int f = (tid < nrow) ? (flagbits[tid] & 1) : 0;
     const uint32_t bal = __ballot_sync(0xffffffffu, f != 0);
     if (lane == 0) misc[MS_WCNT + warp] = __popc(bal);
-    __syncthreads();
+    chain_sync();
     int base = 0, total = 0;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) { const int cnt = misc[MS_WCNT + w]; if (w < warp) base += cnt; total += cnt; }
+    for (int w = 0; w < NWP; ++w) { const int cnt = misc[MS_WCNT + w]; if (w < warp) base += cnt; total += cnt; }
     if (f) fl_j[base + __popc(bal & ((1u << lane) - 1u))] = (plan.x + (tid >> 4)) * 16 + (tid & 15);
     if (tid == 0) {
       misc[MS_NFL] = total;
@@ -637,16 +643,16 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       reinterpret_cast<uint16_t*>(p.dbg_bitmap)[plan.x + (tid >> 4)] = uint16_t((bal >> (lane & 16)) & 0xffffu);
     if (p.dbg_scores && tid < nrow) p.dbg_scores[(plan.x + (tid >> 4)) * 16 + (tid & 15)] = score[tid];
   }
-  __syncthreads();
+  chain_sync();
   const int nfl = misc[MS_NFL];
 
   // ---- result fixing, first half: W1 rows -> z_j -> delta_j, on the tensor cores ----
   // 16 flagged rows form the A operand (row g from the list entry g, row g + 8 from entry g + 8), x the B
   // operand (column 0).  A lane reads 8 consecutive channels of its two rows per step; the same 8
   // channels of x sit in the matching operand slots, so the order of channels inside an MMA does not
-  // matter.  The 16 warps split the channel range; their partial z_j meet in shared memory.
+  // matter.  The chain warps split the channel range; their partial z_j meet in shared memory.
   {
-    const int kw = ((p.dpad / NW) + 31) / 32 * 32;          // channels per warp
+    const int kw = ((p.dpad / NWP) + 31) / 32 * 32;         // channels per warp
     for (int e0 = 0; e0 < nfl; e0 += 16) {
       const int ja = (e0 + g < nfl) ? fl_j[e0 + g] : -1;
       const int jb = (e0 + 8 + g < nfl) ? fl_j[e0 + 8 + g] : -1;
@@ -672,33 +678,42 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         }
       }
       if (t4 == 0) {
-        wpart[g * NW + warp] = z0[0] + z1[0];
-        wpart[(g + 8) * NW + warp] = z0[2] + z1[2];
+        wpart[g * NWP + warp] = z0[0] + z1[0];
+        wpart[(g + 8) * NWP + warp] = z0[2] + z1[2];
       }
-      __syncthreads();
+      chain_sync();
       if (tid < 16 && e0 + tid < nfl) {
         const int row = fl_j[e0 + tid] - plan.x * 16;
         float z = 0.f;
 #pragma unroll
-        for (int ww = 0; ww < NW; ++ww) z += wpart[tid * NW + ww];
+        for (int ww = 0; ww < NWP; ++ww) z += wpart[tid * NWP + ww];
         z += tab[2 * TR + row];
         fl_delta[e0 + tid] = gelu_f32(z, p.act) - tab[3 * TR + row] * z - tab[4 * TR + row];
       }
-      __syncthreads();
+      chain_sync();
     }
   }
 
-  constexpr int FB = FIXLOADS / VPT;   // flagged rows per batch of the second half
-  uint4 w[FB][VPT];
-  float acc[VPT][8];
-#pragma unroll
-  for (int m = 0; m < VPT; ++m)
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc[m][i] = 0.f;
-
   // ---- result fixing, second half: W2T rows scaled by delta_j ----
-  for (int e0 = 0; e0 < nfl; e0 += FB) {
-    {
+  // A chain thread owns VPT vectors of 8 output columns per pass; its sums go to the CTA's accumulator replica.
+  constexpr int FB = FIXLOADS / VPT;   // flagged rows per batch
+  constexpr int NTP = NWP * 32;
+  for (int pass = 0; pass < p.npass && nfl > 0; ++pass) {
+    int col[VPT];
+    bool cval[VPT];
+#pragma unroll
+    for (int m = 0; m < VPT; ++m) {
+      const int vec = (pass * VPT + m) * NTP + tid;
+      cval[m] = vec < p.nvec;
+      col[m] = cval[m] ? vec * 8 : 0;
+    }
+    uint4 w[FB][VPT];
+    float acc[VPT][8];
+#pragma unroll
+    for (int m = 0; m < VPT; ++m)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[m][i] = 0.f;
+    for (int e0 = 0; e0 < nfl; e0 += FB) {
 #pragma unroll
       for (int r = 0; r < FB; ++r) {
         const int j = (e0 + r < nfl) ? fl_j[e0 + r] : -1;
@@ -706,20 +721,13 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         for (int m = 0; m < VPT; ++m)
           w[r][m] = (j >= 0 && cval[m]) ? ldg_stream(p.W2T + size_t(j) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
       }
-    }
 #pragma unroll
-    for (int r = 0; r < FB; ++r) {
-      const float dl = (e0 + r < nfl) ? fl_delta[e0 + r] : 0.f;
+      for (int r = 0; r < FB; ++r) {
+        const float dl = (e0 + r < nfl) ? fl_delta[e0 + r] : 0.f;
 #pragma unroll
-      for (int m = 0; m < VPT; ++m) fma8(acc[m], dl, w[r][m]);
+        for (int m = 0; m < VPT; ++m) fma8(acc[m], dl, w[r][m]);
+      }
     }
-  }
-
-  // ---- the rest of the folded product ----
-  stream_c();
-
-  // ---- combine: add this warp's columns to one replica; the last warp on a column range finishes it ----
-  if (nfl > 0) {
 #pragma unroll
     for (int m = 0; m < VPT; ++m)
       if (cval[m]) {
@@ -727,44 +735,57 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         red_add_v4(rep + col[m] + 4, acc[m][4], acc[m][5], acc[m][6], acc[m][7]);
       }
   }
-  // every warp of every CTA may have added to any column, so the columns are complete when the last CTA
-  // is: the CTAs count themselves, and the last one turns the accumulator into y
+
+  // ---- whatever is left of the folded product ----
+  stream_c(warp, NWP);
+
+  // Any warp of any CTA may have added to any column, so the columns are complete when the last CTA is:
+  // the CTAs count themselves (after their streaming warps have reported), and the last one turns the
+  // accumulator into y.
   __threadfence();
-  __syncthreads();
-  if (tid == 0) misc[MS_LAST] = int(atomicAdd(&p.ctl[CTL_DONE], 1u));
-  __syncthreads();
+  chain_sync();
+  if (tid == 0) {
+    bool all = false;
+    for (uint32_t i = 0; i < SPIN_LIMIT && !all; ++i) {
+      all = misc[MS_SDONE] == NW - NWP;
+      if (!all) __nanosleep(64);
+    }
+    if (!all) atomicExch(&p.counters[CTR_ERROR], 1ull);
+    __threadfence();
+    misc[MS_LAST] = int(atomicAdd(&p.ctl[CTL_DONE], 1u));
+  }
+  chain_sync();
   if (misc[MS_LAST] == int(gridDim.x) - 1) {
     __threadfence();
+    for (int vec = tid; vec < p.nvec; vec += NTP) {
+      const int c0 = vec * 8;
+      float4 a0[NREP + 1], a1[NREP + 1];
+      a0[NREP] = *reinterpret_cast<const float4*>(p.bf + c0);
+      a1[NREP] = *reinterpret_cast<const float4*>(p.bf + c0 + 4);
 #pragma unroll
-    for (int m = 0; m < VPT; ++m)
-      if (cval[m]) {
-        float4 a0[NREP + 1], a1[NREP + 1];
-        a0[NREP] = *reinterpret_cast<const float4*>(p.bf + col[m]);
-        a1[NREP] = *reinterpret_cast<const float4*>(p.bf + col[m] + 4);
-#pragma unroll
-        for (int rp = 0; rp < NREP; ++rp) {
-          const float* q = p.yacc + size_t(rp) * p.dacc + col[m];
-          a0[rp] = __ldcg(reinterpret_cast<const float4*>(q));
-          a1[rp] = __ldcg(reinterpret_cast<const float4*>(q + 4));
-        }
-        float4 s0 = a0[NREP], s1 = a1[NREP];
-#pragma unroll
-        for (int rp = 0; rp < NREP; ++rp) {
-          s0.x += a0[rp].x; s0.y += a0[rp].y; s0.z += a0[rp].z; s0.w += a0[rp].w;
-          s1.x += a1[rp].x; s1.y += a1[rp].y; s1.z += a1[rp].z; s1.w += a1[rp].w;
-          float* q = p.yacc + size_t(rp) * p.dacc + col[m];
-          *reinterpret_cast<float4*>(q) = make_float4(0.f, 0.f, 0.f, 0.f);
-          *reinterpret_cast<float4*>(q + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        __nv_bfloat162 o[4];
-        o[0] = __floats2bfloat162_rn(s0.x, s0.y);
-        o[1] = __floats2bfloat162_rn(s0.z, s0.w);
-        o[2] = __floats2bfloat162_rn(s1.x, s1.y);
-        o[3] = __floats2bfloat162_rn(s1.z, s1.w);
-        *reinterpret_cast<uint4*>(p.y + col[m]) = *reinterpret_cast<const uint4*>(o);
+      for (int rp = 0; rp < NREP; ++rp) {
+        const float* q = p.yacc + size_t(rp) * p.dacc + c0;
+        a0[rp] = __ldcg(reinterpret_cast<const float4*>(q));
+        a1[rp] = __ldcg(reinterpret_cast<const float4*>(q + 4));
       }
+      float4 s0 = a0[NREP], s1 = a1[NREP];
+#pragma unroll
+      for (int rp = 0; rp < NREP; ++rp) {
+        s0.x += a0[rp].x; s0.y += a0[rp].y; s0.z += a0[rp].z; s0.w += a0[rp].w;
+        s1.x += a1[rp].x; s1.y += a1[rp].y; s1.z += a1[rp].z; s1.w += a1[rp].w;
+        float* q = p.yacc + size_t(rp) * p.dacc + c0;
+        *reinterpret_cast<float4*>(q) = make_float4(0.f, 0.f, 0.f, 0.f);
+        *reinterpret_cast<float4*>(q + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      __nv_bfloat162 o[4];
+      o[0] = __floats2bfloat162_rn(s0.x, s0.y);
+      o[1] = __floats2bfloat162_rn(s0.z, s0.w);
+      o[2] = __floats2bfloat162_rn(s1.x, s1.y);
+      o[3] = __floats2bfloat162_rn(s1.z, s1.w);
+      *reinterpret_cast<uint4*>(p.y + c0) = *reinterpret_cast<const uint4*>(o);
+    }
     if (lane == 0) {
-      for (int kc = warp; kc < p.nkc; kc += NW) p.ctl[CTL_TICKET + kc * 32] = 0u;
+      for (int kc = warp; kc < p.nkc; kc += NWP) p.ctl[CTL_TICKET + kc * 32] = 0u;
       if (warp == 0) {   // every CTA has arrived, so every CTA's flagged count is in
         p.ctl[CTL_DONE] = 0u;
         const unsigned int tot = atomicExch(&p.ctl[CTL_NFL], 0u);
@@ -876,10 +897,10 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   if (!(G == 64 || G == 128)) return TARDIS_OK;                     // generic kernels serve other group sizes
   const int NT = h / 16;
   const int nvec = d / 8;
-  const int cw = (nvec + NW - 1) / NW;
-  const int vpt = (cw + 31) / 32;
+  const int vpt = nvec > NWP * 32 ? 2 : 1;
+  const int npass = (nvec + NWP * 32 * vpt - 1) / (NWP * 32 * vpt);
   const int dpad = (d + KC - 1) / KC * KC;
-  if (vpt > 2 || d < 64 || d % 16 || dpad > XVR * NTH * 8 || dpad / KC > 32) return TARDIS_OK;
+  if (d < 64 || d % 16 || dpad > XVR * NTH * 8 || dpad / KC > 32) return TARDIS_OK;
   int max_smem = 0, sm_smem = 0;
   TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, H->device));
   TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, H->device));
@@ -895,7 +916,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   p.nranges = (p.nkc + NW - 1) / NW;
   p.cpr = (p.nkc + p.nranges - 1) / p.nranges;
   p.unit_bytes = p.cpr * p.pbs;
-  p.nvec = nvec; p.cw = cw;
+  p.nvec = nvec; p.npass = npass;
   p.nunits = (d / 16) * p.nkc;
   p.ntk = d / 16;
   S->vpt = vpt;
