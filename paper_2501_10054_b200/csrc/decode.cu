@@ -40,13 +40,13 @@ namespace tardis {
 namespace dec {
 
 constexpr int NW = 16;            // warps per CTA
-constexpr int NWP = 8;            // of them, warps that run the predictor -> flags -> fixing chain; the others only stream the folded matrix
+constexpr int NWP = 8;            // of them, warps that evaluate the predictor; meanwhile the others stream the folded matrix
 constexpr int NTH = NW * 32;      // threads per CTA
 constexpr int KC = 256;           // channels per predictor block
 constexpr int MAXTILES = 16;      // predictor tiles (of 16 neurons) per CTA
 constexpr int MAXRC = 64;         // exact re-checks per CTA before the list overflows (rest handled in place)
-constexpr int FIXLOADS = 8;       // 128-bit loads per thread and batch of flagged rows (rows x slots)
 constexpr int MAXBUF = 8;         // predictor unit buffers in shared memory
+constexpr int MAXSLOTS = 16;      // rows of W1 / W2T per round of the result fixing
 constexpr int kBadRow = 0x40000000;   // row whose group scales do not fit the integer form: always re-evaluated
 constexpr int NREP = 4;           // replicas of the output accumulator
 constexpr int XVR = 2;            // 8-channel vectors of x per thread (padded d <= 8192)
@@ -75,7 +75,8 @@ struct Params {
   int nranges, cpr;        // a tile's chunks are taken in nranges units of cpr chunks (cpr <= NW)
   int nbuf, unit_bytes;    // unit buffers in shared memory and their size
   int tiles_max;
-  int nvec, npass;         // 8-column vectors in a row; passes of the chain warps over them
+  int nvec;                // 8-column vectors in a row
+  int nslots;              // rows of W1 / W2T that fit in the predictor buffers at once (<= MAXSLOTS)
   int nunits;              // folded-matrix units in all
   int ntk;                 // output tiles of the folded matrix (16 outputs each)
 };
@@ -164,12 +165,14 @@ __device__ __forceinline__ float dot8(const uint4& w, const float (&xv)[8]) {
 
 // ---- shared-memory carve-up (host and device agree through this) -----------------------------------
 struct SmemLayout {
-  size_t pbuf, xq, xh, sxi, zpart, wpart, score, tab, fl_j, fl_delta, rc, flagbits, wred, bars, misc, total;
+  size_t pbuf_bytes, pbuf, xq, xh, sxi, zpart, wpart, score, tab, fl_j, fl_delta, rc, flagbits, wred, bars, misc, total;
   __host__ __device__ SmemLayout(int dpad, int ngroups, int tiles_max, int nbuf, int unit_bytes) {
     size_t o = 0;
     auto take = [&](size_t bytes, size_t align) { o = (o + align - 1) / align * align; size_t r = o; o += bytes; return r; };
     const size_t rows = size_t(tiles_max) * 16;
-    pbuf = take(size_t(nbuf) * unit_bytes, 128);
+    pbuf_bytes = size_t(nbuf) * unit_bytes;
+    if (pbuf_bytes < size_t(4) * dpad) pbuf_bytes = size_t(4) * dpad;   // room for two rows of the result fixing
+    pbuf = take(pbuf_bytes, 128);
     xq = take(size_t(4) * (dpad + 64), 128);
     xh = take(size_t(dpad + 16) * 2, 16);     // + 16 zeros: the B operand of lanes that feed the unused columns
     sxi = take(size_t(ngroups + 16) * sizeof(int), 8);
@@ -182,14 +185,13 @@ struct SmemLayout {
     rc = take(MAXRC * sizeof(int), 4);
     flagbits = take(rows * sizeof(int), 4);
     wred = take(size_t(3) * NW * sizeof(float), 4);
-    bars = take(size_t(MAXBUF) * sizeof(uint64_t), 8);
+    bars = take(size_t(MAXBUF + 1) * sizeof(uint64_t), 8);
     misc = take(48 * sizeof(int), 8);
     total = o;
   }
 };
-enum { MS_NFL = 0, MS_NRC = 1, MS_ERR = 2, MS_LAST = 3, MS_SDONE = 4, MS_WCNT = 8, MS_BUFCNT = 32 };
-// Named barrier of the chain warps (the streaming warps have left the CTA by then).
-__device__ __forceinline__ void chain_sync() { asm volatile("bar.sync 2, %0;" ::"n"(NWP * 32) : "memory"); }
+enum { MS_NFL = 0, MS_NRC = 1, MS_ERR = 2, MS_LAST = 3, MS_WCNT = 8, MS_BUFCNT = 32 };
+
 
 // ---- the kernel ---------------------------------------------------------------------------------------
 template <int VPT>
@@ -243,6 +245,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
 
   if (tid == 0) {
     for (int b = 0; b < p.nbuf; ++b) mbar_init(&full[b], 1);
+    mbar_init(&full[MAXBUF], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < 48) misc[tid] = 0;
@@ -437,29 +440,17 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     if (lane == 0) wred[2 * NW + warp] = resid;
   }
   // ---- roles ----
-  // The limbs are complete once all 16 warps have passed here.  The streaming warps only announce their part
-  // (bar.arrive) and go on to the folded product, which needs nothing but x; when the tickets run out they
-  // report to the CTA's counter and leave.  The chain warps wait for everybody's limbs (bar.sync).
+  // The limbs are complete once all 16 warps have passed here.  Warps 8..15 only announce their part
+  // (bar.arrive) and go on to the speculative folded product, which needs nothing but x; warps 0..7 wait for
+  // everybody's limbs (bar.sync) and evaluate the predictor.  Both meet again at the barrier after it.
   if (warp >= NWP) {
     asm volatile("bar.arrive 1, %0;" ::"n"(NTH) : "memory");
     stream_c(warp - NWP, NW - NWP);
-    __threadfence();                               // the additions of this warp are visible before it reports
-    __syncwarp();
-    if (lane == 0) atomicAdd(const_cast<int*>(&misc[MS_SDONE]), 1);
-    return;
+  } else {
+    asm volatile("bar.sync 1, %0;" ::"n"(NTH) : "memory");
   }
-  asm volatile("bar.sync 1, %0;" ::"n"(NTH) : "memory");
-  // tolerance of the fast score: every rounding residual (<= 1/2 unit of 2^E) times |code - zero| <= 3 times the scale
-  double tau;
-  {
-    float rs = 0.f;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) rs += wred[2 * NW + w];
-    tau = double(rs) * 1.001 * 3.0 * double(*p.smax) * ldexp(1.0, E);
-  }
-
-  // ---- predictor: chain warp w takes chunks w, w + 8, ... of every unit; partial scores of a tile go to shared memory ----
-  {
+  // ---- predictor: warp w < 8 takes chunks w, w + 8, ... of every unit; partial scores of a tile go to shared memory ----
+  if (warp < NWP) {
     long long zacc[4] = {0, 0, 0, 0}, zt[2] = {0, 0};
     const int gpc = KC / p.G;                                // groups per chunk: 4 or 2
     int b = 0, tl = 0, r = 0;                                // buffer, tile and chunk range of unit u
@@ -552,7 +543,16 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       if (++r == p.nranges) { r = 0; ++tl; }
     }
   }
-  chain_sync();
+  __syncthreads();
+  // tolerance of the fast score: every rounding residual (<= 1/2 unit of 2^E) times |code - zero| <= 3 times the scale
+  double tau;
+  {
+    float rs = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) rs += wred[2 * NW + w];
+    tau = double(rs) * 1.001 * 3.0 * double(*p.smax) * ldexp(1.0, E);
+  }
+
 
   // ---- scores, flags ----
   const int nrow = plan.y * 16;
@@ -593,12 +593,12 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       score[tid] = tok_nonfinite ? __longlong_as_double(0x7ff8000000000000ll) : zhat;
     }
   }
-  chain_sync();
+  __syncthreads();
   // exact re-evaluation from the original codes (rare): one warp per listed neuron
   {
     const int nrc = min(int(misc[MS_NRC]), MAXRC);
     const int nwords = d / 16;
-    for (int e = warp; e < nrc; e += NWP) {
+    for (int e = warp; e < nrc; e += NW) {
       const int n = rc[e];
       const int j = (plan.x + (n >> 4)) * 16 + (n & 15);
       double a64 = 0.0;
@@ -621,7 +621,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     }
     if (nrc > 0) {
       if (tid == 0) atomicAdd(&p.counters[CTR_RECHECKS], (unsigned long long)nrc);
-      chain_sync();
+      __syncthreads();
     }
   }
   // ---- ascending flagged list: ballot + prefix over the (at most 8) warps that hold rows ----
@@ -629,10 +629,10 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     const int f = (tid < nrow) ? (flagbits[tid] & 1) : 0;
     const uint32_t bal = __ballot_sync(0xffffffffu, f != 0);
     if (lane == 0) misc[MS_WCNT + warp] = __popc(bal);
-    chain_sync();
+    __syncthreads();
     int base = 0, total = 0;
 #pragma unroll
-    for (int w = 0; w < NWP; ++w) { const int cnt = misc[MS_WCNT + w]; if (w < warp) base += cnt; total += cnt; }
+    for (int w = 0; w < NW; ++w) { const int cnt = misc[MS_WCNT + w]; if (w < warp) base += cnt; total += cnt; }
     if (f) fl_j[base + __popc(bal & ((1u << lane) - 1u))] = (plan.x + (tid >> 4)) * 16 + (tid & 15);
     if (tid == 0) {
       misc[MS_NFL] = total;
@@ -643,121 +643,103 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       reinterpret_cast<uint16_t*>(p.dbg_bitmap)[plan.x + (tid >> 4)] = uint16_t((bal >> (lane & 16)) & 0xffffu);
     if (p.dbg_scores && tid < nrow) p.dbg_scores[(plan.x + (tid >> 4)) * 16 + (tid & 15)] = score[tid];
   }
-  chain_sync();
+  __syncthreads();
   const int nfl = misc[MS_NFL];
 
-  // ---- result fixing, first half: W1 rows -> z_j -> delta_j, on the tensor cores ----
-  // 16 flagged rows form the A operand (row g from the list entry g, row g + 8 from entry g + 8), x the B
-  // operand (column 0).  A lane reads 8 consecutive channels of its two rows per step; the same 8
-  // channels of x sit in the matching operand slots, so the order of channels inside an MMA does not
-  // matter.  The chain warps split the channel range; their partial z_j meet in shared memory.
+  // ---- result fixing ----
+  // The predictor buffers are free now and take the rows the fixing needs: first the W1 rows of the flagged
+  // neurons, then their W2T rows, one bulk copy per row, as many as fit per round (all of them in one round
+  // for a typical token).  The copies of a round are issued by different warps and complete on one barrier,
+  // so a round costs one trip to memory.  W1 rows: the warps split the channels, partial dot products meet in
+  // shared memory and give delta_j = GELU(z_j) - a_j z_j - c_j.  W2T rows: a thread owns VPT vectors of 8
+  // output columns and adds delta_j times its slice of the row.
+  float acc[VPT][8];
+#pragma unroll
+  for (int m = 0; m < VPT; ++m)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[m][i] = 0.f;
   {
-    const int kw = ((p.dpad / NWP) + 31) / 32 * 32;         // channels per warp
-    for (int e0 = 0; e0 < nfl; e0 += 16) {
-      const int ja = (e0 + g < nfl) ? fl_j[e0 + g] : -1;
-      const int jb = (e0 + 8 + g < nfl) ? fl_j[e0 + 8 + g] : -1;
-      const __nv_bfloat16* pa = p.W1 + size_t(ja < 0 ? 0 : ja) * d;
-      const __nv_bfloat16* pb = p.W1 + size_t(jb < 0 ? 0 : jb) * d;
-      float z0[4] = {0.f, 0.f, 0.f, 0.f}, z1[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int k0 = warp * kw; k0 < (warp + 1) * kw; k0 += 128) {
-        uint4 wa[4], wb[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int k = k0 + q * 32 + t4 * 8;
-          const bool in = k < d && k < (warp + 1) * kw;
-          wa[q] = (in && ja >= 0) ? ldg_stream(pa + k) : make_uint4(0u, 0u, 0u, 0u);
-          wb[q] = (in && jb >= 0) ? ldg_stream(pb + k) : make_uint4(0u, 0u, 0u, 0u);
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int k = k0 + q * 32 + t4 * 8;
-          uint4 xv = make_uint4(0u, 0u, 0u, 0u);
-          if (g == 0 && k < p.dpad) xv = *reinterpret_cast<const uint4*>(xh + k);
-          mma_bf16(z0, wa[q].x, wb[q].x, wa[q].y, wb[q].y, xv.x, xv.y);
-          mma_bf16(z1, wa[q].z, wb[q].z, wa[q].w, wb[q].w, xv.z, xv.w);
+    uint64_t* fixbar = &full[MAXBUF];
+    const uint32_t rowbytes = uint32_t(d) * 2u;
+    const size_t slot_bytes = size_t(p.dpad) * 2;
+    const int nitems = 2 * nfl;
+    const int kw = p.dpad / NW;                                   // channels per warp (a multiple of 16)
+    uint32_t par = 0u;
+    for (int i0 = 0; i0 < nitems; i0 += p.nslots, par ^= 1u) {
+      const int cnt = min(p.nslots, nitems - i0);
+      if (tid == 0) mbar_expect_tx(fixbar, uint32_t(cnt) * rowbytes);
+      if (lane == 0) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the buffers were read with ordinary loads
+        for (int k = warp; k < cnt; k += NW) {
+          const int i = i0 + k;
+          const __nv_bfloat16* src = i < nfl ? p.W1 + size_t(fl_j[i]) * d : p.W2T + size_t(fl_j[i - nfl]) * d;
+          bulk_g2s(pbuf + size_t(k) * slot_bytes, src, rowbytes, fixbar);
         }
       }
-      if (t4 == 0) {
-        wpart[g * NWP + warp] = z0[0] + z1[0];
-        wpart[(g + 8) * NWP + warp] = z0[2] + z1[2];
+      bool landed = mbar_wait(fixbar, par);
+      if (!landed) {
+        if (lane == 0) { atomicExch(&p.counters[CTR_ERROR], 1ull); misc[MS_ERR] = 1; }
+        landed = mbar_wait(fixbar, par);
       }
-      chain_sync();
-      if (tid < 16 && e0 + tid < nfl) {
-        const int row = fl_j[e0 + tid] - plan.x * 16;
-        float z = 0.f;
+      const int nw1 = max(0, min(cnt, nfl - i0));                 // items of this round that are W1 rows
+      if (nw1 > 0) {
+        for (int k = 0; k < nw1; ++k) {
+          const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(pbuf + size_t(k) * slot_bytes);
+          float part = 0.f;
+          for (int c0 = warp * kw + lane * 8; c0 < (warp + 1) * kw; c0 += 256) {
+            if (c0 < d && landed) {
+              float xv[8];
+              unpack8(xv, *reinterpret_cast<const uint4*>(xh + c0));
+              part += dot8(*reinterpret_cast<const uint4*>(row + c0), xv);
+            }
+          }
 #pragma unroll
-        for (int ww = 0; ww < NWP; ++ww) z += wpart[tid * NWP + ww];
-        z += tab[2 * TR + row];
-        fl_delta[e0 + tid] = gelu_f32(z, p.act) - tab[3 * TR + row] * z - tab[4 * TR + row];
+          for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+          if (lane == 0) wpart[k * NW + warp] = part;
+        }
+        __syncthreads();
+        if (tid < nw1) {
+          const int rowi = fl_j[i0 + tid] - plan.x * 16;
+          float z = 0.f;
+#pragma unroll
+          for (int ww = 0; ww < NW; ++ww) z += wpart[tid * NW + ww];
+          z += tab[2 * TR + rowi];
+          fl_delta[i0 + tid] = gelu_f32(z, p.act) - tab[3 * TR + rowi] * z - tab[4 * TR + rowi];
+        }
+        __syncthreads();
       }
-      chain_sync();
+      for (int k = nw1; k < cnt; ++k) {
+        const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(pbuf + size_t(k) * slot_bytes);
+        const float dl = fl_delta[i0 + k - nfl];
+#pragma unroll
+        for (int m = 0; m < VPT; ++m) {
+          const int vec = m * NTH + tid;
+          if (vec < p.nvec && landed) fma8(acc[m], dl, *reinterpret_cast<const uint4*>(row + vec * 8));
+        }
+      }
+      if (i0 + p.nslots < nitems) __syncthreads();               // the slots are written again
     }
   }
-
-  // ---- result fixing, second half: W2T rows scaled by delta_j ----
-  // A chain thread owns VPT vectors of 8 output columns per pass; its sums go to the CTA's accumulator replica.
-  constexpr int FB = FIXLOADS / VPT;   // flagged rows per batch
-  constexpr int NTP = NWP * 32;
-  for (int pass = 0; pass < p.npass && nfl > 0; ++pass) {
-    int col[VPT];
-    bool cval[VPT];
+  if (nfl > 0) {
 #pragma unroll
     for (int m = 0; m < VPT; ++m) {
-      const int vec = (pass * VPT + m) * NTP + tid;
-      cval[m] = vec < p.nvec;
-      col[m] = cval[m] ? vec * 8 : 0;
-    }
-    uint4 w[FB][VPT];
-    float acc[VPT][8];
-#pragma unroll
-    for (int m = 0; m < VPT; ++m)
-#pragma unroll
-      for (int i = 0; i < 8; ++i) acc[m][i] = 0.f;
-    for (int e0 = 0; e0 < nfl; e0 += FB) {
-#pragma unroll
-      for (int r = 0; r < FB; ++r) {
-        const int j = (e0 + r < nfl) ? fl_j[e0 + r] : -1;
-#pragma unroll
-        for (int m = 0; m < VPT; ++m)
-          w[r][m] = (j >= 0 && cval[m]) ? ldg_stream(p.W2T + size_t(j) * d + col[m]) : make_uint4(0u, 0u, 0u, 0u);
-      }
-#pragma unroll
-      for (int r = 0; r < FB; ++r) {
-        const float dl = (e0 + r < nfl) ? fl_delta[e0 + r] : 0.f;
-#pragma unroll
-        for (int m = 0; m < VPT; ++m) fma8(acc[m], dl, w[r][m]);
+      const int vec = m * NTH + tid;
+      if (vec < p.nvec) {
+        red_add_v4(rep + vec * 8, acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
+        red_add_v4(rep + vec * 8 + 4, acc[m][4], acc[m][5], acc[m][6], acc[m][7]);
       }
     }
-#pragma unroll
-    for (int m = 0; m < VPT; ++m)
-      if (cval[m]) {
-        red_add_v4(rep + col[m], acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
-        red_add_v4(rep + col[m] + 4, acc[m][4], acc[m][5], acc[m][6], acc[m][7]);
-      }
   }
-
-  // ---- whatever is left of the folded product ----
-  stream_c(warp, NWP);
 
   // Any warp of any CTA may have added to any column, so the columns are complete when the last CTA is:
-  // the CTAs count themselves (after their streaming warps have reported), and the last one turns the
-  // accumulator into y.
+  // the CTAs count themselves, and the last one turns the accumulator into y.
   __threadfence();
-  chain_sync();
-  if (tid == 0) {
-    bool all = false;
-    for (uint32_t i = 0; i < SPIN_LIMIT && !all; ++i) {
-      all = misc[MS_SDONE] == NW - NWP;
-      if (!all) __nanosleep(64);
-    }
-    if (!all) atomicExch(&p.counters[CTR_ERROR], 1ull);
-    __threadfence();
-    misc[MS_LAST] = int(atomicAdd(&p.ctl[CTL_DONE], 1u));
-  }
-  chain_sync();
+  __syncthreads();
+  if (tid == 0) misc[MS_LAST] = int(atomicAdd(&p.ctl[CTL_DONE], 1u));
+  __syncthreads();
   if (misc[MS_LAST] == int(gridDim.x) - 1) {
     __threadfence();
-    for (int vec = tid; vec < p.nvec; vec += NTP) {
+    for (int vec = tid; vec < p.nvec; vec += NTH) {
       const int c0 = vec * 8;
       float4 a0[NREP + 1], a1[NREP + 1];
       a0[NREP] = *reinterpret_cast<const float4*>(p.bf + c0);
@@ -785,7 +767,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       *reinterpret_cast<uint4*>(p.y + c0) = *reinterpret_cast<const uint4*>(o);
     }
     if (lane == 0) {
-      for (int kc = warp; kc < p.nkc; kc += NWP) p.ctl[CTL_TICKET + kc * 32] = 0u;
+      for (int kc = warp; kc < p.nkc; kc += NW) p.ctl[CTL_TICKET + kc * 32] = 0u;
       if (warp == 0) {   // every CTA has arrived, so every CTA's flagged count is in
         p.ctl[CTL_DONE] = 0u;
         const unsigned int tot = atomicExch(&p.ctl[CTL_NFL], 0u);
@@ -897,8 +879,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   if (!(G == 64 || G == 128)) return TARDIS_OK;                     // generic kernels serve other group sizes
   const int NT = h / 16;
   const int nvec = d / 8;
-  const int vpt = nvec > NWP * 32 ? 2 : 1;
-  const int npass = (nvec + NWP * 32 * vpt - 1) / (NWP * 32 * vpt);
+  const int vpt = nvec > NTH ? 2 : 1;
   const int dpad = (d + KC - 1) / KC * KC;
   if (d < 64 || d % 16 || dpad > XVR * NTH * 8 || dpad / KC > 32) return TARDIS_OK;
   int max_smem = 0, sm_smem = 0;
@@ -916,7 +897,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   p.nranges = (p.nkc + NW - 1) / NW;
   p.cpr = (p.nkc + p.nranges - 1) / p.nranges;
   p.unit_bytes = p.cpr * p.pbs;
-  p.nvec = nvec; p.npass = npass;
+  p.nvec = nvec;
   p.nunits = (d / 16) * p.nkc;
   p.ntk = d / 16;
   S->vpt = vpt;
@@ -934,6 +915,8 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
       const size_t need = SmemLayout(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes).total;
       if (need <= budget && need <= size_t(max_smem)) {
         S->grid = grid; p.tiles_max = tiles_max; p.nbuf = nbuf; S->smem_bytes = need;
+        const size_t slots = SmemLayout(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes).pbuf_bytes / (size_t(dpad) * 2);
+        p.nslots = slots < size_t(MAXSLOTS) ? int(slots) : MAXSLOTS;
         placed = true;
         break;
       }
