@@ -46,7 +46,8 @@ constexpr int KC = 256;           // channels per predictor block
 constexpr int MAXTILES = 16;      // predictor tiles (of 16 neurons) per CTA
 constexpr int MAXRC = 64;         // exact re-checks per CTA before the list overflows (rest handled in place)
 constexpr int MAXBUF = 8;         // predictor unit buffers in shared memory
-constexpr int MAXSLOTS = 16;      // rows of W1 / W2T per round of the result fixing
+constexpr int MAXSLOTS = 16;      // rows of W1 / W2T held in shared memory at once by the result fixing
+constexpr int MAXGROUPS = 8;      // slot groups (one barrier each) of the result fixing
 constexpr int kBadRow = 0x40000000;   // row whose group scales do not fit the integer form: always re-evaluated
 constexpr int NREP = 4;           // replicas of the output accumulator
 constexpr int XVR = 2;            // 8-channel vectors of x per thread (padded d <= 8192)
@@ -76,7 +77,7 @@ struct Params {
   int nbuf, unit_bytes;    // unit buffers in shared memory and their size
   int tiles_max;
   int nvec;                // 8-column vectors in a row
-  int nslots;              // rows of W1 / W2T that fit in the predictor buffers at once (<= MAXSLOTS)
+  int fix_gs, fix_ng;      // result fixing: row slots per group, groups (fix_gs * fix_ng rows fit in the predictor buffers)
   int nunits;              // folded-matrix units in all
   int ntk;                 // output tiles of the folded matrix (16 outputs each)
 };
@@ -177,7 +178,7 @@ struct SmemLayout {
     xh = take(size_t(dpad + 16) * 2, 16);     // + 16 zeros: the B operand of lanes that feed the unused columns
     sxi = take(size_t(ngroups + 16) * sizeof(int), 8);
     zpart = take(rows * NW * sizeof(double), 8);
-    wpart = take(size_t(16) * NW * sizeof(float), 4);
+    wpart = take(size_t(2) * MAXSLOTS * NW * sizeof(float), 4);
     score = take(rows * sizeof(double), 8);
     tab = take(6 * rows * sizeof(float), 4);
     fl_j = take(rows * sizeof(int), 4);
@@ -185,7 +186,7 @@ struct SmemLayout {
     rc = take(MAXRC * sizeof(int), 4);
     flagbits = take(rows * sizeof(int), 4);
     wred = take(size_t(3) * NW * sizeof(float), 4);
-    bars = take(size_t(MAXBUF + 1) * sizeof(uint64_t), 8);
+    bars = take(size_t(MAXBUF + MAXGROUPS) * sizeof(uint64_t), 8);
     misc = take(48 * sizeof(int), 8);
     total = o;
   }
@@ -245,7 +246,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
 
   if (tid == 0) {
     for (int b = 0; b < p.nbuf; ++b) mbar_init(&full[b], 1);
-    mbar_init(&full[MAXBUF], 1);
+    for (int b = 0; b < MAXGROUPS; ++b) mbar_init(&full[MAXBUF + b], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < 48) misc[tid] = 0;
@@ -253,6 +254,10 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   __syncthreads();
   // predictor blocks first: nothing of them depends on x
   if (lane == 0 && warp < p.nbuf && warp < NU) issue_unit(warp);
+  // and this CTA's share of the folded matrix goes to L2, from where the streaming warps (of any CTA) take it
+  if (lane == 0 && warp >= NWP)
+    for (int u = blockIdx.x * (NW - NWP) + (warp - NWP); u < p.nunits; u += gridDim.x * (NW - NWP))
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.Cp + size_t(u) * 512), "r"(8192) : "memory");
 
   // From here on the kernel touches what earlier work in the stream may still be writing (x, the
   // scratch shared by the calls of one handle): wait until that work has completed and is visible.
@@ -647,12 +652,13 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   const int nfl = misc[MS_NFL];
 
   // ---- result fixing ----
-  // The predictor buffers are free now and take the rows the fixing needs: first the W1 rows of the flagged
-  // neurons, then their W2T rows, one bulk copy per row, as many as fit per round (all of them in one round
-  // for a typical token).  The copies of a round are issued by different warps and complete on one barrier,
-  // so a round costs one trip to memory.  W1 rows: the warps split the channels, partial dot products meet in
-  // shared memory and give delta_j = GELU(z_j) - a_j z_j - c_j.  W2T rows: a thread owns VPT vectors of 8
-  // output columns and adds delta_j times its slice of the row.
+  // The predictor buffers are free now and take the rows the fixing needs, one bulk copy per row: item i < nfl
+  // is the W1 row of the i-th flagged neuron, item nfl + i its W2T row.  The row slots form a ring of groups
+  // with one barrier each; all groups are filled at once (for a typical token that is every row the CTA
+  // needs, so the fixing costs one trip to memory), and a group is filled again as soon as its rows have been
+  // used.  W1 rows: the warps split the channels, partial dot products meet in shared memory and give
+  // delta_j = GELU(z_j) - a_j z_j - c_j.  W2T rows: a thread owns VPT vectors of 8 output columns and adds
+  // delta_j times its slice of the row.
   float acc[VPT][8];
 #pragma unroll
   for (int m = 0; m < VPT; ++m)
@@ -663,53 +669,64 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     const uint32_t rowbytes = uint32_t(d) * 2u;
     const size_t slot_bytes = size_t(p.dpad) * 2;
     const int nitems = 2 * nfl;
+    const int GS = p.fix_gs, NG = p.fix_ng;
     const int kw = p.dpad / NW;                                   // channels per warp (a multiple of 16)
-    uint32_t par = 0u;
-    for (int i0 = 0; i0 < nitems; i0 += p.nslots, par ^= 1u) {
-      const int cnt = min(p.nslots, nitems - i0);
-      if (tid == 0) mbar_expect_tx(fixbar, uint32_t(cnt) * rowbytes);
+    // fills group gr with the items of step st (all threads call it; thread 0 arms the barrier, lane 0 of
+    // warp k issues the copy of the k-th item)
+    auto fill = [&](int gr, int st) {
+      const int i0 = st * GS, cnt = min(GS, nitems - i0);
+      if (cnt <= 0) return;
+      if (tid == 0) mbar_expect_tx(&fixbar[gr], uint32_t(cnt) * rowbytes);
       if (lane == 0) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the buffers were read with ordinary loads
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the slots were read with ordinary loads
         for (int k = warp; k < cnt; k += NW) {
           const int i = i0 + k;
           const __nv_bfloat16* src = i < nfl ? p.W1 + size_t(fl_j[i]) * d : p.W2T + size_t(fl_j[i - nfl]) * d;
-          bulk_g2s(pbuf + size_t(k) * slot_bytes, src, rowbytes, fixbar);
+          bulk_g2s(pbuf + size_t(gr * GS + k) * slot_bytes, src, rowbytes, &fixbar[gr]);
         }
       }
-      bool landed = mbar_wait(fixbar, par);
+    };
+    const int nsteps = (nitems + GS - 1) / GS;
+    for (int gr = 0; gr < NG; ++gr) fill(gr, gr);
+    int gr = 0;
+    uint32_t par = 0u;
+    for (int st = 0; st < nsteps; ++st) {
+      const int i0 = st * GS, cnt = min(GS, nitems - i0);
+      bool landed = mbar_wait(&fixbar[gr], par);
       if (!landed) {
         if (lane == 0) { atomicExch(&p.counters[CTR_ERROR], 1ull); misc[MS_ERR] = 1; }
-        landed = mbar_wait(fixbar, par);
+        landed = mbar_wait(&fixbar[gr], par);
       }
-      const int nw1 = max(0, min(cnt, nfl - i0));                 // items of this round that are W1 rows
-      if (nw1 > 0) {
-        for (int k = 0; k < nw1; ++k) {
-          const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(pbuf + size_t(k) * slot_bytes);
-          float part = 0.f;
-          for (int c0 = warp * kw + lane * 8; c0 < (warp + 1) * kw; c0 += 256) {
-            if (c0 < d && landed) {
-              float xv[8];
-              unpack8(xv, *reinterpret_cast<const uint4*>(xh + c0));
-              part += dot8(*reinterpret_cast<const uint4*>(row + c0), xv);
-            }
+      const int nw1 = max(0, min(cnt, nfl - i0));                 // items of this step that are W1 rows
+      float* wp = wpart + (st & 1) * MAXSLOTS * NW;
+      for (int k = 0; k < nw1; ++k) {
+        const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(pbuf + size_t(gr * GS + k) * slot_bytes);
+        float part = 0.f;
+        for (int c0 = warp * kw + lane * 8; c0 < (warp + 1) * kw; c0 += 256) {
+          if (c0 < d && landed) {
+            float xv[8];
+            unpack8(xv, *reinterpret_cast<const uint4*>(xh + c0));
+            part += dot8(*reinterpret_cast<const uint4*>(row + c0), xv);
           }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-          if (lane == 0) wpart[k * NW + warp] = part;
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+        if (lane == 0) wp[k * NW + warp] = part;
+      }
+      if (nw1 > 0) {
         __syncthreads();
         if (tid < nw1) {
           const int rowi = fl_j[i0 + tid] - plan.x * 16;
           float z = 0.f;
 #pragma unroll
-          for (int ww = 0; ww < NW; ++ww) z += wpart[tid * NW + ww];
+          for (int ww = 0; ww < NW; ++ww) z += wp[tid * NW + ww];
           z += tab[2 * TR + rowi];
           fl_delta[i0 + tid] = gelu_f32(z, p.act) - tab[3 * TR + rowi] * z - tab[4 * TR + rowi];
         }
-        __syncthreads();
+        if (nw1 < cnt) __syncthreads();                           // W2T rows of the same step need these deltas
       }
       for (int k = nw1; k < cnt; ++k) {
-        const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(pbuf + size_t(k) * slot_bytes);
+        const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(pbuf + size_t(gr * GS + k) * slot_bytes);
         const float dl = fl_delta[i0 + k - nfl];
 #pragma unroll
         for (int m = 0; m < VPT; ++m) {
@@ -717,7 +734,11 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
           if (vec < p.nvec && landed) fma8(acc[m], dl, *reinterpret_cast<const uint4*>(row + vec * 8));
         }
       }
-      if (i0 + p.nslots < nitems) __syncthreads();               // the slots are written again
+      if (st + 1 < nsteps) {
+        __syncthreads();                                          // rows used, deltas visible
+        fill(gr, st + NG);
+      }
+      if (++gr == NG) { gr = 0; par ^= 1u; }
     }
   }
   if (nfl > 0) {
@@ -915,8 +936,11 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
       const size_t need = SmemLayout(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes).total;
       if (need <= budget && need <= size_t(max_smem)) {
         S->grid = grid; p.tiles_max = tiles_max; p.nbuf = nbuf; S->smem_bytes = need;
-        const size_t slots = SmemLayout(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes).pbuf_bytes / (size_t(dpad) * 2);
-        p.nslots = slots < size_t(MAXSLOTS) ? int(slots) : MAXSLOTS;
+        size_t slots = SmemLayout(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes).pbuf_bytes / (size_t(dpad) * 2);
+        if (slots > size_t(MAXSLOTS)) slots = MAXSLOTS;
+        p.fix_gs = slots >= 6 ? int(slots) / 3 : 1;
+        p.fix_ng = int(slots) / p.fix_gs;
+        if (p.fix_ng > MAXGROUPS) p.fix_ng = MAXGROUPS;
         placed = true;
         break;
       }
