@@ -84,7 +84,7 @@ struct Params {
 
 struct Scratch {           // handle-owned device memory of the fused path
   uint8_t* pblocks; int2* plan; float* smax; float* yacc; unsigned int* ctl; int* rowexp; uint4* Cp;
-  Params base; size_t smem_bytes; size_t bytes; int grid; int vpt;
+  Params base; size_t smem_bytes; size_t bytes; int grid; int vpt; const void* kernel;
 };
 
 // ---- small wrappers ---------------------------------------------------------------------------------
@@ -166,7 +166,7 @@ __device__ __forceinline__ float dot8(const uint4& w, const float (&xv)[8]) {
 
 // ---- shared-memory carve-up (host and device agree through this) -----------------------------------
 struct SmemLayout {
-  size_t pbuf_bytes, pbuf, xq, xh, sxi, zpart, wpart, score, tab, fl_j, fl_delta, rc, flagbits, wred, bars, misc, total;
+  size_t pbuf_bytes, pbuf, xq, zeros, xh, sxi, zpart, wpart, score, tab, fl_j, fl_delta, rc, flagbits, wred, bars, misc, total;
   __host__ __device__ SmemLayout(int dpad, int ngroups, int tiles_max, int nbuf, int unit_bytes) {
     size_t o = 0;
     auto take = [&](size_t bytes, size_t align) { o = (o + align - 1) / align * align; size_t r = o; o += bytes; return r; };
@@ -175,6 +175,7 @@ struct SmemLayout {
     if (pbuf_bytes < size_t(4) * dpad) pbuf_bytes = size_t(4) * dpad;   // room for two rows of the result fixing
     pbuf = take(pbuf_bytes, 128);
     xq = take(size_t(4) * (dpad + 64), 128);
+    zeros = take(256, 16);                    // what the lanes that feed unused operand columns read
     xh = take(size_t(dpad + 16) * 2, 16);     // + 16 zeros: the B operand of lanes that feed the unused columns
     sxi = take(size_t(ngroups + 16) * sizeof(int), 8);
     zpart = take(rows * NW * sizeof(double), 8);
@@ -195,7 +196,7 @@ enum { MS_NFL = 0, MS_NRC = 1, MS_ERR = 2, MS_LAST = 3, MS_WCNT = 8, MS_BUFCNT =
 
 
 // ---- the kernel ---------------------------------------------------------------------------------------
-template <int VPT>
+template <int VPT, int G>
 __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const SmemLayout L(p.dpad, p.ngroups, p.tiles_max, p.nbuf, p.unit_bytes);
@@ -251,6 +252,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   }
   if (tid < 48) misc[tid] = 0;
   if (tid < 8) reinterpret_cast<uint32_t*>(xh + p.dpad)[tid] = 0u;
+  if (tid >= 32 && tid < 96) reinterpret_cast<uint32_t*>(smem + L.zeros)[tid - 32] = 0u;
   __syncthreads();
   // predictor blocks first: nothing of them depends on x
   if (lane == 0 && warp < p.nbuf && warp < NU) issue_unit(warp);
@@ -457,7 +459,11 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   // ---- predictor: warp w < 8 takes chunks w, w + 8, ... of every unit; partial scores of a tile go to shared memory ----
   if (warp < NWP) {
     long long zacc[4] = {0, 0, 0, 0}, zt[2] = {0, 0};
-    const int gpc = KC / p.G;                                // groups per chunk: 4 or 2
+    constexpr int GPC = KC / G;                              // groups per chunk: 4 or 2
+    // Everything a block needs sits at fixed offsets from four per-lane pointers (codes, group words, group sums
+    // of x, limbs of x); lanes whose operand columns are unused (g >= 4) read a block of zeros instead.
+    const uint8_t* const xql = g < 4 ? xq + size_t(g) * xq_stride + t4 * 16 : smem + L.zeros + t4 * 16;
+    const int xqs = g < 4 ? KC : 0;                          // bytes of limbs per chunk
     int b = 0, tl = 0, r = 0;                                // buffer, tile and chunk range of unit u
     uint32_t par = 0u;                                       // phase of the buffer's barrier
     for (int u = 0; u < NU; ++u) {
@@ -468,37 +474,34 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       }
       const int nch = min(p.cpr, p.nkc - r * p.cpr);
       const bool usable = landed && !misc[MS_ERR];
+      const uint8_t* const ubase = pbuf + size_t(b) * p.unit_bytes;
       for (int cc = warp; cc < nch && usable; cc += NWP) {
         const int kc = r * p.cpr + cc;
-        const uint8_t* blk = pbuf + size_t(b) * p.unit_bytes + size_t(cc) * p.pbs;
-        const uint4* cp = reinterpret_cast<const uint4*>(blk);
-        const uint2* mp = reinterpret_cast<const uint2*>(blk + 1024);
-        // group g2 of the chunk done: sums (|.| < 2^22) times the integer scales (|.| < 2^15), all exact
+        const uint8_t* const blk = ubase + cc * p.pbs;
+        const uint4* const cp = reinterpret_cast<const uint4*>(blk) + lane;
+        const uint2* const mp = reinterpret_cast<const uint2*>(blk + 1024) + g;
+        const int* const sxp = sxi + kc * GPC;
+        const uint4* const xp = reinterpret_cast<const uint4*>(xql + kc * xqs);
+        // group gl of the chunk done: sums (|.| < 2^22) times the integer scales (|.| < 2^15), all exact
         auto scale_group = [&](const int (&ia)[4], int gl) {
-          const uint2 mw = mp[gl * 8 + g];
+          const uint2 mw = mp[gl * 8];
           const int m0 = int(mw.x) >> 16, m1 = int(mw.y) >> 16;
           zacc[0] += (long long)m0 * ia[0]; zacc[1] += (long long)m0 * ia[1];
           zacc[2] += (long long)m1 * ia[2]; zacc[3] += (long long)m1 * ia[3];
-          const int sx = sxi[min(kc * gpc + gl, p.ngroups - 1)];
+          const int sx = sxp[gl];
           zt[0] += (long long)(m0 * int(mw.x & 3u)) * sx;
           zt[1] += (long long)(m1 * int(mw.y & 3u)) * sx;
         };
-
 #pragma unroll
         for (int pair = 0; pair < 2; ++pair) {            // 128 channels: four independent MMAs
-          const uint4 cw = cp[pair * 32 + lane];
-          const int kb = kc * 4 + pair * 2;
-          uint4 xb0 = make_uint4(0u, 0u, 0u, 0u), xb1 = xb0;
-          if (g < 4) {
-            xb0 = *reinterpret_cast<const uint4*>(xq + size_t(g) * xq_stride + size_t(kb) * 64 + t4 * 16);
-            xb1 = *reinterpret_cast<const uint4*>(xq + size_t(g) * xq_stride + size_t(kb + 1) * 64 + t4 * 16);
-          }
+          const uint4 cw = cp[pair * 32];
+          const uint4 xb0 = xp[pair * 8], xb1 = xp[pair * 8 + 4];
           int q0[4], q1[4], q2[4], q3[4];
           mma_u8s8_z(q0, cw.x & 0x03030303u, cw.y & 0x03030303u, cw.x & 0x0C0C0C0Cu, cw.y & 0x0C0C0C0Cu, xb0.x, xb0.y);
           mma_u8s8_z(q1, cw.x & 0x30303030u, cw.y & 0x30303030u, cw.x & 0xC0C0C0C0u, cw.y & 0xC0C0C0C0u, xb0.z, xb0.w);
           mma_u8s8_z(q2, cw.z & 0x03030303u, cw.w & 0x03030303u, cw.z & 0x0C0C0C0Cu, cw.w & 0x0C0C0C0Cu, xb1.x, xb1.y);
           mma_u8s8_z(q3, cw.z & 0x30303030u, cw.w & 0x30303030u, cw.z & 0xC0C0C0C0u, cw.w & 0xC0C0C0C0u, xb1.z, xb1.w);
-          if (p.G == 64) {
+          if (G == 64) {
             int ga[4], gb[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) { ga[i] = q0[i] + q1[i]; gb[i] = q2[i] + q3[i]; }
@@ -511,7 +514,6 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
             scale_group(ga, pair);
           }
         }
-
       }
       if (r == p.nranges - 1) {
         // limbs: lane t4 = 0 holds limbs 0,1 ; t4 = 1 holds limbs 2,3 (columns 4..7 are unused for one token)
@@ -984,8 +986,9 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   k_pack_folded<<<p.nunits, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->C), S->Cp, d, p.nkc);
   k_max_scale<<<64, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->scale), size_t(h) * H->ngroups, S->smax);
   e = cudaGetLastError();
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+  S->kernel = vpt == 1 ? (G == 64 ? (const void*)k_decode<1, 64> : (const void*)k_decode<1, 128>)
+                       : (G == 64 ? (const void*)k_decode<2, 64> : (const void*)k_decode<2, 128>);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(S->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
   if (e != cudaSuccess) { set_last_error(e, "decode_prepare launch"); return fail(TARDIS_ERR_CUDA); }
 
   p.pblocks = S->pblocks; p.plan = S->plan; p.smax = S->smax; p.rowexp = S->rowexp; p.yacc = S->yacc; p.ctl = S->ctl;
@@ -1016,8 +1019,8 @@ tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (S->vpt == 1) TARDIS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode<1>, p));
-    else TARDIS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode<2>, p));
+    void* args[] = {&p};
+    TARDIS_CUDA_TRY(cudaLaunchKernelExC(&cfg, S->kernel, args));
     H->launches += 1;
   }
   return TARDIS_OK;
