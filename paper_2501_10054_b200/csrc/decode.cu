@@ -123,7 +123,7 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {   // read-only, no 
 }
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -131,7 +131,7 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
 // four times better than a chain through one accumulator, so each MMA of a group starts its own sum.
 __device__ __forceinline__ void mma_u8s8_z(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                            uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
                : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
 }
@@ -496,21 +496,19 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
         for (int pair = 0; pair < 2; ++pair) {            // 128 channels: four independent MMAs
           const uint4 cw = cp[pair * 32];
           const uint4 xb0 = xp[pair * 8], xb1 = xp[pair * 8 + 4];
-          int q0[4], q1[4], q2[4], q3[4];
-          mma_u8s8_z(q0, cw.x & 0x03030303u, cw.y & 0x03030303u, cw.x & 0x0C0C0C0Cu, cw.y & 0x0C0C0C0Cu, xb0.x, xb0.y);
-          mma_u8s8_z(q1, cw.x & 0x30303030u, cw.y & 0x30303030u, cw.x & 0xC0C0C0C0u, cw.y & 0xC0C0C0C0u, xb0.z, xb0.w);
-          mma_u8s8_z(q2, cw.z & 0x03030303u, cw.w & 0x03030303u, cw.z & 0x0C0C0C0Cu, cw.w & 0x0C0C0C0Cu, xb1.x, xb1.y);
-          mma_u8s8_z(q3, cw.z & 0x30303030u, cw.w & 0x30303030u, cw.z & 0xC0C0C0C0u, cw.w & 0xC0C0C0C0u, xb1.z, xb1.w);
+          // two accumulator chains of two MMAs each (a longer chain through one accumulator would stall the pipe)
+          int qa[4], qb[4];
+          mma_u8s8_z(qa, cw.x & 0x03030303u, cw.y & 0x03030303u, cw.x & 0x0C0C0C0Cu, cw.y & 0x0C0C0C0Cu, xb0.x, xb0.y);
+          mma_u8s8_z(qb, cw.z & 0x03030303u, cw.w & 0x03030303u, cw.z & 0x0C0C0C0Cu, cw.w & 0x0C0C0C0Cu, xb1.x, xb1.y);
+          mma_u8s8(qa, cw.x & 0x30303030u, cw.y & 0x30303030u, cw.x & 0xC0C0C0C0u, cw.y & 0xC0C0C0C0u, xb0.z, xb0.w);
+          mma_u8s8(qb, cw.z & 0x30303030u, cw.w & 0x30303030u, cw.z & 0xC0C0C0C0u, cw.w & 0xC0C0C0C0u, xb1.z, xb1.w);
           if (G == 64) {
-            int ga[4], gb[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { ga[i] = q0[i] + q1[i]; gb[i] = q2[i] + q3[i]; }
-            scale_group(ga, pair * 2);
-            scale_group(gb, pair * 2 + 1);
+            scale_group(qa, pair * 2);
+            scale_group(qb, pair * 2 + 1);
           } else {                                        // G == 128
             int ga[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) ga[i] = (q0[i] + q1[i]) + (q2[i] + q3[i]);
+            for (int i = 0; i < 4; ++i) ga[i] = qa[i] + qb[i];
             scale_group(ga, pair);
           }
         }
