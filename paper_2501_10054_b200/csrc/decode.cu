@@ -3,33 +3,34 @@
 // One launch does the whole token: predictor score (Section 5.3), flagging and compaction,
 // speculative folded product, result fixing.  The grid is (up to) two 512-thread CTAs per SM.
 //
-//   * A CTA owns a few 16-neuron tiles.  Their predictor blocks (packed 2-bit codes + group
-//     scales) are one contiguous region per tile, fetched with a few large bulk async copies
-//     (cp.async.bulk + mbarrier) that are issued before anything else and land while x is
-//     prepared.  The codes are evaluated on the integer tensor cores: they are masked straight
-//     out of the packed words (no shifts: the field position is a power-of-4 weight that the
-//     pre-scaling of x undoes) and multiplied with a 4-limb signed base-256 fixed-point copy of x
-//     (mma.m16n8k32.u8.s8, s32 accumulators, exact).  The bf16 group scales of a neuron are held as
-//     16-bit integers over one power of two per neuron, so group sums are scaled and accumulated in
-//     64-bit integers (exact) and the score equals the mathematical one up to the (tracked)
-//     truncation of tiny x elements and one fp64 rounding; a score that close to a range end is
-//     re-evaluated in fp64 from the original codes.  The 16 warps split the channel chunks of a
-//     tile; partial scores meet in shared memory.
-//   * Flags are compacted by ballot + prefix sum into the CTA's ascending list.
-//   * Result fixing, first half: the W1 rows of the CTA's flagged neurons are the A operand of bf16
-//     MMAs (16 flagged rows at a time, 128-bit read-only loads), x the B operand; the 16 warps split
-//     the channels and their partial z_j meet in shared memory, giving
-//     delta_j = GELU(z_j) - a_j z_j - c_j.  Second half: every thread owns 8 output columns (per
-//     slot) and adds delta_j times its slice of the W2T rows into fp32 column accumulators.
-//   * The speculative folded product runs on the bf16 tensor cores too: the fold leaves W_f in
-//     A-fragment order (units of 16 outputs x 256 channels, 8 KB, contiguous).  Warp w works on
-//     channel chunk w and draws output tiles from a global ticket of that chunk, so CTAs with few
-//     flagged neurons take more of the folded product and all finish together.
+//   * Prologue (before griddepcontrol.wait, so it overlaps the tail of the previous launch in the
+//     stream): a CTA owns a few 16-neuron tiles; their predictor blocks (packed 2-bit codes + group
+//     words) are one contiguous region per tile and are fetched with a few large bulk async copies
+//     (cp.async.bulk + mbarrier) into shared memory; the CTA's share of the folded matrix is
+//     prefetched into L2 (cp.async.bulk.prefetch.L2).  Both read constant state of the layer only.
+//   * x is loaded once: a bf16 copy in shared memory, and a 4-limb signed base-256 fixed-point copy in
+//     tensor-core operand order.
+//   * Then the warps split.  Warps 0..7 evaluate the predictor on the integer tensor cores: the codes are
+//     masked straight out of the packed words (no shifts: the field position is a power-of-4 weight that
+//     the pre-scaling of x undoes) and multiplied with the limbs (mma.m16n8k32.u8.s8, s32 accumulators,
+//     exact).  The bf16 group scales of a neuron are held as 16-bit integers over one power of two per
+//     neuron, so group sums are scaled and accumulated in 64-bit integers (exact) and the score equals the
+//     mathematical one up to the (tracked) truncation of tiny x elements and one fp64 rounding; a score
+//     that close to a range end is re-evaluated in fp64 from the original codes.  This phase is bound by
+//     the integer pipe, which is why only half of the warps are given to it.
+//   * Meanwhile warps 8..15 run the speculative folded product on the bf16 tensor cores: the fold leaves
+//     W_f in A-fragment order (units of 16 outputs x 256 channels, 8 KB, contiguous).  A warp works on
+//     one channel chunk at a time and draws output tiles from a global ticket of that chunk, so the
+//     units spread over all CTAs however busy each one is.
+//   * All 16 warps meet; flags are compacted by ballot + prefix sum into the CTA's ascending list.
+//   * Result fixing: the predictor buffers are free by now and become row slots.  The W1 rows of the
+//     CTA's flagged neurons, then their W2T rows, are fetched by one bulk copy per row, all slots at once
+//     (a ring of slot groups when there are more rows than slots).  W1 rows give z_j (the warps split
+//     the channels) and delta_j = GELU(z_j) - a_j z_j - c_j; then every thread owns 8 output columns
+//     (per slot of 512 vectors) and adds delta_j times its slice of the W2T rows.
 //   * All partial outputs are added (red.global) into one of a few replicas of an fp32 accumulator
 //     (the replicas keep the number of reductions per address small).  CTAs count themselves when
 //     done; the last one sums the replicas, adds b_f, rounds to bf16, and re-zeroes the scratch.
-//   * The launch uses programmatic dependent launch: everything up to griddepcontrol.wait (tables,
-//     predictor copies) reads constant state only and overlaps the tail of the previous launch.
 #include <stdio.h>
 
 #include <vector>
@@ -40,7 +41,7 @@ namespace tardis {
 namespace dec {
 
 constexpr int NW = 16;            // warps per CTA
-constexpr int NWP = 8;            // of them, warps that evaluate the predictor; meanwhile the others stream the folded matrix
+constexpr int NWP = 8;            // of them, warps that evaluate the predictor while the others stream the folded matrix
 constexpr int NTH = NW * 32;      // threads per CTA
 constexpr int KC = 256;           // channels per predictor block
 constexpr int MAXTILES = 16;      // predictor tiles (of 16 neurons) per CTA
