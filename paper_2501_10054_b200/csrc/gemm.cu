@@ -1,12 +1,13 @@
 // bf16 GEMM on the 5th-generation tensor cores (see gemm.cuh for what it computes).
 //
-// One CTA computes a 128 x BN tile of the output.  Warp 0 stages 128 x 64 (A) and BN x 64 (B) operand
-// boxes into a ring of shared-memory stages with TMA (cp.async.bulk.tensor, 128-byte swizzle, no
-// multicast); warp 1 issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) from one thread,
-// accumulating in tensor memory (TMEM, 128 lanes x BN fp32 columns) and releasing each stage with
-// tcgen05.commit; warps 2..5 read the accumulator back with tcgen05.ld (each warp its own 32 lanes)
-// and run the epilogue.  Every wait on an mbarrier is bounded: when it runs out the waiter sets an
-// error word and the CTA falls through to the end, where TMEM is released.
+// A CTA computes 128 x BN tiles of the output, one after the other (persistent, one CTA per SM).  Warp 0 stages
+// 128 x 64 (A) and BN x 64 (B) operand boxes into a ring of shared-memory stages with TMA
+// (cp.async.bulk.tensor, 128-byte swizzle, no multicast); warp 1 issues tcgen05.mma (M = 128, N = BN,
+// K = 16 per instruction) from one thread, accumulating in tensor memory (TMEM, 128 lanes x BN fp32 columns,
+// two accumulators used in turn) and releasing each stage with tcgen05.commit; warps 2..5 read a finished
+// accumulator back with tcgen05.ld (each warp its own 32 lanes) and run the epilogue while the next tile's
+// main loop fills the other accumulator.  Every wait on an mbarrier is bounded: when it runs out the waiter
+// sets an error word and the CTA falls through to the end, where TMEM is released.
 #include "gemm.cuh"
 
 #include <cuda.h>
@@ -29,6 +30,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
 }
 __device__ __forceinline__ bool mbar_test(uint64_t* b, uint32_t parity) {
   uint32_t ok;
@@ -111,8 +115,81 @@ template <int BN> struct Cfg {
   static constexpr int STAGE_BYTES = BM * BK * 2 + BN * BK * 2;
   static constexpr int NS = (BN == 256) ? 4 : 6;                      // stages
   static constexpr int SMEM = NS * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+  static constexpr int TMEM_COLS = 2 * BN;                            // two accumulators
 };
 
+// The epilogue of 32 consecutive columns n .. n + nv - 1 of output row m (one thread).
+__device__ __forceinline__ void epilogue_chunk(const KParams& p, float (&v)[32], int m, int n, int nv, bool first_split, bool have_acc) {
+  if (p.epilogue == GEMM_EPI_F32 && p.splits > 1) {
+    float* o = p.out_f32 + size_t(m) * p.ldo + n;
+    const bool with_bias = p.bias && first_split;
+    if (have_acc || with_bias) {
+      if (nv == 32 && (p.ldo & 3) == 0) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          float4 t = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+          if (with_bias) { t.x += p.bias[n + i]; t.y += p.bias[n + i + 1]; t.z += p.bias[n + i + 2]; t.w += p.bias[n + i + 3]; }
+          asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + i), "f"(t.x), "f"(t.y), "f"(t.z), "f"(t.w) : "memory");
+        }
+      } else {
+        for (int i = 0; i < nv; ++i) atomicAdd(o + i, v[i] + (with_bias ? p.bias[n + i] : 0.f));
+      }
+    }
+  } else if (p.epilogue == GEMM_EPI_F32) {
+    float* o = p.out_f32 + size_t(m) * p.ldo + n;
+    if (nv == 32 && (p.ldo & 3) == 0) {
+#pragma unroll
+      for (int i = 0; i < 32; i += 4) {
+        float4 t = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        if (p.bias) { t.x += p.bias[n + i]; t.y += p.bias[n + i + 1]; t.z += p.bias[n + i + 2]; t.w += p.bias[n + i + 3]; }
+        *reinterpret_cast<float4*>(o + i) = t;
+      }
+    } else {
+      for (int i = 0; i < nv; ++i) o[i] = v[i] + (p.bias ? p.bias[n + i] : 0.f);
+    }
+  } else {
+    // bf16 outputs: this thread's 32 values become four 16-byte stores
+    if (p.epilogue == GEMM_EPI_ADD_BF16) {
+      const float* ad = p.addend + size_t(m) * p.ldo + n;
+      if (nv == 32 && (p.ldo & 3) == 0) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          const float4 t = *reinterpret_cast<const float4*>(ad + i);
+          v[i] += t.x; v[i + 1] += t.y; v[i + 2] += t.z; v[i + 3] += t.w;
+        }
+      } else {
+        for (int i = 0; i < nv; ++i) v[i] += ad[i];
+      }
+    } else {   // GEMM_EPI_DELTA: one flag word covers this thread's 32 columns
+      const uint32_t word = p.bitmap[size_t(m) * (p.N / 32) + (n >> 5)];
+#pragma unroll 8
+      for (int i = 0; i < 32; ++i) {
+        float dl = 0.f;
+        if (((word >> i) & 1u) && i < nv) {
+          const float z = v[i] + (p.bias ? p.bias[n + i] : 0.f);
+          dl = gelu_f32(z, p.act) - p.a[n + i] * z - p.c[n + i];
+        }
+        v[i] = dl;
+      }
+    }
+    __nv_bfloat16* o = p.out_bf16 + size_t(m) * p.ldo + n;
+    if (nv == 32 && (p.ldo & 7) == 0) {
+#pragma unroll
+      for (int i = 0; i < 32; i += 8) {
+        __nv_bfloat162 h[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) h[q] = __floats2bfloat162_rn(v[i + 2 * q], v[i + 2 * q + 1]);
+        *reinterpret_cast<uint4*>(o + i) = *reinterpret_cast<const uint4*>(h);
+      }
+    } else {
+      for (int i = 0; i < nv; ++i) o[i] = __float2bfloat16_rn(v[i]);
+    }
+  }
+}
+
+// Persistent: CTA c works on tiles c, c + gridDim.x, ... (row tiles fastest, so that the CTAs running at the same
+// time share few column blocks of B).  Two accumulators in tensor memory: while the epilogue warps drain one, the
+// MMA warp is already filling the other with the next tile.
 template <int BN>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
@@ -122,163 +199,134 @@ k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtenso
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::NS * C::STAGE_BYTES);
   uint64_t* empty = full + C::NS;
-  uint64_t* accum_full = empty + C::NS;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_full + 1);
+  uint64_t* accum_full = empty + C::NS;        // [2]
+  uint64_t* accum_empty = accum_full + 2;      // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_empty + 2);
   volatile uint32_t* failed = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  // this CTA's share of the k blocks (all of them unless the launch splits the channel range)
+  const int nm = (p.M + BM - 1) / BM, nn = (p.N + BN - 1) / BN;
+  const int ntiles = nm * nn * p.splits;
   const int nkb_all = p.kb1 + p.kb2;
-  const int per = (nkb_all + p.splits - 1) / p.splits;
-  const int kb_lo = blockIdx.z * per;
-  const int nkb = max(0, min(nkb_all, kb_lo + per) - kb_lo);
+  const int per = (nkb_all + p.splits - 1) / p.splits;   // k blocks per split of the channel range
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(accum_full, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&accum_full[b], 1); mbar_init(&accum_empty[b], 4); }
     *failed = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA1) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB1) : "memory");
   }
-  if (warp == 1) tmem_alloc(tmem_slot, BN);          // the whole warp; BN fp32 columns (a power of two >= 32)
+  if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);  // the whole warp; a power of two >= 32 fp32 columns
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // tile -> first row, first column, k-block range
+  auto decode = [&](int tile, int& m0, int& n0, int& kb_lo, int& nkb, int& z) {
+    z = tile / (nm * nn);
+    const int rem = tile - z * (nm * nn);
+    const int ni = rem / nm, mi = rem - ni * nm;
+    m0 = mi * BM; n0 = ni * BN;
+    kb_lo = z * per;
+    nkb = max(0, min(nkb_all, kb_lo + per) - kb_lo);
+  };
+
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % C::NS;
-        if (!mbar_wait(&empty[s], ((kb / C::NS) & 1) ^ 1)) { *failed = 1u; break; }
-        uint8_t* sa = smem + s * C::STAGE_BYTES;
-        uint8_t* sb = sa + BM * BK * 2;
-        mbar_expect_tx(&full[s], C::STAGE_BYTES);
-        const int kg = kb_lo + kb;                   // k block in the whole channel range
-        const bool second = kg >= p.kb1;
-        const int kx = (second ? kg - p.kb1 : kg) * BK;
-        tma_load_2d(sa, second ? &tmA2 : &tmA1, kx, m0, &full[s]);
-        tma_load_2d(sb, second ? &tmB2 : &tmB1, kx, n0, &full[s]);
+      uint32_t it = 0;                                 // k blocks staged so far (over all tiles)
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+        int m0, n0, kb_lo, nkb, z;
+        decode(tile, m0, n0, kb_lo, nkb, z);
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % C::NS;
+          if (*failed || !mbar_wait(&empty[s], ((it / C::NS) & 1) ^ 1)) { *failed = 1u; ok = false; break; }
+          uint8_t* sa = smem + s * C::STAGE_BYTES;
+          uint8_t* sb = sa + BM * BK * 2;
+          mbar_expect_tx(&full[s], C::STAGE_BYTES);
+          const int kg = kb_lo + kb;                   // k block in the whole channel range
+          const bool second = kg >= p.kb1;
+          const int kx = (second ? kg - p.kb1 : kg) * BK;
+          tma_load_2d(sa, second ? &tmA2 : &tmA1, kx, m0, &full[s]);
+          tma_load_2d(sb, second ? &tmB2 : &tmB1, kx, n0, &full[s]);
+        }
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_bf16(BM, BN);
+      uint32_t it = 0, use = 0;                        // k blocks consumed; accumulator uses so far
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % C::NS;
-        if (!mbar_wait(&full[s], (kb / C::NS) & 1)) { *failed = 1u; ok = false; break; }
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+        int m0, n0, kb_lo, nkb, z;
+        decode(tile, m0, n0, kb_lo, nkb, z);
+        if (nkb == 0) continue;                        // nothing to add: the epilogue takes zeros
+        const uint32_t ab = use & 1u;
+        // the epilogue warps have drained this accumulator's previous tile
+        if (*failed || !mbar_wait(&accum_empty[ab], ((use >> 1) & 1) ^ 1)) { *failed = 1u; ok = false; break; }
         tc_fence_after();
-        const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES);
-        const uint32_t sb = sa + BM * BK * 2;
+        const uint32_t tacc = tmem_base + ab * BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % C::NS;
+          if (!mbar_wait(&full[s], (it / C::NS) & 1)) { *failed = 1u; ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES);
+          const uint32_t sb = sa + BM * BK * 2;
 #pragma unroll
-        for (int k = 0; k < BK / 16; ++k) {
-          const uint64_t adesc = smem_desc_k_major_sw128(sa + k * 32);
-          const uint64_t bdesc = smem_desc_k_major_sw128(sb + k * 32);
-          umma_f16(tmem_base, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t adesc = smem_desc_k_major_sw128(sa + k * 32);
+            const uint64_t bdesc = smem_desc_k_major_sw128(sb + k * 32);
+            umma_f16(tacc, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(&empty[s]);                      // frees the stage when these MMAs have read it
         }
-        umma_commit(&empty[s]);                      // frees the stage when these MMAs have read it
+        if (ok) umma_commit(&accum_full[ab]);          // accumulator complete
+        ++use;
       }
-      if (ok) umma_commit(accum_full);               // accumulator complete
     }
   } else {
     // ---------------- epilogue: warp q reads TMEM lanes 32 (warp % 4) .. + 31 ----------------
     const int q = warp & 3;
-    const int m = m0 + q * 32 + lane;
+    uint32_t use = 0;
     bool ok = true;
-    if (nkb > 0) {
-      ok = mbar_wait(accum_full, 0);
-      if (!ok) *failed = 1u;
-    }
-    tc_fence_after();
-    if (ok) {
+    for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+      int m0, n0, kb_lo, nkb, z;
+      decode(tile, m0, n0, kb_lo, nkb, z);
+      const int m = m0 + q * 32 + lane;
+      const uint32_t ab = use & 1u;
+      if (nkb > 0) {
+        ok = !*failed && mbar_wait(&accum_full[ab], (use >> 1) & 1);
+        if (!ok) { *failed = 1u; break; }
+        tc_fence_after();
+      }
       for (int ch = 0; ch < BN / 32; ++ch) {
         float v[32];
-        if (nkb > 0) tmem_ld32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(ch * 32), v);
+        if (nkb > 0) tmem_ld32(tmem_base + ab * BN + (uint32_t(q * 32) << 16) + uint32_t(ch * 32), v);
         else {
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = 0.f;
         }
         const int n = n0 + ch * 32;
         const int nv = min(32, p.N - n);
-        if (m < p.M && nv > 0) {                      // (no early exit: the next tcgen05.ld needs the whole warp)
-          if (p.epilogue == GEMM_EPI_F32 && p.splits > 1) {
-            float* o = p.out_f32 + size_t(m) * p.ldo + n;
-            const bool with_bias = p.bias && blockIdx.z == 0;
-            if (nkb > 0 || with_bias) {
-              if (nv == 32 && (p.ldo & 3) == 0) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                  float4 t = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                  if (with_bias) { t.x += p.bias[n + i]; t.y += p.bias[n + i + 1]; t.z += p.bias[n + i + 2]; t.w += p.bias[n + i + 3]; }
-                  asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + i), "f"(t.x), "f"(t.y), "f"(t.z), "f"(t.w) : "memory");
-                }
-              } else {
-                for (int i = 0; i < nv; ++i) atomicAdd(o + i, v[i] + (with_bias ? p.bias[n + i] : 0.f));
-              }
-            }
-          } else if (p.epilogue == GEMM_EPI_F32) {
-            float* o = p.out_f32 + size_t(m) * p.ldo + n;
-            if (nv == 32 && (p.ldo & 3) == 0) {
-#pragma unroll
-              for (int i = 0; i < 32; i += 4) {
-                float4 t = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                if (p.bias) { t.x += p.bias[n + i]; t.y += p.bias[n + i + 1]; t.z += p.bias[n + i + 2]; t.w += p.bias[n + i + 3]; }
-                *reinterpret_cast<float4*>(o + i) = t;
-              }
-            } else {
-              for (int i = 0; i < nv; ++i) o[i] = v[i] + (p.bias ? p.bias[n + i] : 0.f);
-            }
-          } else {
-            // bf16 outputs: this thread's 32 values become four 16-byte stores
-            if (p.epilogue == GEMM_EPI_ADD_BF16) {
-              const float* ad = p.addend + size_t(m) * p.ldo + n;
-              if (nv == 32 && (p.ldo & 3) == 0) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                  const float4 t = *reinterpret_cast<const float4*>(ad + i);
-                  v[i] += t.x; v[i + 1] += t.y; v[i + 2] += t.z; v[i + 3] += t.w;
-                }
-              } else {
-                for (int i = 0; i < nv; ++i) v[i] += ad[i];
-              }
-            } else {   // GEMM_EPI_DELTA: one flag word covers this thread's 32 columns
-              const uint32_t word = p.bitmap[size_t(m) * (p.N / 32) + (n >> 5)];
-#pragma unroll 8
-              for (int i = 0; i < 32; ++i) {
-                float dl = 0.f;
-                if (((word >> i) & 1u) && i < nv) {
-                  const float z = v[i] + (p.bias ? p.bias[n + i] : 0.f);
-                  dl = gelu_f32(z, p.act) - p.a[n + i] * z - p.c[n + i];
-                }
-                v[i] = dl;
-              }
-            }
-            __nv_bfloat16* o = p.out_bf16 + size_t(m) * p.ldo + n;
-            if (nv == 32 && (p.ldo & 7) == 0) {
-#pragma unroll
-              for (int i = 0; i < 32; i += 8) {
-                __nv_bfloat162 h[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) h[q] = __floats2bfloat162_rn(v[i + 2 * q], v[i + 2 * q + 1]);
-                *reinterpret_cast<uint4*>(o + i) = *reinterpret_cast<const uint4*>(h);
-              }
-            } else {
-              for (int i = 0; i < nv; ++i) o[i] = __float2bfloat16_rn(v[i]);
-            }
-          }
-        }
+        if (m < p.M && nv > 0) epilogue_chunk(p, v, m, n, nv, z == 0, nkb > 0);   // (no early exit: tcgen05.ld needs the whole warp)
+      }
+      if (nkb > 0) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&accum_empty[ab]);  // this warp's lanes of the accumulator may be overwritten
+        ++use;
       }
     }
   }
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *failed && p.error_word) atomicExch(p.error_word, 1ull);
-  if (warp == 1) tmem_dealloc(tmem_base, BN);
+  if (warp == 1) tmem_dealloc(tmem_base, C::TMEM_COLS);
 }
 
 // ---- host side ------------------------------------------------------------------------------------------
@@ -327,7 +375,11 @@ static tardis_status_t launch_bn(const GemmArgs& g, cudaStream_t s) {
   p.out_f32 = g.out_f32; p.out_bf16 = static_cast<__nv_bfloat16*>(g.out_bf16);
   p.bias = g.bias; p.addend = g.addend; p.a = g.a; p.c = g.c; p.bitmap = g.bitmap; p.error_word = g.error_word;
   TARDIS_CUDA_TRY(cudaFuncSetAttribute(k_gemm<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM));
-  dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, p.splits);
+  const long tiles = long((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * p.splits;
+  int dev = 0, sms = 0;
+  TARDIS_CUDA_TRY(cudaGetDevice(&dev));
+  TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const unsigned grid = unsigned(tiles < sms ? tiles : sms);          // one CTA per SM (shared memory), persistent
   k_gemm<BN><<<grid, NTHREADS, Cfg<BN>::SMEM, s>>>(a1, b1, a2, b2, p);
   TARDIS_CUDA_TRY(cudaGetLastError());
   return TARDIS_OK;
