@@ -14,6 +14,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "exact.cuh"
 #include "gemm.cuh"
 
 namespace tardis {
@@ -84,71 +85,6 @@ __global__ void k_xnorm(const __nv_bfloat16* __restrict__ x, int d, float* __res
   }
 }
 
-__device__ double exact_score(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
-                              const uint8_t* __restrict__ zero, const __nv_bfloat16* __restrict__ xt, int j, int d, int G,
-                              int lane) {   // one warp; every lane returns the sum
-  const int nwords = d / 16, ng = d / G;
-  double acc = 0.0;
-  for (int w = lane; w < nwords; w += 32) {
-    const uint32_t word = codes[size_t(j) * nwords + w];
-    const int g = (w * 16) / G;
-    const double zp = double(zero[size_t(j) * ng + g]);
-    double inner = 0.0;
-#pragma unroll
-    for (int q = 0; q < 16; ++q) inner += (double((word >> (2 * q)) & 3u) - zp) * double(__bfloat162float(xt[w * 16 + q]));
-    acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-  return acc;
-}
-
-__device__ double exact_score_single(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
-                                     const uint8_t* __restrict__ zero, const __nv_bfloat16* __restrict__ xt, int j, int d, int G) {
-  const int nwords = d / 16, ng = d / G;
-  double acc = 0.0;
-  for (int w = 0; w < nwords; ++w) {
-    const uint32_t word = codes[size_t(j) * nwords + w];
-    const int g = (w * 16) / G;
-    const double zp = double(zero[size_t(j) * ng + g]);
-    double inner = 0.0;
-    for (int q = 0; q < 16; ++q) inner += (double((word >> (2 * q)) & 3u) - zp) * double(__bfloat162float(xt[w * 16 + q]));
-    acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
-  }
-  return acc;
-}
-
-// One thread per (token, neuron), one warp per flag word: flags from the fast scores; scores too close to a
-// range end are queued for exact re-evaluation (their bit is settled there).
-__global__ void k_flags(const float* __restrict__ zhat, const float* __restrict__ lo, const float* __restrict__ hi,
-                        const float* __restrict__ smaxrow, const float* __restrict__ x1, int n, int h,
-                        uint32_t* __restrict__ bitmap, uint2* __restrict__ rlist, unsigned int* __restrict__ rcount,
-                        const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
-                        const uint8_t* __restrict__ zero, const float* __restrict__ b1,
-                        const __nv_bfloat16* __restrict__ x, int d, int G) {
-  const size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x;     // n * h is a multiple of the block size
-  if (e >= size_t(n) * h) return;
-  const int t = int(e / h), j = int(e - size_t(t) * h);
-  const float xn = x1[t];
-  bool flag = true;                                                    // non-finite token: every neuron flagged
-  if (xn <= 3.0e38f) {
-    const float z = zhat[e], l = lo[j], u = hi[j];
-    const float tau = kEps * 3.f * smaxrow[j] * xn + 1e-30f;
-    flag = !((l <= z) && (z < u));
-    if (fabsf(z - l) <= tau || fabsf(z - u) <= tau) {
-      const unsigned int slot = atomicAdd(&rcount[0], 1u);
-      if (slot < (unsigned int)kMaxRecheck) rlist[slot] = make_uint2((unsigned int)t, (unsigned int)j);
-      else {                                                           // queue full: settle this one here (slow, but exact)
-        const double ze = exact_score_single(codes, scale, zero, x + size_t(t) * d, j, d, G) + double(b1[j]);
-        flag = !((double(l) <= ze) && (ze < double(u)));
-        atomicAdd(&rcount[1], 1u);
-      }
-    }
-  }
-  const uint32_t word = __ballot_sync(0xffffffffu, flag);
-  if ((threadIdx.x & 31) == 0) bitmap[e >> 5] = word;
-}
-
 // One warp per queued pair: exact fp64 score from the packed codes decides the flag.
 __global__ void k_recheck(const uint2* __restrict__ rlist, const unsigned int* __restrict__ rcount,
                           const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
@@ -167,7 +103,7 @@ __global__ void k_recheck(const uint2* __restrict__ rlist, const unsigned int* _
       uint32_t* wp = bitmap + size_t(t) * (h / 32) + (j >> 5);
       if (inside) atomicAnd(wp, ~(1u << (j & 31)));
       else atomicOr(wp, 1u << (j & 31));
-      zhat[size_t(t) * h + j] = float(z);
+      if (zhat) zhat[size_t(t) * h + j] = float(z);
     }
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -365,14 +301,18 @@ tardis_status_t launch_batched_forward(Handle* H, const void* xv, void* yv, int6
     GemmArgs g = {};
     g.M = n; g.N = h; g.K1 = d; g.K2 = d;
     g.A1 = xc; g.lda1 = d; g.B1 = S->What_hi; g.ldb1 = d; g.A2 = xc; g.lda2 = d; g.B2 = S->What_lo; g.ldb2 = d;
-    g.epilogue = GEMM_EPI_F32; g.out_f32 = S->zhat; g.ldo = h; g.bias = H->b1; g.error_word = &H->counters[CTR_ERROR];
+    // its epilogue turns the scores into flag words and queues the pairs too close to a range end; the scores
+    // themselves are stored only for the debug capture
+    const bool keep_scores = H->dbg_bitmap || H->dbg_scores;
+    g.epilogue = GEMM_EPI_FLAGS; g.out_f32 = keep_scores ? S->zhat : nullptr; g.ldo = h; g.bias = H->b1;
+    g.error_word = &H->counters[CTR_ERROR];
+    g.lo = H->lo; g.hi = H->hi; g.colscale = S->smaxrow; g.rowscale = S->x1; g.keps = kEps * 3.f;
+    g.bitmap_out = S->bitmap; g.rlist = S->rlist; g.rcount = S->rcount; g.rcap = kMaxRecheck;
+    g.codes = H->codes; g.scale = H->scale; g.zero = H->zero; g.xsrc = xc; g.d = d; g.G = H->G;
     tardis_status_t st = launch_gemm(g, s);
     if (st != TARDIS_OK) return st;
-    const size_t ne = size_t(n) * h;
-    k_flags<<<unsigned((ne + 255) / 256), 256, 0, s>>>(S->zhat, H->lo, H->hi, S->smaxrow, S->x1, n, h, S->bitmap, S->rlist, S->rcount,
-                                                       H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, H->b1, xc, d, H->G);
     k_recheck<<<H->num_sms * 4, 256, 0, s>>>(S->rlist, S->rcount, H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, H->b1,
-                                             H->lo, H->hi, xc, d, h, H->G, S->bitmap, S->zhat, H->counters);
+                                             H->lo, H->hi, xc, d, h, H->G, S->bitmap, keep_scores ? S->zhat : nullptr, H->counters);
     k_flag_counts<<<n, 256, 0, s>>>(S->bitmap, h / 32, H->counters);
     if (H->dbg_bitmap || H->dbg_scores) {
       const size_t cnt = size_t(n) * h;

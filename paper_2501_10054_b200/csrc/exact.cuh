@@ -1,0 +1,44 @@
+// Exact fp64 predictor sums (Section 5.3: s[j,g] (q - zp) x over the channels of neuron j, without the bias) from the
+// packed 2-bit codes: what decides a flag when a fast score is too close to a range end.
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace tardis {
+
+// one warp; every lane returns the sum
+__device__ inline double exact_score(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
+                              const uint8_t* __restrict__ zero, const __nv_bfloat16* __restrict__ xt, int j, int d, int G,
+                              int lane) {   // one warp; every lane returns the sum
+  const int nwords = d / 16, ng = d / G;
+  double acc = 0.0;
+  for (int w = lane; w < nwords; w += 32) {
+    const uint32_t word = codes[size_t(j) * nwords + w];
+    const int g = (w * 16) / G;
+    const double zp = double(zero[size_t(j) * ng + g]);
+    double inner = 0.0;
+#pragma unroll
+    for (int q = 0; q < 16; ++q) inner += (double((word >> (2 * q)) & 3u) - zp) * double(__bfloat162float(xt[w * 16 + q]));
+    acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  return acc;
+}
+
+__device__ inline double exact_score_single(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
+                                     const uint8_t* __restrict__ zero, const __nv_bfloat16* __restrict__ xt, int j, int d, int G) {
+  const int nwords = d / 16, ng = d / G;
+  double acc = 0.0;
+  for (int w = 0; w < nwords; ++w) {
+    const uint32_t word = codes[size_t(j) * nwords + w];
+    const int g = (w * 16) / G;
+    const double zp = double(zero[size_t(j) * ng + g]);
+    double inner = 0.0;
+    for (int q = 0; q < 16; ++q) inner += (double((word >> (2 * q)) & 3u) - zp) * double(__bfloat162float(xt[w * 16 + q]));
+    acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
+  }
+  return acc;
+}
+
+}  // namespace tardis

@@ -15,6 +15,7 @@
 #include <stdio.h>
 
 #include "common.cuh"
+#include "exact.cuh"
 
 namespace tardis {
 namespace gemm {
@@ -109,17 +110,77 @@ struct KParams {
   const float *bias, *addend, *a, *c;
   const uint32_t* bitmap;
   unsigned long long* error_word;
+  const float *lo, *hi, *colscale, *rowscale;
+  float keps;
+  uint32_t* bitmap_out;
+  uint2* rlist; unsigned int* rcount; int rcap;
+  const uint32_t* codes; const __nv_bfloat16* scale; const uint8_t* zero;
+  const __nv_bfloat16* xsrc; int d, G;
 };
 
 template <int BN> struct Cfg {
   static constexpr int STAGE_BYTES = BM * BK * 2 + BN * BK * 2;
   static constexpr int NS = (BN == 256) ? 4 : 6;                      // stages
-  static constexpr int SMEM = NS * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+  static constexpr int SMEM = NS * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + 4 * 4096 /* epilogue staging */;
   static constexpr int TMEM_COLS = 2 * BN;                            // two accumulators
 };
 
 // The epilogue of 32 consecutive columns n .. n + nv - 1 of output row m (one thread).
-__device__ __forceinline__ void epilogue_chunk(const KParams& p, float (&v)[32], int m, int n, int nv, bool first_split, bool have_acc) {
+// A&S 7.1.26 form of erf (absolute error below 2e-7, far inside the bf16 rounding of the correction it feeds)
+__device__ __forceinline__ float gelu_quick(float z, int act) {
+  if (act == TARDIS_ACT_GELU_TANH) return gelu_f32(z, act);
+  const float x = fabsf(z) * 0.7071067811865476f;
+  const float t = __fdividef(1.f, fmaf(0.3275911f, x, 1.f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float e = 1.f - poly * t * __expf(-x * x);          // erf(|z| / sqrt 2)
+  return 0.5f * z * (1.f + copysignf(e, z));
+}
+
+// `stage`: 32 x 32 floats of shared memory of the calling warp (element [i][lane]).
+__device__ __forceinline__ void epilogue_chunk(const KParams& p, float (&v)[32], int m, int n, int nv, bool first_split, bool have_acc,
+                                               float* stage, int lane) {
+  if (p.epilogue == GEMM_EPI_FLAGS) {
+    const float xn = p.rowscale[m];
+    const uint32_t valid = nv == 32 ? 0xffffffffu : ((1u << nv) - 1u);
+    uint32_t word = valid;                                   // a non-finite token: every neuron flagged
+    if (xn <= 3.0e38f) {
+      const float kx = p.keps * xn;
+      word = 0u;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        if (i < nv) {
+          const float z = v[i] + p.bias[n + i], l = p.lo[n + i], u = p.hi[n + i];
+          const float tau = fmaf(p.colscale[n + i], kx, 1e-30f);
+          bool flag = !((l <= z) && (z < u));
+          if (fabsf(z - l) <= tau || fabsf(z - u) <= tau) {  // rare
+            const unsigned int slot = atomicAdd(&p.rcount[0], 1u);
+            if (slot < (unsigned int)p.rcap) p.rlist[slot] = make_uint2((unsigned int)m, (unsigned int)(n + i));
+            else {                                           // queue full: settle this one here (slow, but exact)
+              const double ze = exact_score_single(p.codes, p.scale, p.zero, p.xsrc + size_t(m) * p.d, n + i, p.d, p.G) + double(p.bias[n + i]);
+              flag = !((double(l) <= ze) && (ze < double(u)));
+              atomicAdd(&p.rcount[1], 1u);
+            }
+          }
+          word |= (flag ? 1u : 0u) << i;
+          v[i] = z;
+        }
+      }
+    }
+    p.bitmap_out[size_t(m) * (p.N / 32) + (n >> 5)] = word;
+    if (p.out_f32) {
+      float* o = p.out_f32 + size_t(m) * p.ldo + n;
+      if (nv == 32 && (p.ldo & 3) == 0) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(o + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+      } else {
+        for (int i = 0; i < nv; ++i) o[i] = v[i];
+      }
+    }
+    return;
+  }
   if (p.epilogue == GEMM_EPI_F32 && p.splits > 1) {
     float* o = p.out_f32 + size_t(m) * p.ldo + n;
     const bool with_bias = p.bias && first_split;
@@ -161,16 +222,20 @@ __device__ __forceinline__ void epilogue_chunk(const KParams& p, float (&v)[32],
         for (int i = 0; i < nv; ++i) v[i] += ad[i];
       }
     } else {   // GEMM_EPI_DELTA: one flag word covers this thread's 32 columns
-      const uint32_t word = p.bitmap[size_t(m) * (p.N / 32) + (n >> 5)];
-#pragma unroll 8
-      for (int i = 0; i < 32; ++i) {
-        float dl = 0.f;
-        if (((word >> i) & 1u) && i < nv) {
-          const float z = v[i] + (p.bias ? p.bias[n + i] : 0.f);
-          dl = gelu_f32(z, p.act) - p.a[n + i] * z - p.c[n + i];
-        }
-        v[i] = dl;
+      // Only the flagged tenth of the elements needs the activation, at different columns in every row: the
+      // accumulators go to shared memory, each thread walks the set bits of its own word, and the corrections come
+      // back under the word's mask.
+      uint32_t word = p.bitmap[size_t(m) * (p.N / 32) + (n >> 5)];
+      if (nv < 32) word &= (1u << nv) - 1u;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) stage[i * 32 + lane] = v[i];
+      for (uint32_t w = word; w; w &= w - 1u) {
+        const int i = __ffs(w) - 1;
+        const float z = stage[i * 32 + lane] + (p.bias ? p.bias[n + i] : 0.f);
+        stage[i * 32 + lane] = gelu_quick(z, p.act) - p.a[n + i] * z - p.c[n + i];
       }
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = ((word >> i) & 1u) ? stage[i * 32 + lane] : 0.f;
     }
     __nv_bfloat16* o = p.out_bf16 + size_t(m) * p.ldo + n;
     if (nv == 32 && (p.ldo & 7) == 0) {
@@ -292,6 +357,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtenso
   } else {
     // ---------------- epilogue: warp q reads TMEM lanes 32 (warp % 4) .. + 31 ----------------
     const int q = warp & 3;
+    float* const stage = reinterpret_cast<float*>(smem + C::NS * C::STAGE_BYTES + 256) + q * 1024;
     uint32_t use = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
@@ -313,7 +379,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtenso
         }
         const int n = n0 + ch * 32;
         const int nv = min(32, p.N - n);
-        if (m < p.M && nv > 0) epilogue_chunk(p, v, m, n, nv, z == 0, nkb > 0);   // (no early exit: tcgen05.ld needs the whole warp)
+        if (m < p.M && nv > 0) epilogue_chunk(p, v, m, n, nv, z == 0, nkb > 0, stage, lane);   // (no early exit: tcgen05.ld needs the whole warp)
       }
       if (nkb > 0) {
         tc_fence_before();
@@ -374,6 +440,9 @@ static tardis_status_t launch_bn(const GemmArgs& g, cudaStream_t s) {
   p.epilogue = g.epilogue; p.ldo = g.ldo; p.act = g.act; p.splits = g.splits > 1 ? g.splits : 1;
   p.out_f32 = g.out_f32; p.out_bf16 = static_cast<__nv_bfloat16*>(g.out_bf16);
   p.bias = g.bias; p.addend = g.addend; p.a = g.a; p.c = g.c; p.bitmap = g.bitmap; p.error_word = g.error_word;
+  p.lo = g.lo; p.hi = g.hi; p.colscale = g.colscale; p.rowscale = g.rowscale; p.keps = g.keps; p.bitmap_out = g.bitmap_out;
+  p.rlist = g.rlist; p.rcount = g.rcount; p.rcap = g.rcap; p.codes = g.codes; p.scale = static_cast<const __nv_bfloat16*>(g.scale);
+  p.zero = g.zero; p.xsrc = static_cast<const __nv_bfloat16*>(g.xsrc); p.d = g.d; p.G = g.G;
   TARDIS_CUDA_TRY(cudaFuncSetAttribute(k_gemm<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM));
   const long tiles = long((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * p.splits;
   int dev = 0, sms = 0;
@@ -394,7 +463,10 @@ tardis_status_t launch_gemm(const GemmArgs& g, cudaStream_t s) {
   auto bad = [](const void* p, int ld, int K) { return !p || (reinterpret_cast<uintptr_t>(p) & 15u) || (ld & 7) || (K & 7) || ld < K; };
   if (bad(g.A1, g.lda1, g.K1) || bad(g.B1, g.ldb1, g.K1)) return TARDIS_ERR_INVALID_ARG;
   if (g.K2 > 0 && (bad(g.A2, g.lda2, g.K2) || bad(g.B2, g.ldb2, g.K2))) return TARDIS_ERR_INVALID_ARG;
-  if (g.epilogue == GEMM_EPI_DELTA && (g.N % 32)) return TARDIS_ERR_INVALID_ARG;
+  if ((g.epilogue == GEMM_EPI_DELTA || g.epilogue == GEMM_EPI_FLAGS) && (g.N % 32)) return TARDIS_ERR_INVALID_ARG;
+  if (g.epilogue == GEMM_EPI_FLAGS && !(g.bias && g.lo && g.hi && g.colscale && g.rowscale && g.bitmap_out && g.rlist && g.rcount &&
+                                         g.codes && g.scale && g.zero && g.xsrc))
+    return TARDIS_ERR_INVALID_ARG;
   if (g.splits > 1 && g.epilogue != GEMM_EPI_F32) return TARDIS_ERR_INVALID_ARG;
   // wide tiles when they still fill the machine, narrow ones for skinny problems
   const long tiles256 = long((g.N + 255) / 256) * ((g.M + BM - 1) / BM) * (g.splits > 1 ? g.splits : 1);

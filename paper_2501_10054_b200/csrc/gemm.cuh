@@ -13,7 +13,11 @@ namespace tardis {
 enum GemmEpilogue {
   GEMM_EPI_F32 = 0,        // out_f32[m, n] = acc + (bias ? bias[n] : 0)
   GEMM_EPI_ADD_BF16 = 1,   // out_bf16[m, n] = bf16(acc + addend_f32[m, n])
-  GEMM_EPI_DELTA = 2       // z = acc + bias[n]; out_bf16[m, n] = flagged(m, n) ? GELU(z) - a[n] z - c[n] : 0
+  GEMM_EPI_DELTA = 2,      // z = acc + bias[n]; out_bf16[m, n] = flagged(m, n) ? GELU(z) - a[n] z - c[n] : 0
+  GEMM_EPI_FLAGS = 3       // z = acc + bias[n]; bit (m, n) of bitmap_out = !(lo[n] <= z < hi[n]); a z within
+                           // keps * colscale[n] * rowscale[m] of lo[n] or hi[n] is queued in rlist for exact
+                           // re-evaluation (settled in place from the codes when the queue is full); a row whose
+                           // rowscale is not finite is flagged throughout; z is also stored when out_f32 is given
 };
 
 struct GemmArgs {
@@ -31,6 +35,13 @@ struct GemmArgs {
   const uint32_t* bitmap;           // [M, N / 32] flag words (GEMM_EPI_DELTA)
   int act;
   unsigned long long* error_word;   // device counter slot that receives 1 when a bounded wait runs out
+  // GEMM_EPI_FLAGS
+  const float *lo, *hi, *colscale, *rowscale;   // [N], [N], [N], [M]
+  float keps;
+  uint32_t* bitmap_out;             // [M, N / 32]
+  uint2* rlist; unsigned int* rcount; int rcap;   // queue of (m, n) pairs, its fill count ([1]: pairs settled in place), capacity
+  const uint32_t* codes; const void* scale; const uint8_t* zero;   // the packed predictor (rows n)
+  const void* xsrc; int d, G;       // the bf16 rows A1 came from (leading dimension d), group size
 };
 
 // Enqueues the GEMM on `s`.  Returns UNSUPPORTED when the tensor-map entry point of the driver is not
