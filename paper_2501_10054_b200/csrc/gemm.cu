@@ -106,6 +106,7 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N) {
 struct KParams {
   int M, N, kb1, kb2;          // k blocks (of 64) of the two operand pairs
   int epilogue, ldo, act, splits;
+  int fast_m, band;            // tile raster (see decode() in the kernel)
   float* out_f32; __nv_bfloat16* out_bf16;
   const float *bias, *addend, *a, *c;
   const uint32_t* bitmap;
@@ -252,9 +253,8 @@ __device__ __forceinline__ void epilogue_chunk(const KParams& p, float (&v)[32],
   }
 }
 
-// Persistent: CTA c works on tiles c, c + gridDim.x, ... (row tiles fastest, so that the CTAs running at the same
-// time share few column blocks of B).  Two accumulators in tensor memory: while the epilogue warps drain one, the
-// MMA warp is already filling the other with the next tile.
+// Persistent: CTA c works on tiles c, c + gridDim.x, ... of a banded raster.  Two accumulators in tensor memory:
+// while the epilogue warps drain one, the MMA warp is already filling the other with the next tile.
 template <int BN>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
@@ -293,7 +293,13 @@ k_gemm(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtenso
   auto decode = [&](int tile, int& m0, int& n0, int& kb_lo, int& nkb, int& z) {
     z = tile / (nm * nn);
     const int rem = tile - z * (nm * nn);
-    const int ni = rem / nm, mi = rem - ni * nm;
+    // raster: bands of `band` tiles along the dimension with fewer tiles, walked across the other dimension, so
+    // that the CTAs running at the same time cover a compact block and share its operand tiles in L2
+    const int F = p.fast_m ? nm : nn, S = p.fast_m ? nn : nm;
+    const int bi = rem / (p.band * S), r2 = rem - bi * (p.band * S);
+    const int w = min(p.band, F - bi * p.band);
+    const int slow = r2 / w, fast = bi * p.band + (r2 - slow * w);
+    const int mi = p.fast_m ? fast : slow, ni = p.fast_m ? slow : fast;
     m0 = mi * BM; n0 = ni * BN;
     kb_lo = z * per;
     nkb = max(0, min(nkb_all, kb_lo + per) - kb_lo);
@@ -444,7 +450,11 @@ static tardis_status_t launch_bn(const GemmArgs& g, cudaStream_t s) {
   p.rlist = g.rlist; p.rcount = g.rcount; p.rcap = g.rcap; p.codes = g.codes; p.scale = static_cast<const __nv_bfloat16*>(g.scale);
   p.zero = g.zero; p.xsrc = static_cast<const __nv_bfloat16*>(g.xsrc); p.d = g.d; p.G = g.G;
   TARDIS_CUDA_TRY(cudaFuncSetAttribute(k_gemm<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM));
-  const long tiles = long((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * p.splits;
+  const int nm = (g.M + BM - 1) / BM, nn = (g.N + BN - 1) / BN;
+  p.fast_m = nm <= nn ? 1 : 0;
+  const int fcount = p.fast_m ? nm : nn;
+  p.band = fcount <= 16 ? fcount : 12;
+  const long tiles = long(nm) * nn * p.splits;
   int dev = 0, sms = 0;
   TARDIS_CUDA_TRY(cudaGetDevice(&dev));
   TARDIS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
