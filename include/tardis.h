@@ -176,7 +176,9 @@ tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf
                                      tardis_stream_t stream);
 
 /* Chooses the kernel path: 0 = automatic (default), 1 = always the generic
- * kernels.  For testing one path against the other. */
+ * kernels, 3 = the batched tensor-core path for every token count (bf16
+ * layers; other layers fall back to the generic kernels).  For testing one
+ * path against the other. */
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
 
 /* Frees everything the handle owns (synchronises the device first). */

@@ -130,7 +130,7 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   H->last_stream = s;
   tardis_status_t st;
   const bool fused = H->path_override == 0 && H->codes_mma != nullptr && n_tokens <= kDecodeMaxTokens;
-  const bool batched = H->path_override == 0 && !fused && H->bstate != nullptr;
+  const bool batched = ((H->path_override == 0 && !fused) || H->path_override == 3) && H->bstate != nullptr;
   if (fused) {
     st = launch_decode_forward(H, x, y, int(n_tokens), s);
     H->last_path = 2;
@@ -214,7 +214,7 @@ tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf
 
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path) {
   Handle* H = check(handle);
-  if (!H || path < 0 || path > 1) return TARDIS_ERR_INVALID_ARG;
+  if (!H || !(path == 0 || path == 1 || path == 3)) return TARDIS_ERR_INVALID_ARG;
   H->path_override = path;
   return TARDIS_OK;
 }
