@@ -3,9 +3,11 @@
 //
 // For a chunk of up to kChunk tokens X[n, d]:
 //   1. fast predictor scores  Zhat = X What^T + b1, What = s (q - zp) (Section 5.3).  What needs 10 significant
-//      bits, so it is held as an exact sum of two bf16 matrices (hi + lo); one GEMM runs over both.  Products
+//      bits, so it is held as an exact sum of two bf16 matrices (hi + lo); one GEMM runs over both and its
+//      epilogue turns the scores into flag words (they are stored only for the debug capture).  Products
 //      are exact, the fp32 accumulation is not: a score within tau(t, j) = kEps * 3 max_g s[j,g] * |x_t|_1 of a
-//      range end is re-evaluated in fp64 from the packed codes (k_recheck), so the flags are the exact ones;
+//      range end is queued by the epilogue and re-evaluated in fp64 from the packed codes (k_recheck), so the
+//      flags are the exact ones;
 //   2. speculative product    Yacc = X W_f^T + b_f                               (fp32);
 //   3. result fixing          Delta = flag .* (GELU(Z) - a Z - c), Z = X W1^T + b1   (GEMM with that epilogue, bf16),
 //                             y = bf16(Yacc + Delta W2^T)                            (GEMM over all neurons:
