@@ -6,8 +6,8 @@
 //   * Prologue (before griddepcontrol.wait, so it overlaps the tail of the previous launch in the
 //     stream): a CTA owns a few 16-neuron tiles; their predictor blocks (packed 2-bit codes + group
 //     words) are one contiguous region per tile and are fetched with a few large bulk async copies
-//     (cp.async.bulk + mbarrier) into shared memory; the CTA's share of the folded matrix is
-//     prefetched into L2 (cp.async.bulk.prefetch.L2).  Both read constant state of the layer only.
+//     (cp.async.bulk + mbarrier) into shared memory.  They read constant state of the layer only.
+//     (Prefetching the folded matrix into L2 here as well was measured: no gain, left out.)
 //   * x is loaded once: a bf16 copy in shared memory, and a 4-limb signed base-256 fixed-point copy in
 //     tensor-core operand order.
 //   * Then the warps split.  Warps 0..7 evaluate the predictor on the integer tensor cores: the codes are
@@ -257,10 +257,6 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   __syncthreads();
   // predictor blocks first: nothing of them depends on x
   if (lane == 0 && warp < p.nbuf && warp < NU) issue_unit(warp);
-  // and this CTA's share of the folded matrix goes to L2, from where the streaming warps (of any CTA) take it
-  if (lane == 0 && warp >= NWP)
-    for (int u = blockIdx.x * (NW - NWP) + (warp - NWP); u < p.nunits; u += gridDim.x * (NW - NWP))
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.Cp + size_t(u) * 512), "r"(8192) : "memory");
 
   // From here on the kernel touches what earlier work in the stream may still be writing (x, the
   // scratch shared by the calls of one handle): wait until that work has completed and is visible.
