@@ -22,8 +22,10 @@ the per-neuron linear function on the half-open range [l1, l2) = [lo_j, hi_j)
 Pins (tests, CPU only): the worked two-neuron example of Section 4.2, the fold
 example of Section 3.1, the linear-activation identity, the all-flagged = dense
 GELU FFN identity, brute force over every flag subset for d, h <= 16, the
-exact-predictor special case, closed forms of GELU, the packing convention.
-No function in this file is "parity unpinned".
+exact-predictor special case, closed forms of GELU, the packing convention;
+for the offline range / fit functions: the quantile routine of numpy, arithmetic
+sequences, the normal equations, numpy's polynomial fit, two-sample lines and
+the analytic tangent.  No function in this file is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -248,3 +250,80 @@ def rel_error(y, y_ref):
     den = np.maximum(np.abs(y_ref), rms)
     den = np.where(den > 0, den, 1.0)
     return np.abs(y - y_ref) / den
+
+
+# --------------------------------------------------------------------------
+# offline: per-neuron range and linear fit from calibration pre-activations
+# --------------------------------------------------------------------------
+def quantile_ranges(z, q_lo, q_hi):
+    """Range of every neuron as "the input range containing a certain portion
+    of activation inputs based on the profiled distribution" (Section 3.2,
+    Insight 2): the central portion between the q_lo and q_hi quantiles of the
+    neuron's calibration pre-activations.  z[h, N]: row j = the N samples of
+    neuron j.  The quantile at level p is the linear interpolation between the
+    order statistics around position p (N - 1).  (The greedy search of
+    Algorithm 1 is a different way to pick the same kind of range; the
+    configurations of this repository use quantiles.)  Returns (lo, hi) as
+    float32 arrays: the range is stored in single precision."""
+    z = _as64(z)
+    h, N = z.shape
+    zs = np.sort(z, axis=1)
+    out = []
+    for p in (q_lo, q_hi):
+        pos = float(p) * (N - 1)
+        i0 = int(math.floor(pos))
+        i1 = min(i0 + 1, N - 1)
+        w = pos - i0
+        out.append((zs[:, i0] * (1.0 - w) + zs[:, i1] * w).astype(np.float32))
+    return out[0], out[1]
+
+
+def gelu_derivative(z, act=ACT_GELU_TANH):
+    """d/dz GELU(z), analytic, float64."""
+    z = np.asarray(z, dtype=_F64)
+    if act == ACT_GELU_TANH:
+        k = math.sqrt(2.0 / math.pi)
+        u = k * (z + 0.044715 * z ** 3)
+        t = np.tanh(u)
+        return 0.5 * (1.0 + t) + 0.5 * z * (1.0 - t * t) * k * (1.0 + 3.0 * 0.044715 * z * z)
+    if act == ACT_GELU_ERF:
+        from scipy.special import erf
+        return 0.5 * (1.0 + erf(z / math.sqrt(2.0))) + z * np.exp(-0.5 * z * z) / math.sqrt(2.0 * math.pi)
+    raise ValueError("unknown activation %r" % (act,))
+
+
+def least_squares_fit(z, lo, hi, act=ACT_GELU_TANH):
+    """The linear function y = a z + c of every neuron, "obtained using least
+    squares regression" (Section 4.1 step 3, Section 5.1.2 step 4) of GELU(z)
+    on z over the calibration samples inside the neuron's range lo <= z < hi:
+        a = cov(z, GELU(z)) / var(z),   c = mean(GELU(z)) - a mean(z).
+    A neuron with fewer than two samples in range, or whose in-range samples
+    have variance below 1e-30, takes the tangent of GELU at the range midpoint.
+    z[h, N] float (samples as stored, i.e. float32 values), lo/hi[h] float32.
+    Returns (a, c) as float32 arrays."""
+    z = _as64(z)
+    lo64, hi64 = _as64(lo), _as64(hi)
+    h, N = z.shape
+    a = np.empty(h, dtype=np.float32)
+    c = np.empty(h, dtype=np.float32)
+    for j in range(h):
+        zj = z[j]
+        inside = (zj >= lo64[j]) & (zj < hi64[j])
+        zz = zj[inside]
+        ok = False
+        if zz.size >= 2:
+            sg = gelu(zz, act)
+            mz, ms = zz.mean(), sg.mean()
+            var = ((zz - mz) ** 2).mean()
+            if var > 1e-30:
+                cov = ((zz - mz) * (sg - ms)).mean()
+                aj = cov / var
+                cj = ms - aj * mz
+                ok = True
+        if not ok:
+            mid = 0.5 * (lo64[j] + hi64[j])
+            aj = float(gelu_derivative(mid, act))
+            cj = float(gelu(mid, act)) - aj * mid
+        a[j] = np.float32(aj)
+        c[j] = np.float32(cj)
+    return a, c

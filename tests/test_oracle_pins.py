@@ -301,3 +301,66 @@ def test_rel_error_metric():
     y_ref = np.array([[3.0, 4.0, 0.0, 0.0]])            # rms = 2.5
     y = y_ref + np.array([[0.3, 0.0, 0.25, 0.0]])
     np.testing.assert_allclose(O.rel_error(y, y_ref)[0], [0.1, 0.0, 0.1, 0.0])
+
+
+# ---- offline range / fit functions -------------------------------------------------------------------
+def test_quantile_ranges_match_numpy_and_arithmetic_sequences():
+    rng = np.random.default_rng(5)
+    z = rng.standard_normal((7, 257)).astype(np.float32)
+    lo, hi = O.quantile_ranges(z, 0.05, 0.95)
+    ref_lo = np.quantile(z.astype(np.float64), 0.05, axis=1, method="linear")
+    ref_hi = np.quantile(z.astype(np.float64), 0.95, axis=1, method="linear")
+    assert lo.dtype == np.float32 and hi.dtype == np.float32
+    assert np.array_equal(lo, ref_lo.astype(np.float32)) and np.array_equal(hi, ref_hi.astype(np.float32))
+    # samples 0, 1, ..., N-1 in any order: the quantile at level p is p (N - 1) itself
+    N = 101
+    seq = rng.permutation(N).astype(np.float64)[None, :]
+    lo, hi = O.quantile_ranges(seq, 0.125, 0.9)
+    assert lo[0] == np.float32(12.5) and hi[0] == np.float32(90.0)
+    # p = 0 and p = 1 are the extremes; one sample: both ends are that sample
+    lo, hi = O.quantile_ranges(z, 0.0, 1.0)
+    assert np.array_equal(lo, z.min(1)) and np.array_equal(hi, z.max(1))
+    lo, hi = O.quantile_ranges(np.array([[3.0]]), 0.3, 0.6)
+    assert lo[0] == 3.0 and hi[0] == 3.0
+
+
+@pytest.mark.parametrize("act", [O.ACT_GELU_TANH, O.ACT_GELU_ERF])
+def test_least_squares_fit_normal_equations_polyfit_and_range_rule(act):
+    rng = np.random.default_rng(6)
+    z = (rng.standard_normal((5, 400)) * 1.3).astype(np.float32)
+    lo = np.array([-1.0, -0.5, -2.0, 0.0, -3.0], dtype=np.float32)
+    hi = np.array([0.5, 0.25, 2.0, 1.5, 3.0], dtype=np.float32)
+    a, c = O.least_squares_fit(z, lo, hi, act)
+    for j in range(5):
+        zz = z[j].astype(np.float64)
+        zz = zz[(zz >= lo[j]) & (zz < hi[j])]
+        sg = O.gelu(zz, act)
+        # library cross-check: degree-1 polynomial least squares
+        pa, pc = np.polyfit(zz, sg, 1)
+        assert abs(a[j] - pa) <= 2e-6 * max(1.0, abs(pa)) and abs(c[j] - pc) <= 2e-6 * max(1.0, abs(pc))
+        # normal equations: the residual is orthogonal to 1 and to z (float32 rounding of a, c allowed for)
+        r = sg - (float(a[j]) * zz + float(c[j]))
+        assert abs(r.sum()) <= 1e-5 * zz.size and abs((r * zz).sum()) <= 1e-5 * zz.size
+    # half-open range: a sample equal to hi is outside, one equal to lo is inside
+    zz = np.array([[0.0, 1.0, 2.0, 5.0]])
+    a1, c1 = O.least_squares_fit(zz, np.array([0.0], np.float32), np.array([2.0], np.float32), act)
+    g0, g1 = O.gelu(0.0, act), O.gelu(1.0, act)
+    assert abs(a1[0] - (g1 - g0)) < 1e-6 and abs(c1[0] - g0) < 1e-6          # the line through the two samples in range
+
+
+@pytest.mark.parametrize("act", [O.ACT_GELU_TANH, O.ACT_GELU_ERF])
+def test_least_squares_fit_degenerate_takes_the_tangent_at_the_midpoint(act):
+    # no sample in range / a single one / identical ones: tangent of GELU at (lo + hi) / 2
+    z = np.array([[5.0, 6.0, 7.0], [0.25, 9.0, 9.5], [0.5, 0.5, 0.5]])
+    lo = np.array([-1.0, 0.0, 0.0], np.float32)
+    hi = np.array([1.0, 1.0, 1.0], np.float32)
+    a, c = O.least_squares_fit(z, lo, hi, act)
+    for j in range(3):
+        m = 0.5 * (float(lo[j]) + float(hi[j]))
+        eps = 1e-6
+        slope = (O.gelu(m + eps, act) - O.gelu(m - eps, act)) / (2 * eps)      # derivative pinned numerically
+        assert abs(a[j] - slope) < 1e-6 and abs(c[j] - (O.gelu(m, act) - slope * m)) < 1e-6
+    # a neuron that is linear where it is sampled: GELU(z) -> z for large z, so a -> 1, c -> 0
+    zz = np.linspace(20.0, 30.0, 50)[None, :]
+    a, c = O.least_squares_fit(zz, np.array([0.0], np.float32), np.array([100.0], np.float32), act)
+    assert abs(a[0] - 1.0) < 1e-6 and abs(c[0]) < 1e-5
