@@ -175,6 +175,28 @@ tardis_status_t tardis_set_debug_capture(tardis_handle_t handle, uint32_t* flag_
 tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf,
                                      tardis_stream_t stream);
 
+/* Offline statistics of one layer: the range and the linear function of every
+ * neuron from calibration pre-activations.  The paper picks, per neuron, the
+ * input range that holds a given portion of the profiled activation inputs and
+ * fits y = a z + c to the activation inside it by least squares (Section 3.2,
+ * Insight 2; Section 4.1 step 3; Section 5.1.2 step 4).  Here the range is
+ * the one between the quantiles q_lo and q_hi of the neuron's samples (linear
+ * interpolation between the order statistics around position q (n_cal - 1),
+ * evaluated in double precision, stored in single); the fit is ordinary least
+ * squares of GELU(z) on z over the samples with lo <= z < hi, in double
+ * precision; a neuron with fewer than two samples in range (or in-range
+ * variance below 1e-30) takes the tangent of GELU at (lo + hi) / 2.
+ *   z      device [d_ff, n_cal] float, row j = samples of neuron j, leading
+ *          dimension ldz >= n_cal (e.g. the output of tardis_gemm_bf16 with
+ *          A = W1, B = calibration tokens); samples must be finite
+ *   b1     device [d_ff] added to the samples, or NULL
+ *   lo, hi, a, c   device [d_ff] float, outputs (what tardis_fold takes)
+ * 1 <= n_cal <= 8192 (TARDIS_ERR_UNSUPPORTED beyond), 0 <= q_lo <= q_hi <= 1.
+ * Asynchronous on `stream`; allocates nothing; nothing is kept. */
+tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, int64_t ldz, const float* b1,
+                                 double q_lo, double q_hi, int32_t act, float* lo, float* hi, float* a, float* c,
+                                 tardis_stream_t stream);
+
 /* Chooses the kernel path: 0 = automatic (default), 1 = always the generic
  * kernels, 3 = the batched tensor-core path for every token count (bf16
  * layers; other layers fall back to the generic kernels).  For testing one

@@ -21,7 +21,7 @@ TARDIS_F32, TARDIS_BF16 = 0, 1
 TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF = 0, 1
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
-           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy",
+           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_calibrate",
            "tardis_status_string", "tardis_last_error"]
 
 
@@ -74,7 +74,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_set_path.argtypes = [vp, i32]
     lib.tardis_destroy.argtypes = [vp]
     lib.tardis_gemm_bf16.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, i32, vp]
-    for name in EXPORTS[:9]:
+    lib.tardis_calibrate.argtypes = [i32, i32, vp, i64, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp]
+    for name in EXPORTS[:10]:
         getattr(lib, name).restype = ctypes.c_int
     lib.tardis_status_string.argtypes = [ctypes.c_int]
     lib.tardis_status_string.restype = ctypes.c_char_p
@@ -156,6 +157,19 @@ def tardis_gemm_bf16(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, stream=N
     _check(lib.tardis_gemm_bf16(M, N, K, A.data_ptr(), A.stride(0), B.data_ptr(), B.stride(0), C.data_ptr(), C.stride(0),
                                 _stream(stream)), "tardis_gemm_bf16")
     return C
+
+
+def tardis_calibrate(z: torch.Tensor, b1: Optional[torch.Tensor], q_lo: float, q_hi: float, act: int, stream=None):
+    """Per-neuron ranges and linear fits from calibration pre-activations z[d_ff, n_cal] (float32, CUDA, unit inner
+    stride): returns (lo, hi, a, c), float32 tensors of d_ff elements on z's device."""
+    if z.dtype != torch.float32 or not z.is_cuda or z.stride(1) != 1:
+        raise TardisError(1, "z must be a float32 CUDA tensor with unit inner stride")
+    h, n = z.shape
+    out = [torch.empty(h, dtype=torch.float32, device=z.device) for _ in range(4)]
+    _check(load_library().tardis_calibrate(h, n, z.data_ptr(), z.stride(0), _ptr(b1), float(q_lo), float(q_hi), int(act),
+                                           out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), out[3].data_ptr(),
+                                           _stream(stream)), "tardis_calibrate")
+    return tuple(out)
 
 
 def tardis_stats(handle: int) -> dict:

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtardis.so")
-SOURCES = ["api.cu", "fold.cu", "generic.cu", "decode.cu", "gemm.cu", "batched.cu"]
+SOURCES = ["api.cu", "fold.cu", "generic.cu", "decode.cu", "gemm.cu", "batched.cu", "calibrate.cu"]
 
 
 def nvcc_path() -> str:

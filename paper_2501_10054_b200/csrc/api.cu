@@ -177,6 +177,14 @@ tardis_status_t tardis_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A,
   return launch_gemm(g, reinterpret_cast<cudaStream_t>(stream));
 }
 
+tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, int64_t ldz, const float* b1, double q_lo,
+                                 double q_hi, int32_t act, float* lo, float* hi, float* a, float* c, tardis_stream_t stream) {
+  if (d_ff <= 0 || n_cal <= 0 || !z || ldz < n_cal || !lo || !hi || !a || !c) return TARDIS_ERR_INVALID_ARG;
+  if (!(q_lo >= 0.0 && q_lo <= q_hi && q_hi <= 1.0)) return TARDIS_ERR_INVALID_ARG;
+  if (act != TARDIS_ACT_GELU_TANH && act != TARDIS_ACT_GELU_ERF) return TARDIS_ERR_INVALID_ARG;
+  return launch_calibrate(d_ff, n_cal, z, ldz, b1, q_lo, q_hi, act, lo, hi, a, c, reinterpret_cast<cudaStream_t>(stream));
+}
+
 tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
   Handle* H = check(handle);
   if (!H || !out) return TARDIS_ERR_INVALID_ARG;

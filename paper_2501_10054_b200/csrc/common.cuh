@@ -85,6 +85,10 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+// offline statistics (calibrate.cu)
+tardis_status_t launch_calibrate(int h, int n, const float* z, long long ldz, const float* b1, double q_lo, double q_hi, int act,
+                                 float* lo, float* hi, float* a, float* c, cudaStream_t s);
+
 __device__ __forceinline__ float gelu_f32(float z, int act) {
   if (act == TARDIS_ACT_GELU_TANH) {
     float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);

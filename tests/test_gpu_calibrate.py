@@ -1,0 +1,88 @@
+"""GPU parity of the offline statistics (tardis_calibrate) against the oracle, through the C ABI.
+
+Both sides get the same float32 pre-activations, so every decision that float arithmetic makes for an integer
+(which samples lie inside [lo, hi)) is taken on identical numbers: the ranges must agree bit for bit, the fits
+within the float32 rounding of sums taken in a different order."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2501_10054_b200 as T
+import workloads as W
+from oracle import tardis_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(z, b1, q_lo, q_hi, act):
+    lo, hi, a, c = T.tardis_calibrate(z, b1, q_lo, q_hi, act)
+    torch.cuda.synchronize()
+    zc = z.cpu().numpy()
+    if b1 is not None:
+        zc = zc + b1.cpu().numpy()[:, None]                     # float32 sum, as the kernel forms it
+    lo_ref, hi_ref = O.quantile_ranges(zc, q_lo, q_hi)
+    a_ref, c_ref = O.least_squares_fit(zc, lo_ref, hi_ref, act)
+    assert np.array_equal(lo.cpu().numpy(), lo_ref) and np.array_equal(hi.cpu().numpy(), hi_ref)
+    a, c = a.cpu().numpy().astype(np.float64), c.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(a - a_ref) <= 2e-6 * np.maximum(1.0, np.abs(a_ref)))
+    assert np.all(np.abs(c - c_ref) <= 2e-6 * np.maximum(1.0, np.abs(c_ref)))
+    return lo_ref, hi_ref, a_ref, c_ref
+
+
+@pytest.mark.parametrize("act", [W.ACT_GELU_TANH, W.ACT_GELU_ERF])
+@pytest.mark.parametrize("shape", [(64, 1), (40, 2), (96, 257), (33, 1000), (16, 2048), (8, 8192)])
+def test_ranges_and_fits_match_oracle(shape, act):
+    h, n = shape
+    g = torch.Generator().manual_seed(100 * h + n)
+    z = (torch.randn(h, n, generator=g) * torch.linspace(0.3, 3.0, h)[:, None] + torch.linspace(-1, 1, h)[:, None]).cuda()
+    b1 = (0.1 * torch.randn(h, generator=g)).cuda()
+    _check(z, b1, 0.05, 0.95, act)
+    _check(z, None, 0.0, 1.0, act)
+    _check(z, None, 0.4, 0.4, act)                              # empty range: every neuron takes the tangent
+
+
+def test_padded_rows_ties_and_degenerate_neurons():
+    # leading dimension larger than n, many equal samples, constant neurons
+    g = torch.Generator().manual_seed(7)
+    buf = torch.randn(50, 700, generator=g).cuda()
+    buf[:10] = torch.round(buf[:10] * 2) / 2                   # ties
+    buf[10:13] = 0.25                                           # constant: zero variance in range
+    z = buf[:, :613]
+    assert z.stride(0) == 700
+    _check(z, None, 0.1, 0.9, W.ACT_GELU_TANH)
+
+
+def test_layer_calibration_through_the_gemm_entry():
+    # pre-activations of a bf16 layer from the library's own GEMM, then ranges and fits; the recipe of the synthetic
+    # workloads (float32 pre-activations from torch) gives the same statistics up to the accumulation order of z
+    cfg = W.LayerConfig("cal", 512, 2048, n_calib=1024)
+    L = W.make_layer(cfg, 3)
+    xcal = W.make_tokens(cfg, 1024, 3, tag="calib").cuda()
+    W1 = L.W1.cuda()
+    z = torch.empty(cfg.d_ff, 1024, dtype=torch.float32, device="cuda")
+    T.tardis_gemm_bf16(W1, xcal, z)
+    b1 = L.b1.cuda() if L.b1 is not None else None
+    lo, hi, a, c = _check(z, b1, 0.05, 0.95, cfg.act)
+    assert np.all(lo < hi)
+    z_ref = xcal.float() @ W1.float().t()
+    if b1 is not None:
+        z_ref = z_ref + b1[None, :]
+    q = torch.quantile(z_ref, torch.tensor([0.05, 0.95], device="cuda"), dim=0).cpu().numpy()
+    assert np.abs(lo - q[0]).max() < 1e-3 and np.abs(hi - q[1]).max() < 1e-3
+
+
+def test_argument_errors():
+    lib = T.load_library()
+    z = torch.zeros(4, 16, device="cuda")
+    o = [torch.zeros(4, device="cuda") for _ in range(4)]
+    def call(h, n, zp, ld, qlo, qhi, act):
+        return lib.tardis_calibrate(h, n, zp, ld, None, qlo, qhi, act, o[0].data_ptr(), o[1].data_ptr(), o[2].data_ptr(),
+                                    o[3].data_ptr(), None)
+    assert call(4, 16, z.data_ptr(), 16, 0.1, 0.9, 0) == T.TARDIS_OK
+    assert call(4, 16, None, 16, 0.1, 0.9, 0) == 1              # null samples
+    assert call(4, 16, z.data_ptr(), 8, 0.1, 0.9, 0) == 1       # leading dimension below n_cal
+    assert call(4, 16, z.data_ptr(), 16, 0.9, 0.1, 0) == 1      # q_lo > q_hi
+    assert call(4, 16, z.data_ptr(), 16, 0.1, 1.5, 0) == 1
+    assert call(4, 16, z.data_ptr(), 16, 0.1, 0.9, 7) == 1      # unknown activation
+    assert call(4, 9000, z.data_ptr(), 9000, 0.1, 0.9, 0) == 2  # more samples than the kernel sorts
+    torch.cuda.synchronize()
