@@ -387,7 +387,21 @@ def main():
         torch.cuda.synchronize()
         out["fold_ms_per_layer"] = ef0.elapsed_time(ef1)
         T.tardis_destroy(hf)
-        del Lf
+        # offline statistics of one layer: pre-activations of 2048 calibration tokens (tensor-core product), then the
+        # quantile ranges and least-squares fits of all neurons
+        ncal = 2048
+        xcal = W.make_tokens(cfg, ncal, rank * 1000 + 998, device=dev, tag="calib")
+        zcal = torch.empty(h, ncal, dtype=torch.float32, device=dev)
+
+        def calib_step():
+            T.tardis_gemm_bf16(Lf.W1, xcal, zcal)
+            T.tardis_calibrate(zcal, Lf.b1, cfg.q_lo, cfg.q_hi, cfg.act)
+
+        msc = timed(calib_step, 5, 3)
+        msk = timed(lambda: T.tardis_calibrate(zcal, Lf.b1, cfg.q_lo, cfg.q_hi, cfg.act), 5, 1)
+        out["calibrate_context"] = {"ms_per_layer": msc, "ms_ranges_and_fits": msk, "n_cal": ncal,
+                                    "what": "z = W1 Xcal^T (tcgen05 GEMM) + quantile ranges + least-squares fits, 16384 neurons"}
+        del Lf, xcal, zcal
 
         def dense_step():
             for i in range(NT // B):

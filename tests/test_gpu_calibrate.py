@@ -86,3 +86,31 @@ def test_argument_errors():
     assert call(4, 16, z.data_ptr(), 16, 0.1, 0.9, 7) == 1      # unknown activation
     assert call(4, 9000, z.data_ptr(), 9000, 0.1, 0.9, 0) == 2  # more samples than the kernel sorts
     torch.cuda.synchronize()
+
+
+def test_full_size_layer_sampled_neurons():
+    # the shape bench.py times (16384 neurons x 2048 calibration tokens, pre-activations from the library's GEMM):
+    # the GPU does every neuron, the oracle a seeded sample of them
+    cfg = W.CONFIGS["decode_7b"]
+    dev = torch.device("cuda", 0)
+    W1, _, b1, _ = W.make_weights(cfg, 0, device=dev)
+    xcal = W.make_tokens(cfg, 2048, 0, device=dev, tag="calib")
+    z = torch.empty(cfg.d_ff, 2048, dtype=torch.float32, device=dev)
+    T.tardis_gemm_bf16(W1, xcal, z)
+    lo, hi, a, c = T.tardis_calibrate(z, b1, 0.05, 0.95, cfg.act)
+    torch.cuda.synchronize()
+    rows = np.sort(np.random.default_rng(0).choice(cfg.d_ff, size=256, replace=False))
+    idx = torch.as_tensor(rows, device=dev)
+    zc = z[idx].cpu().numpy()
+    if b1 is not None:
+        zc = zc + b1[idx].cpu().numpy()[:, None]
+    lo_ref, hi_ref = O.quantile_ranges(zc, 0.05, 0.95)
+    a_ref, c_ref = O.least_squares_fit(zc, lo_ref, hi_ref, cfg.act)
+    assert np.array_equal(lo[idx].cpu().numpy(), lo_ref) and np.array_equal(hi[idx].cpu().numpy(), hi_ref)
+    assert np.all(np.abs(a[idx].cpu().numpy() - a_ref) <= 2e-6 * np.maximum(1.0, np.abs(a_ref)))
+    assert np.all(np.abs(c[idx].cpu().numpy() - c_ref) <= 2e-6 * np.maximum(1.0, np.abs(c_ref)))
+    # everywhere: a proper range, about 90 percent of the samples inside, a finite fit
+    zb = z + (b1[:, None] if b1 is not None else 0.0)
+    inside = ((zb >= lo[:, None]) & (zb < hi[:, None])).float().mean(1)
+    assert bool((lo < hi).all()) and float((inside - 0.9).abs().max()) < 2e-3
+    assert bool(torch.isfinite(a).all()) and bool(torch.isfinite(c).all())
