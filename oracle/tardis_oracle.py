@@ -35,6 +35,7 @@ import numpy as np
 
 ACT_GELU_TANH = 0
 ACT_GELU_ERF = 1
+ACT_RELU = 2
 
 _F64 = np.float64
 
@@ -47,9 +48,11 @@ def _as64(v):
 # activation
 # --------------------------------------------------------------------------
 def gelu(z, act=ACT_GELU_TANH):
-    """GELU in float64.  The paper only says "GELU" (Section 3.2); both common
-    forms are provided: tanh form 0.5 z (1 + tanh(sqrt(2/pi)(z + 0.044715 z^3)))
-    and the exact form z * Phi(z) with Phi the standard normal CDF."""
+    """The activation sigma in float64.  The paper only says "GELU" (Section
+    3.2); both common forms are provided: tanh form 0.5 z (1 + tanh(sqrt(2/pi)
+    (z + 0.044715 z^3))) and the exact form z * Phi(z) with Phi the standard
+    normal CDF.  ReLU, max(z, 0), is the activation of the OPT model in the
+    paper's evaluation (Section 7.1)."""
     z = np.asarray(z, dtype=_F64)
     if act == ACT_GELU_TANH:
         u = math.sqrt(2.0 / math.pi) * (z + 0.044715 * z * z * z)
@@ -57,6 +60,8 @@ def gelu(z, act=ACT_GELU_TANH):
     if act == ACT_GELU_ERF:
         from scipy.special import erf          # library primitive: the error function
         return 0.5 * z * (1.0 + erf(z / math.sqrt(2.0)))
+    if act == ACT_RELU:
+        return np.where(z > 0.0, z, 0.0 * z)              # 0 * z keeps NaN a NaN
     raise ValueError("unknown activation %r" % (act,))
 
 
@@ -279,7 +284,7 @@ def quantile_ranges(z, q_lo, q_hi):
 
 
 def gelu_derivative(z, act=ACT_GELU_TANH):
-    """d/dz GELU(z), analytic, float64."""
+    """d/dz sigma(z), analytic, float64 (ReLU: 1 for z > 0, else 0)."""
     z = np.asarray(z, dtype=_F64)
     if act == ACT_GELU_TANH:
         k = math.sqrt(2.0 / math.pi)
@@ -289,6 +294,8 @@ def gelu_derivative(z, act=ACT_GELU_TANH):
     if act == ACT_GELU_ERF:
         from scipy.special import erf
         return 0.5 * (1.0 + erf(z / math.sqrt(2.0))) + z * np.exp(-0.5 * z * z) / math.sqrt(2.0 * math.pi)
+    if act == ACT_RELU:
+        return np.where(z > 0.0, 1.0, 0.0)
     raise ValueError("unknown activation %r" % (act,))
 
 

@@ -135,6 +135,8 @@ def _loops_partially_linear(x, F, W1, W2, b1, b2, a, c, act):
             if F[t][j]:
                 u = math.sqrt(2.0 / math.pi) * (z + 0.044715 * z ** 3)
                 phi = 0.5 * z * (1.0 + math.tanh(u)) if act == O.ACT_GELU_TANH else z * Phi(z)
+                if act == O.ACT_RELU:
+                    phi = z if z > 0.0 else 0.0
             else:
                 phi = a[j] * z + c[j]
             for i in range(d):
@@ -161,7 +163,7 @@ def test_linear_activation_identity(bias):
     np.testing.assert_array_equal(O.fix(O.speculate(Wf, bf, x), x, none, W1, W2, a, c, b1), O.speculate(Wf, bf, x))
 
 
-@pytest.mark.parametrize("act", [O.ACT_GELU_TANH, O.ACT_GELU_ERF])
+@pytest.mark.parametrize("act", [O.ACT_GELU_TANH, O.ACT_GELU_ERF, O.ACT_RELU])
 def test_all_flagged_equals_dense_ffn(act):
     rng = np.random.default_rng(2)
     W1, W2, b1, b2, a, c, x = _random_problem(rng, 6, 13, 5)
@@ -324,7 +326,7 @@ def test_quantile_ranges_match_numpy_and_arithmetic_sequences():
     assert lo[0] == 3.0 and hi[0] == 3.0
 
 
-@pytest.mark.parametrize("act", [O.ACT_GELU_TANH, O.ACT_GELU_ERF])
+@pytest.mark.parametrize("act", [O.ACT_GELU_TANH, O.ACT_GELU_ERF, O.ACT_RELU])
 def test_least_squares_fit_normal_equations_polyfit_and_range_rule(act):
     rng = np.random.default_rng(6)
     z = (rng.standard_normal((5, 400)) * 1.3).astype(np.float32)
@@ -364,3 +366,20 @@ def test_least_squares_fit_degenerate_takes_the_tangent_at_the_midpoint(act):
     zz = np.linspace(20.0, 30.0, 50)[None, :]
     a, c = O.least_squares_fit(zz, np.array([0.0], np.float32), np.array([100.0], np.float32), act)
     assert abs(a[0] - 1.0) < 1e-6 and abs(c[0]) < 1e-5
+
+
+def test_relu_values_and_fit_special_cases():
+    z = np.array([-3.0, -0.0, 0.0, 1e-300, 2.5])
+    np.testing.assert_array_equal(O.gelu(z, O.ACT_RELU), np.array([0.0, 0.0, 0.0, 1e-300, 2.5]))
+    assert np.isnan(O.gelu(np.array([np.nan]), O.ACT_RELU))[0]
+    np.testing.assert_array_equal(O.gelu_derivative(np.array([-1.0, 0.0, 2.0]), O.ACT_RELU), np.array([0.0, 0.0, 1.0]))
+    # a range left of zero fits the zero function, one right of zero the identity: the linear function is then
+    # exact inside the range, which is why one function serves ReLU models at every ratio (Section 7.2)
+    rng = np.random.default_rng(9)
+    zz = rng.standard_normal((2, 300))
+    a, c = O.least_squares_fit(zz, np.array([-5.0, 0.0], np.float32), np.array([0.0, 5.0], np.float32), O.ACT_RELU)
+    assert a[0] == 0.0 and c[0] == 0.0 and abs(a[1] - 1.0) < 1e-7 and abs(c[1]) < 1e-7
+    # degenerate fallback: the tangent at the midpoint is 0 left of zero and the identity right of it
+    a, c = O.least_squares_fit(np.array([[9.0], [9.0]]), np.array([-2.0, 1.0], np.float32), np.array([-1.0, 2.0], np.float32),
+                               O.ACT_RELU)
+    assert (a[0], c[0], a[1], c[1]) == (0.0, 0.0, 1.0, 0.0)

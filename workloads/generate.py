@@ -42,6 +42,7 @@ import torch
 
 ACT_GELU_TANH = 0
 ACT_GELU_ERF = 1
+ACT_RELU = 2
 
 
 @dataclasses.dataclass(frozen=True)
@@ -156,6 +157,8 @@ def gelu_f64(z: torch.Tensor, act: int) -> torch.Tensor:
     z = z.double()
     if act == ACT_GELU_TANH:
         return torch.nn.functional.gelu(z, approximate="tanh")
+    if act == ACT_RELU:
+        return torch.relu(z)
     return torch.nn.functional.gelu(z)
 
 
