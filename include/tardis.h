@@ -46,7 +46,8 @@ typedef enum {
 } tardis_status_t;
 
 typedef enum { TARDIS_F32 = 0, TARDIS_BF16 = 1 } tardis_dtype_t;
-typedef enum { TARDIS_ACT_GELU_TANH = 0, TARDIS_ACT_GELU_ERF = 1 } tardis_act_t;
+/* TARDIS_ACT_RELU: max(z, 0), the activation of the OPT model in the paper's evaluation (Section 7.1). */
+typedef enum { TARDIS_ACT_GELU_TANH = 0, TARDIS_ACT_GELU_ERF = 1, TARDIS_ACT_RELU = 2 } tardis_act_t;
 
 /* Inputs of the offline fold.  Every array is read on `stream` during
  * tardis_fold and copied or transformed into handle-owned memory; once that

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libtardis.so")
 
 TARDIS_OK = 0
 TARDIS_F32, TARDIS_BF16 = 0, 1
-TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF = 0, 1
+TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_calibrate",

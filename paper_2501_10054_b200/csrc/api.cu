@@ -60,7 +60,7 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   const int d = desc->d_model, h = desc->d_ff, G = desc->pred_group;
   if (d <= 0 || h <= 0 || G <= 0) return TARDIS_ERR_INVALID_ARG;
   if (desc->dtype != TARDIS_F32 && desc->dtype != TARDIS_BF16) return TARDIS_ERR_INVALID_ARG;
-  if (desc->act != TARDIS_ACT_GELU_TANH && desc->act != TARDIS_ACT_GELU_ERF) return TARDIS_ERR_INVALID_ARG;
+  if (desc->act != TARDIS_ACT_GELU_TANH && desc->act != TARDIS_ACT_GELU_ERF && desc->act != TARDIS_ACT_RELU) return TARDIS_ERR_INVALID_ARG;
   if (desc->flags != 0) return TARDIS_ERR_INVALID_ARG;
   if (d % 8 || h % 32 || G % 16 || d % G) return TARDIS_ERR_INVALID_ARG;
   if (desc->pred_bits != 2) return desc->pred_bits > 0 && desc->pred_bits <= 8 ? TARDIS_ERR_UNSUPPORTED : TARDIS_ERR_INVALID_ARG;
@@ -181,7 +181,7 @@ tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, in
                                  double q_hi, int32_t act, float* lo, float* hi, float* a, float* c, tardis_stream_t stream) {
   if (d_ff <= 0 || n_cal <= 0 || !z || ldz < n_cal || !lo || !hi || !a || !c) return TARDIS_ERR_INVALID_ARG;
   if (!(q_lo >= 0.0 && q_lo <= q_hi && q_hi <= 1.0)) return TARDIS_ERR_INVALID_ARG;
-  if (act != TARDIS_ACT_GELU_TANH && act != TARDIS_ACT_GELU_ERF) return TARDIS_ERR_INVALID_ARG;
+  if (act != TARDIS_ACT_GELU_TANH && act != TARDIS_ACT_GELU_ERF && act != TARDIS_ACT_RELU) return TARDIS_ERR_INVALID_ARG;
   return launch_calibrate(d_ff, n_cal, z, ldz, b1, q_lo, q_hi, act, lo, hi, a, c, reinterpret_cast<cudaStream_t>(stream));
 }
 

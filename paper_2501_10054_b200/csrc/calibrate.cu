@@ -26,6 +26,7 @@ __device__ __forceinline__ double block_sum(double v, double* red) {     // ever
 }
 
 __device__ __forceinline__ double gelu_slope_f64(double z, int act) {
+  if (act == TARDIS_ACT_RELU) return z > 0.0 ? 1.0 : 0.0;
   if (act == TARDIS_ACT_GELU_TANH) {
     const double k = 0.7978845608028654;
     const double u = k * (z + 0.044715 * z * z * z), t = tanh(u);

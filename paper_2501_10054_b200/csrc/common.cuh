@@ -89,7 +89,9 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 tardis_status_t launch_calibrate(int h, int n, const float* z, long long ldz, const float* b1, double q_lo, double q_hi, int act,
                                  float* lo, float* hi, float* a, float* c, cudaStream_t s);
 
+// the activation (the name is historical: ReLU is served too)
 __device__ __forceinline__ float gelu_f32(float z, int act) {
+  if (act == TARDIS_ACT_RELU) return z > 0.f ? z : 0.f * z;      // 0 * z keeps NaN a NaN
   if (act == TARDIS_ACT_GELU_TANH) {
     float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
     return 0.5f * z * (1.0f + tanhf(u));
@@ -97,6 +99,7 @@ __device__ __forceinline__ float gelu_f32(float z, int act) {
   return 0.5f * z * (1.0f + erff(z * 0.7071067811865476f));
 }
 __device__ __forceinline__ double gelu_f64(double z, int act) {
+  if (act == TARDIS_ACT_RELU) return z > 0.0 ? z : 0.0 * z;
   if (act == TARDIS_ACT_GELU_TANH) {
     double u = 0.7978845608028654 * (z + 0.044715 * z * z * z);
     return 0.5 * z * (1.0 + tanh(u));

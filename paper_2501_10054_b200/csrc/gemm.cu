@@ -129,7 +129,7 @@ template <int BN> struct Cfg {
 // The epilogue of 32 consecutive columns n .. n + nv - 1 of output row m (one thread).
 // A&S 7.1.26 form of erf (absolute error below 2e-7, far inside the bf16 rounding of the correction it feeds)
 __device__ __forceinline__ float gelu_quick(float z, int act) {
-  if (act == TARDIS_ACT_GELU_TANH) return gelu_f32(z, act);
+  if (act != TARDIS_ACT_GELU_ERF) return gelu_f32(z, act);
   const float x = fabsf(z) * 0.7071067811865476f;
   const float t = __fdividef(1.f, fmaf(0.3275911f, x, 1.f));
   float poly = fmaf(1.061405429f, t, -1.453152027f);

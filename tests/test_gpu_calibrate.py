@@ -29,7 +29,7 @@ def _check(z, b1, q_lo, q_hi, act):
     return lo_ref, hi_ref, a_ref, c_ref
 
 
-@pytest.mark.parametrize("act", [W.ACT_GELU_TANH, W.ACT_GELU_ERF])
+@pytest.mark.parametrize("act", [W.ACT_GELU_TANH, W.ACT_GELU_ERF, W.ACT_RELU])
 @pytest.mark.parametrize("shape", [(64, 1), (40, 2), (96, 257), (33, 1000), (16, 2048), (8, 8192)])
 def test_ranges_and_fits_match_oracle(shape, act):
     h, n = shape
@@ -84,6 +84,7 @@ def test_argument_errors():
     assert call(4, 16, z.data_ptr(), 16, 0.9, 0.1, 0) == 1      # q_lo > q_hi
     assert call(4, 16, z.data_ptr(), 16, 0.1, 1.5, 0) == 1
     assert call(4, 16, z.data_ptr(), 16, 0.1, 0.9, 7) == 1      # unknown activation
+    assert call(4, 16, z.data_ptr(), 16, 0.1, 0.9, 2) == T.TARDIS_OK   # ReLU
     assert call(4, 9000, z.data_ptr(), 9000, 0.1, 0.9, 0) == 2  # more samples than the kernel sorts
     torch.cuda.synchronize()
 

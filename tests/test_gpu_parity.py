@@ -91,6 +91,15 @@ def test_batched_path_forced_for_calls_of_a_few_tokens():
     assert 0.02 < info["flag_frac"] < 0.5
 
 
+def test_relu_activation_on_every_path():
+    # ReLU layer (the OPT model of the paper's evaluation): per-token kernel, batched path, generic kernels, fp32
+    cfg = W.LayerConfig("relu", 512, 2048, dtype="bf16", act=W.ACT_RELU, n_calib=512)
+    _run(cfg, 30, [1, 5, 24], seed=2)
+    _run(cfg, 12, [2, 10], seed=2, path=1)
+    cfg = W.LayerConfig("relu32", 128, 512, dtype="f32", act=W.ACT_RELU, n_calib=512)
+    _run(cfg, 9, seed=4)
+
+
 def test_erf_activation_and_other_seed():
     cfg = W.LayerConfig("erf", 256, 1024, dtype="bf16", act=W.ACT_GELU_ERF, n_calib=512)
     _run(cfg, 17, [1, 16], seed=5)
