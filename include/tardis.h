@@ -200,8 +200,12 @@ tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, in
 
 /* Chooses the kernel path: 0 = automatic (default), 1 = always the generic
  * kernels, 3 = the batched tensor-core path for every token count (bf16
- * layers; other layers fall back to the generic kernels).  For testing one
- * path against the other. */
+ * layers; other layers fall back to the generic kernels), 4 = the generic
+ * kernels with the range check taken on the true pre-activations
+ * z = W1 x + b1 instead of the predictor's scores: the paper's third scenario
+ * of Section 7.7, which takes the predictor out of the result to show its
+ * effect (the debug capture then holds z).  For testing one path against the
+ * other. */
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
 
 /* Frees everything the handle owns (synchronises the device first). */

@@ -261,10 +261,10 @@ def rel_error(y, y_ref):
 # offline: per-neuron range and linear fit from calibration pre-activations
 # --------------------------------------------------------------------------
 def quantile_ranges(z, q_lo, q_hi):
-    """Range of every neuron as "the input range containing a certain portion
-    of activation inputs based on the profiled distribution" (Section 3.2,
-    Insight 2): the central portion between the q_lo and q_hi quantiles of the
-    neuron's calibration pre-activations.  z[h, N]: row j = the N samples of
+    """Range of every neuron: the interval that holds a chosen share of the
+    activation inputs profiled for it (Section 3.2, Insight 2), taken here as
+    the central portion between the q_lo and q_hi quantiles of the neuron's
+    calibration pre-activations.  z[h, N]: row j = the N samples of
     neuron j.  The quantile at level p is the linear interpolation between the
     order statistics around position p (N - 1).  (The greedy search of
     Algorithm 1 is a different way to pick the same kind of range; the
@@ -300,12 +300,13 @@ def gelu_derivative(z, act=ACT_GELU_TANH):
 
 
 def least_squares_fit(z, lo, hi, act=ACT_GELU_TANH):
-    """The linear function y = a z + c of every neuron, "obtained using least
-    squares regression" (Section 4.1 step 3, Section 5.1.2 step 4) of GELU(z)
-    on z over the calibration samples inside the neuron's range lo <= z < hi:
-        a = cov(z, GELU(z)) / var(z),   c = mean(GELU(z)) - a mean(z).
+    """The linear function y = a z + c of every neuron: the least-squares
+    regression (Section 4.1 step 3, Section 5.1.2 step 4) of the activation
+    sigma(z) on z over the calibration samples inside the neuron's range
+    lo <= z < hi:
+        a = cov(z, sigma(z)) / var(z),   c = mean(sigma(z)) - a mean(z).
     A neuron with fewer than two samples in range, or whose in-range samples
-    have variance below 1e-30, takes the tangent of GELU at the range midpoint.
+    have variance below 1e-30, takes the tangent of sigma at the range midpoint.
     z[h, N] float (samples as stored, i.e. float32 values), lo/hi[h] float32.
     Returns (a, c) as float32 arrays."""
     z = _as64(z)

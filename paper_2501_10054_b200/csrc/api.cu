@@ -222,7 +222,7 @@ tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf
 
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path) {
   Handle* H = check(handle);
-  if (!H || !(path == 0 || path == 1 || path == 3)) return TARDIS_ERR_INVALID_ARG;
+  if (!H || !(path == 0 || path == 1 || path == 3 || path == 4)) return TARDIS_ERR_INVALID_ARG;
   H->path_override = path;
   return TARDIS_OK;
 }

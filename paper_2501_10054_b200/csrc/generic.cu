@@ -55,6 +55,43 @@ __global__ void __launch_bounds__(1024) k_predictor_exact(
   }
 }
 
+// ---- range check on the true pre-activations ----------------------------------------------
+// The third scenario of the precision study (Section 7.7): the flag comes from z_j = W1[j,:] x + b1_j itself,
+// evaluated in fp64, instead of from the predictor, which shows what the predictor's mistakes cost.  Same layout
+// as the kernel above.
+template <typename T>
+__global__ void __launch_bounds__(1024) k_range_check_exact(
+    const T* __restrict__ W1, const float* __restrict__ b1, const float* __restrict__ lo, const float* __restrict__ hi,
+    const T* __restrict__ x, int n, int d, int h, uint32_t* __restrict__ bitmap, uint32_t* __restrict__ dbg_bitmap,
+    double* __restrict__ dbg_scores) {
+  __shared__ int flag_s[32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int j = blockIdx.x * 32 + warp;
+  const double lo_j = double(lo[j]), hi_j = double(hi[j]), b1_j = double(b1[j]);
+  for (int t = 0; t < n; ++t) {
+    const T* xt = x + size_t(t) * d;
+    double acc = 0.0;
+    for (int k = lane; k < d; k += 32) acc += double(to_f32(W1[size_t(j) * d + k])) * double(to_f32(xt[k]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    const double z = acc + b1_j;
+    const bool inside = (lo_j <= z) && (z < hi_j);
+    if (lane == 0) {
+      flag_s[warp] = inside ? 0 : 1;
+      if (dbg_scores) dbg_scores[size_t(t) * h + j] = z;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t word = __ballot_sync(0xffffffffu, flag_s[lane] != 0);
+      if (lane == 0) {
+        bitmap[size_t(t) * (h / 32) + blockIdx.x] = word;
+        if (dbg_bitmap) dbg_bitmap[size_t(t) * (h / 32) + blockIdx.x] = word;
+      }
+    }
+    __syncthreads();
+  }
+}
+
 // ---- flagged-count statistics ----------------------------------------------------------------
 __global__ void k_flag_stats(const uint32_t* __restrict__ bitmap, int words, unsigned long long* counters) {
   __shared__ unsigned int total;
@@ -185,8 +222,11 @@ static tardis_status_t generic_typed(Handle* H, const T* x, T* y, int64_t n_tota
     const T* xc = x + size_t(t0) * d;
     uint32_t* dbgb = H->dbg_bitmap ? H->dbg_bitmap + size_t(t0) * (h / 32) : nullptr;
     double* dbgs = H->dbg_scores ? H->dbg_scores + size_t(t0) * h : nullptr;
-    k_predictor_exact<T><<<h / 32, 1024, 0, s>>>(H->codes, static_cast<const T*>(H->scale), H->zero, H->b1, H->lo, H->hi,
-                                                 xc, n, d, h, H->G, H->bitmap, dbgb, dbgs);
+    if (H->path_override == 4)
+      k_range_check_exact<T><<<h / 32, 1024, 0, s>>>(static_cast<const T*>(H->W1), H->b1, H->lo, H->hi, xc, n, d, h, H->bitmap, dbgb, dbgs);
+    else
+      k_predictor_exact<T><<<h / 32, 1024, 0, s>>>(H->codes, static_cast<const T*>(H->scale), H->zero, H->b1, H->lo, H->hi,
+                                                   xc, n, d, h, H->G, H->bitmap, dbgb, dbgs);
     k_flag_stats<<<n, 256, 0, s>>>(H->bitmap, h / 32, H->counters);
     const size_t cnt = size_t(n) * d;
     k_init_yacc<<<unsigned((cnt + 255) / 256), 256, 0, s>>>(H->yacc, H->bf, n, d);

@@ -100,6 +100,32 @@ def test_relu_activation_on_every_path():
     _run(cfg, 9, seed=4)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_exact_range_mode_flags_from_true_preactivations(dtype):
+    # path 4: the range check runs on z = W1 x + b1 itself (the paper's ablation that takes the predictor out)
+    cfg = W.LayerConfig("hybrid_" + dtype, 256, 1024, dtype=dtype, n_calib=512)
+    L = _layer(cfg, 1)
+    s = L.numpy64()
+    x = W.make_tokens(cfg, 11, 1).cuda()
+    h = T.fold_layer(L)
+    try:
+        T.tardis_set_path(h, 4)
+        y, F, S = Hp.gpu_forward(h, L, x, [1, 10])
+        x64 = x.double().cpu().numpy()
+        z = x64 @ s["W1"].T + s["b1"][None, :]
+        F_ref = O.flags_from_score(z, s["lo"], s["hi"])
+        band = O.near_threshold(z, s["lo"], s["hi"], Hp.BAND)
+        assert not ((F != F_ref) & ~band).any()
+        assert np.abs(S - z).max() < 1e-9                       # the captured score is the pre-activation
+        y_ref = O.direct_partially_linear(x64, np.where(band, F, F_ref), s["W1"], s["W2"], s["a"], s["c"], s["b1"], s["b2"], s["act"])
+        assert np.nanmax(O.rel_error(y.double().cpu().numpy(), y_ref)) <= Hp.TOL[dtype]
+        # the predictor's flags differ from these on some neurons (that difference is what the mode measures)
+        zhat = O.predictor_score(x64, s["codes"], s["scale"], s["zero"], s["group"], s["b1"], s["bits"])
+        assert (O.flags_from_score(zhat, s["lo"], s["hi"]) != F_ref).any()
+    finally:
+        T.tardis_destroy(h)
+
+
 def test_erf_activation_and_other_seed():
     cfg = W.LayerConfig("erf", 256, 1024, dtype="bf16", act=W.ACT_GELU_ERF, n_calib=512)
     _run(cfg, 17, [1, 16], seed=5)
