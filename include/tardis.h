@@ -65,10 +65,13 @@ typedef struct {
   const float* hi;            /* device [d_ff]                                            */
   const float* a;             /* device [d_ff]; linear fit a*z + c on the range           */
   const float* c;             /* device [d_ff]                                            */
-  int32_t pred_bits;          /* 2                                                        */
+  int32_t pred_bits;          /* bits per predictor code: 2 (the paper's setting, Section 6;
+                                 every path), 4 (batched and generic paths) or 8 (generic
+                                 kernels only); the paper sweeps this size in Section 7.6  */
   int32_t pred_group;         /* G: channels per quantisation group; multiple of 16       */
-  const uint32_t* pred_codes; /* device [d_ff, d_model*pred_bits/32]; channel k of row j in
-                                 word k/16, bits 2*(k%16) .. 2*(k%16)+1                   */
+  const uint32_t* pred_codes; /* device [d_ff, d_model*pred_bits/32]; with p = 32/pred_bits
+                                 codes per word, channel k of row j sits in word k/p, bits
+                                 pred_bits*(k%p) upwards                                  */
   const void* pred_scale;     /* device [d_ff, d_model/G], type `dtype`                   */
   const uint8_t* pred_zero;   /* device [d_ff, d_model/G], integer zero-point 0..3        */
   uint32_t flags;             /* reserved, 0                                              */

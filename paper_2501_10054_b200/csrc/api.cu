@@ -63,7 +63,8 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   if (desc->act != TARDIS_ACT_GELU_TANH && desc->act != TARDIS_ACT_GELU_ERF && desc->act != TARDIS_ACT_RELU) return TARDIS_ERR_INVALID_ARG;
   if (desc->flags != 0) return TARDIS_ERR_INVALID_ARG;
   if (d % 8 || h % 32 || G % 16 || d % G) return TARDIS_ERR_INVALID_ARG;
-  if (desc->pred_bits != 2) return desc->pred_bits > 0 && desc->pred_bits <= 8 ? TARDIS_ERR_UNSUPPORTED : TARDIS_ERR_INVALID_ARG;
+  if (desc->pred_bits != 2 && desc->pred_bits != 4 && desc->pred_bits != 8)
+    return desc->pred_bits > 0 && desc->pred_bits <= 8 ? TARDIS_ERR_UNSUPPORTED : TARDIS_ERR_INVALID_ARG;
   const void* required[] = {desc->W1, desc->W2, desc->lo, desc->hi, desc->a, desc->c,
                             desc->pred_codes, desc->pred_scale, desc->pred_zero};
   for (const void* p : required)
@@ -77,6 +78,7 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   memset(H, 0, sizeof(*H));
   H->magic = kMagic;
   H->d = d; H->h = h; H->dtype = desc->dtype; H->act = desc->act; H->G = G; H->ngroups = d / G;
+  H->bits = desc->pred_bits;
   H->esize = desc->dtype == TARDIS_F32 ? 4 : 2;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   H->last_stream = s;
@@ -96,7 +98,7 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   A(&H->a, size_t(h), &H->bytes_tables);
   A(&H->c, size_t(h), &H->bytes_tables);
   A(&H->b1, size_t(h), &H->bytes_tables);
-  A(&H->codes, hd / 16, &H->bytes_predictor);
+  A(&H->codes, hd * H->bits / 32, &H->bytes_predictor);
   A(reinterpret_cast<char**>(&H->scale), size_t(h) * H->ngroups * H->esize, &H->bytes_predictor);
   A(&H->zero, size_t(h) * H->ngroups, &H->bytes_predictor);
   A(&H->yacc, size_t(kGenericChunk) * d, &H->bytes_scratch);
@@ -130,7 +132,8 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   H->last_stream = s;
   tardis_status_t st;
   const bool fused = H->path_override == 0 && H->codes_mma != nullptr && n_tokens <= kDecodeMaxTokens;
-  const bool batched = ((H->path_override == 0 && !fused) || H->path_override == 3) && H->bstate != nullptr;
+  // (8-bit codes times a bf16 scale do not fit the exact two-term bf16 form the batched scores rely on)
+  const bool batched = ((H->path_override == 0 && !fused) || H->path_override == 3) && H->bstate != nullptr && H->bits <= 4;
   if (fused) {
     st = launch_decode_forward(H, x, y, int(n_tokens), s);
     H->last_path = 2;

@@ -3,9 +3,9 @@
 //
 // For a chunk of up to kChunk tokens X[n, d]:
 //   1. fast predictor scores  Zhat = X What^T + b1, What = s (q - zp) (Section 5.3).  What needs 10 significant
-//      bits, so it is held as an exact sum of two bf16 matrices (hi + lo); one GEMM runs over both and its
+//      bits (13 with 4-bit codes), so it is held as an exact sum of two bf16 matrices (hi + lo); one GEMM runs over both and its
 //      epilogue turns the scores into flag words (they are stored only for the debug capture).  Products
-//      are exact, the fp32 accumulation is not: a score within tau(t, j) = kEps * 3 max_g s[j,g] * |x_t|_1 of a
+//      are exact, the fp32 accumulation is not: a score within tau(t, j) = kEps * (2^bits - 1) max_g s[j,g] * |x_t|_1 of a
 //      range end is queued by the epilogue and re-evaluated in fp64 from the packed codes (k_recheck), so the
 //      flags are the exact ones;
 //   2. speculative product    Yacc = X W_f^T + b_f                               (fp32);
@@ -41,19 +41,20 @@ struct State {
 // What = s (q - zp) split exactly into hi = bf16(What) and lo = What - hi (at most 2 significant bits left).
 __global__ void k_dequant_split(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
                                 const uint8_t* __restrict__ zero, __nv_bfloat16* __restrict__ hi,
-                                __nv_bfloat16* __restrict__ lo, float* __restrict__ smaxrow, int d, int G) {
-  const int j = blockIdx.x, ng = d / G, nwords = d / 16;
+                                __nv_bfloat16* __restrict__ lo, float* __restrict__ smaxrow, int d, int G, int bits) {
+  const int per = 32 / bits;                    // codes per word
+  const uint32_t cmask = (1u << bits) - 1u;
+  const int j = blockIdx.x, ng = d / G, nwords = d / per;
   for (int w = threadIdx.x; w < nwords; w += blockDim.x) {
     const uint32_t word = codes[size_t(j) * nwords + w];
-    const int g = (w * 16) / G;
+    const int g = (w * per) / G;
     const float s = __bfloat162float(scale[size_t(j) * ng + g]);
     const float zp = float(zero[size_t(j) * ng + g]);
-#pragma unroll
-    for (int q = 0; q < 16; ++q) {
-      const float v = s * (float((word >> (2 * q)) & 3u) - zp);     // exact: 8-bit significand times |int| <= 3
+    for (int q = 0; q < per; ++q) {
+      const float v = s * (float((word >> (bits * q)) & cmask) - zp);   // exact: 8-bit significand times |int| <= 15
       const __nv_bfloat16 h = __float2bfloat16_rn(v);
-      hi[size_t(j) * d + w * 16 + q] = h;
-      lo[size_t(j) * d + w * 16 + q] = __float2bfloat16_rn(v - __bfloat162float(h));
+      hi[size_t(j) * d + w * per + q] = h;
+      lo[size_t(j) * d + w * per + q] = __float2bfloat16_rn(v - __bfloat162float(h));
     }
   }
   if (threadIdx.x == 0) {
@@ -91,7 +92,7 @@ __global__ void k_xnorm(const __nv_bfloat16* __restrict__ x, int d, float* __res
 __global__ void k_recheck(const uint2* __restrict__ rlist, const unsigned int* __restrict__ rcount,
                           const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
                           const uint8_t* __restrict__ zero, const float* __restrict__ b1, const float* __restrict__ lo,
-                          const float* __restrict__ hi, const __nv_bfloat16* __restrict__ x, int d, int h, int G,
+                          const float* __restrict__ hi, const __nv_bfloat16* __restrict__ x, int d, int h, int G, int bits,
                           uint32_t* __restrict__ bitmap, float* __restrict__ zhat, unsigned long long* counters) {
   const int lane = threadIdx.x & 31;
   const unsigned int total = min(rcount[0], (unsigned int)kMaxRecheck);
@@ -99,7 +100,7 @@ __global__ void k_recheck(const uint2* __restrict__ rlist, const unsigned int* _
   for (unsigned int e = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; e < total; e += nwarps) {
     const uint2 pr = rlist[e];
     const int t = int(pr.x), j = int(pr.y);
-    const double z = exact_score(codes, scale, zero, x + size_t(t) * d, j, d, G, lane) + double(b1[j]);
+    const double z = exact_score(codes, scale, zero, x + size_t(t) * d, j, d, G, bits, lane) + double(b1[j]);
     if (lane == 0) {
       const bool inside = (double(lo[j]) <= z) && (z < double(hi[j]));
       uint32_t* wp = bitmap + size_t(t) * (h / 32) + (j >> 5);
@@ -272,8 +273,9 @@ tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaSt
   // W_f[i][k] row-major (the GEMMs want the channel index contiguous in both operands): transpose of C
   k_transpose_b<__nv_bfloat16><<<dim3((d + 31) / 32, (d + 31) / 32), tb, 0, s>>>(static_cast<const __nv_bfloat16*>(H->C), S->Wf, d, d);
   TARDIS_CUDA_TRY(cudaMemcpyAsync(S->W2, desc->W2, hd * 2, cudaMemcpyDeviceToDevice, s));
-  k_dequant_split<<<h, 256, 0, s>>>(H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, S->What_hi, S->What_lo,
-                                    S->smaxrow, d, H->G);
+  if (H->bits <= 4)   // (8-bit codes: the batched path is not used, see the dispatch)
+    k_dequant_split<<<h, 256, 0, s>>>(H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, S->What_hi, S->What_lo,
+                                    S->smaxrow, d, H->G, H->bits);
   TARDIS_CUDA_TRY(cudaGetLastError());
   return TARDIS_OK;
 }
@@ -308,13 +310,13 @@ tardis_status_t launch_batched_forward(Handle* H, const void* xv, void* yv, int6
     const bool keep_scores = H->dbg_bitmap || H->dbg_scores;
     g.epilogue = GEMM_EPI_FLAGS; g.out_f32 = keep_scores ? S->zhat : nullptr; g.ldo = h; g.bias = H->b1;
     g.error_word = &H->counters[CTR_ERROR];
-    g.lo = H->lo; g.hi = H->hi; g.colscale = S->smaxrow; g.rowscale = S->x1; g.keps = kEps * 3.f;
+    g.lo = H->lo; g.hi = H->hi; g.colscale = S->smaxrow; g.rowscale = S->x1; g.keps = kEps * float((1 << H->bits) - 1);
     g.bitmap_out = S->bitmap; g.rlist = S->rlist; g.rcount = S->rcount; g.rcap = kMaxRecheck;
-    g.codes = H->codes; g.scale = H->scale; g.zero = H->zero; g.xsrc = xc; g.d = d; g.G = H->G;
+    g.codes = H->codes; g.scale = H->scale; g.zero = H->zero; g.xsrc = xc; g.d = d; g.G = H->G; g.bits = H->bits;
     tardis_status_t st = launch_gemm(g, s);
     if (st != TARDIS_OK) return st;
     k_recheck<<<H->num_sms * 4, 256, 0, s>>>(S->rlist, S->rcount, H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, H->b1,
-                                             H->lo, H->hi, xc, d, h, H->G, S->bitmap, keep_scores ? S->zhat : nullptr, H->counters);
+                                             H->lo, H->hi, xc, d, h, H->G, H->bits, S->bitmap, keep_scores ? S->zhat : nullptr, H->counters);
     k_flag_counts<<<n, 256, 0, s>>>(S->bitmap, h / 32, H->counters);
     if (H->dbg_bitmap || H->dbg_scores) {
       const size_t cnt = size_t(n) * h;

@@ -19,6 +19,7 @@ enum { CTR_FLAGGED_TOTAL = 0, CTR_FLAGGED_MAX = 1, CTR_ERROR = 2, CTR_RECHECKS =
 struct Handle {
   uint64_t magic;
   int d, h, dtype, act, G, ngroups;
+  int bits;              // bits per predictor code (2, 4 or 8)
   size_t esize;
   int device;
   // state (device)

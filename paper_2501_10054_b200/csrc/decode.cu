@@ -893,7 +893,7 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   H->dscratch = nullptr;
   H->codes_mma = nullptr;
   const int d = H->d, h = H->h, G = H->G;
-  if (H->dtype != TARDIS_BF16) return TARDIS_OK;
+  if (H->dtype != TARDIS_BF16 || H->bits != 2) return TARDIS_OK;   // (the integer tensor-core predictor is built for 2-bit codes)
   if (!(G == 64 || G == 128)) return TARDIS_OK;                     // generic kernels serve other group sizes
   const int NT = h / 16;
   const int nvec = d / 8;

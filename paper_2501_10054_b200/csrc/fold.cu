@@ -132,7 +132,7 @@ tardis_status_t launch_fold(Handle* H, const tardis_fold_desc_t* desc, cudaStrea
   TARDIS_CUDA_TRY(cudaMemcpyAsync(H->c, desc->c, h * 4, D2D, s));
   if (desc->b1) TARDIS_CUDA_TRY(cudaMemcpyAsync(H->b1, desc->b1, h * 4, D2D, s));
   else TARDIS_CUDA_TRY(cudaMemsetAsync(H->b1, 0, h * 4, s));
-  TARDIS_CUDA_TRY(cudaMemcpyAsync(H->codes, desc->pred_codes, h * d / 4, D2D, s));
+  TARDIS_CUDA_TRY(cudaMemcpyAsync(H->codes, desc->pred_codes, h * d / 8 * H->bits, D2D, s));
   TARDIS_CUDA_TRY(cudaMemcpyAsync(H->scale, desc->pred_scale, h * ng * H->esize, D2D, s));
   TARDIS_CUDA_TRY(cudaMemcpyAsync(H->zero, desc->pred_zero, h * ng, D2D, s));
   TARDIS_CUDA_TRY(cudaMemsetAsync(H->counters, 0, CTR_COUNT * sizeof(unsigned long long), s));

@@ -116,7 +116,7 @@ struct KParams {
   uint32_t* bitmap_out;
   uint2* rlist; unsigned int* rcount; int rcap;
   const uint32_t* codes; const __nv_bfloat16* scale; const uint8_t* zero;
-  const __nv_bfloat16* xsrc; int d, G;
+  const __nv_bfloat16* xsrc; int d, G, bits;
 };
 
 template <int BN> struct Cfg {
@@ -160,7 +160,7 @@ __device__ __forceinline__ void epilogue_chunk(const KParams& p, float (&v)[32],
             const unsigned int slot = atomicAdd(&p.rcount[0], 1u);
             if (slot < (unsigned int)p.rcap) p.rlist[slot] = make_uint2((unsigned int)m, (unsigned int)(n + i));
             else {                                           // queue full: settle this one here (slow, but exact)
-              const double ze = exact_score_single(p.codes, p.scale, p.zero, p.xsrc + size_t(m) * p.d, n + i, p.d, p.G) + double(p.bias[n + i]);
+              const double ze = exact_score_single(p.codes, p.scale, p.zero, p.xsrc + size_t(m) * p.d, n + i, p.d, p.G, p.bits) + double(p.bias[n + i]);
               flag = !((double(l) <= ze) && (ze < double(u)));
               atomicAdd(&p.rcount[1], 1u);
             }
@@ -448,7 +448,7 @@ static tardis_status_t launch_bn(const GemmArgs& g, cudaStream_t s) {
   p.bias = g.bias; p.addend = g.addend; p.a = g.a; p.c = g.c; p.bitmap = g.bitmap; p.error_word = g.error_word;
   p.lo = g.lo; p.hi = g.hi; p.colscale = g.colscale; p.rowscale = g.rowscale; p.keps = g.keps; p.bitmap_out = g.bitmap_out;
   p.rlist = g.rlist; p.rcount = g.rcount; p.rcap = g.rcap; p.codes = g.codes; p.scale = static_cast<const __nv_bfloat16*>(g.scale);
-  p.zero = g.zero; p.xsrc = static_cast<const __nv_bfloat16*>(g.xsrc); p.d = g.d; p.G = g.G;
+  p.zero = g.zero; p.xsrc = static_cast<const __nv_bfloat16*>(g.xsrc); p.d = g.d; p.G = g.G; p.bits = g.bits;
   TARDIS_CUDA_TRY(cudaFuncSetAttribute(k_gemm<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM));
   const int nm = (g.M + BM - 1) / BM, nn = (g.N + BN - 1) / BN;
   p.fast_m = nm <= nn ? 1 : 0;

@@ -41,7 +41,7 @@ struct GemmArgs {
   uint32_t* bitmap_out;             // [M, N / 32]
   uint2* rlist; unsigned int* rcount; int rcap;   // queue of (m, n) pairs, its fill count ([1]: pairs settled in place), capacity
   const uint32_t* codes; const void* scale; const uint8_t* zero;   // the packed predictor (rows n)
-  const void* xsrc; int d, G;       // the bf16 rows A1 came from (leading dimension d), group size
+  const void* xsrc; int d, G, bits; // the bf16 rows A1 came from (leading dimension d), group size, bits per code
 };
 
 // Enqueues the GEMM on `s`.  Returns UNSUPPORTED when the tensor-map entry point of the driver is not

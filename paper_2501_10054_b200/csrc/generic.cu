@@ -13,25 +13,26 @@ template <typename T>
 __global__ void __launch_bounds__(1024) k_predictor_exact(
     const uint32_t* __restrict__ codes, const T* __restrict__ scale, const uint8_t* __restrict__ zero,
     const float* __restrict__ b1, const float* __restrict__ lo, const float* __restrict__ hi,
-    const T* __restrict__ x, int n, int d, int h, int G, uint32_t* __restrict__ bitmap,
+    const T* __restrict__ x, int n, int d, int h, int G, int bits, uint32_t* __restrict__ bitmap,
     uint32_t* __restrict__ dbg_bitmap, double* __restrict__ dbg_scores) {
   __shared__ int flag_s[32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j = blockIdx.x * 32 + warp;
-  const int nwords = d / 16, ng = d / G;
+  const int per = 32 / bits;                    // codes per word
+  const uint32_t cmask = (1u << bits) - 1u;
+  const int nwords = d / per, ng = d / G;
   const double lo_j = double(lo[j]), hi_j = double(hi[j]), b1_j = double(b1[j]);
   for (int t = 0; t < n; ++t) {
     const T* xt = x + size_t(t) * d;
     double acc = 0.0;
     for (int w = lane; w < nwords; w += 32) {
       const uint32_t word = codes[size_t(j) * nwords + w];
-      const int g = (w * 16) / G;
+      const int g = (w * per) / G;
       const double zp = double(zero[size_t(j) * ng + g]);
       double inner = 0.0;
-#pragma unroll
-      for (int p = 0; p < 16; ++p) {
-        const double q = double((word >> (2 * p)) & 3u);
-        inner += (q - zp) * double(to_f32(xt[w * 16 + p]));
+      for (int p = 0; p < per; ++p) {
+        const double q = double((word >> (bits * p)) & cmask);
+        inner += (q - zp) * double(to_f32(xt[w * per + p]));
       }
       acc += double(to_f32(scale[size_t(j) * ng + g])) * inner;
     }
@@ -226,7 +227,7 @@ static tardis_status_t generic_typed(Handle* H, const T* x, T* y, int64_t n_tota
       k_range_check_exact<T><<<h / 32, 1024, 0, s>>>(static_cast<const T*>(H->W1), H->b1, H->lo, H->hi, xc, n, d, h, H->bitmap, dbgb, dbgs);
     else
       k_predictor_exact<T><<<h / 32, 1024, 0, s>>>(H->codes, static_cast<const T*>(H->scale), H->zero, H->b1, H->lo, H->hi,
-                                                   xc, n, d, h, H->G, H->bitmap, dbgb, dbgs);
+                                                   xc, n, d, h, H->G, H->bits, H->bitmap, dbgb, dbgs);
     k_flag_stats<<<n, 256, 0, s>>>(H->bitmap, h / 32, H->counters);
     const size_t cnt = size_t(n) * d;
     k_init_yacc<<<unsigned((cnt + 255) / 256), 256, 0, s>>>(H->yacc, H->bf, n, d);
@@ -271,7 +272,7 @@ template <typename T, typename Acc>
 static tardis_status_t static_typed(Handle* H, const T* x, T* y, int n, float* yacc, uint32_t* bitmap, cudaStream_t s) {
   const int d = H->d, h = H->h;
   k_predictor_exact<T><<<h / 32, 1024, 0, s>>>(H->codes, static_cast<const T*>(H->scale), H->zero, H->b1, H->lo, H->hi,
-                                               x, n, d, h, H->G, bitmap, H->dbg_bitmap, H->dbg_scores);
+                                               x, n, d, h, H->G, H->bits, bitmap, H->dbg_bitmap, H->dbg_scores);
   k_flag_stats<<<n, 256, 0, s>>>(bitmap, h / 32, H->counters);
   const size_t cnt = size_t(n) * d;
   k_init_yacc<<<unsigned((cnt + 255) / 256), 256, 0, s>>>(yacc, H->bf, n, d);

@@ -64,7 +64,7 @@ def test_invalid_arguments_return_status_before_any_launch(lib):
     assert status(act=5) == 1
     assert status(W1=None) == 1
     assert status(W1=24) == 1                 # misaligned
-    assert status(pred_bits=4) == 2           # valid but not built
+    assert status(pred_bits=3) == 2           # valid but not built (2, 4 and 8 are)
     assert status(pred_bits=0) == 1
     assert status(flags=1) == 1
     assert out.value is None
