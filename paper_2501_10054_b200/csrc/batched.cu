@@ -3,11 +3,11 @@
 //
 // For a chunk of up to kChunk tokens X[n, d]:
 //   1. fast predictor scores  Zhat = X What^T + b1, What = s (q - zp) (Section 5.3).  What needs 10 significant
-//      bits (13 with 4-bit codes), so it is held as an exact sum of two bf16 matrices (hi + lo); one GEMM runs over both and its
-//      epilogue turns the scores into flag words (they are stored only for the debug capture).  Products
-//      are exact, the fp32 accumulation is not: a score within tau(t, j) = kEps * (2^bits - 1) max_g s[j,g] * |x_t|_1 of a
-//      range end is queued by the epilogue and re-evaluated in fp64 from the packed codes (k_recheck), so the
-//      flags are the exact ones;
+//      bits (13 with 4-bit codes), so it is held as an exact sum of two bf16 matrices (hi + lo); one GEMM runs
+//      over both and its epilogue turns the scores into flag words (they are stored only for the debug
+//      capture).  Products are exact, the fp32 accumulation is not: a score within
+//      tau(t, j) = kEps * (2^bits - 1) max_g s[j,g] * |x_t|_1 of a range end is queued by the epilogue and
+//      re-evaluated in fp64 from the packed codes (k_recheck), so the flags are the exact ones;
 //   2. speculative product    Yacc = X W_f^T + b_f                               (fp32);
 //   3. result fixing          Delta = flag .* (GELU(Z) - a Z - c), Z = X W1^T + b1   (GEMM with that epilogue, bf16),
 //                             y = bf16(Yacc + Delta W2^T)                            (GEMM over all neurons:
@@ -22,14 +22,17 @@
 namespace tardis {
 namespace bat {
 
-constexpr int kChunk = 1024;                 // tokens per pass (scratch is sized for this)
+// Tokens per pass (the scratch is sized for this).  With 2048 the big products have 16 x 64 tiles = 6.9 waves of
+// 148 CTAs; 1024-token chunks lost 15 % of the time to their last, partial wave.
+constexpr int kChunk = 2048;
+constexpr int kChunkCapture = 1024;          // ... while the debug capture is on (the score buffer holds that many)
 constexpr float kEps = 7.62939453125e-6f;    // 2^-17: relative accumulation-error allowance of the fast scores
 constexpr int kMaxRecheck = 1 << 21;         // (token, neuron) pairs per chunk that can queue for re-evaluation
 
 struct State {
   __nv_bfloat16 *Wf, *W2, *What_hi, *What_lo;     // [d,d], [d,h], [h,d], [h,d]
   float* smaxrow;                                  // [h] largest group scale of a neuron
-  float *zhat, *yacc, *x1;                         // [kChunk,h], [kChunk,d], [kChunk]
+  float *zhat, *yacc, *x1;                         // [kChunkCapture,h] (scores for the capture; fold temporary), [kChunk,d], [kChunk]
   __nv_bfloat16* delta;                            // [kChunk,h]
   uint32_t* bitmap;                                // [kChunk,h/32]
   uint2* rlist;                                    // [kMaxRecheck] (token, neuron)
@@ -183,7 +186,7 @@ tardis_status_t batched_prepare(Handle* H) {
       {reinterpret_cast<void**>(&S->Wf), size_t(d) * d * 2, false}, {reinterpret_cast<void**>(&S->W2), hd * 2, false},
       {reinterpret_cast<void**>(&S->What_hi), hd * 2, false},       {reinterpret_cast<void**>(&S->What_lo), hd * 2, false},
       {reinterpret_cast<void**>(&S->smaxrow), size_t(h) * 4, false},
-      {reinterpret_cast<void**>(&S->zhat), size_t(kChunk) * h * 4, true}, {reinterpret_cast<void**>(&S->yacc), size_t(kChunk) * d * 4, true},
+      {reinterpret_cast<void**>(&S->zhat), size_t(kChunkCapture) * h * 4, true}, {reinterpret_cast<void**>(&S->yacc), size_t(kChunk) * d * 4, true},
       {reinterpret_cast<void**>(&S->x1), size_t(kChunk) * 4, true},       {reinterpret_cast<void**>(&S->delta), size_t(kChunk) * h * 2, true},
       {reinterpret_cast<void**>(&S->bitmap), size_t(kChunk) * (h / 32) * 4, true},
       {reinterpret_cast<void**>(&S->rlist), size_t(kMaxRecheck) * 8, true}, {reinterpret_cast<void**>(&S->rcount), 16, true}};
@@ -245,7 +248,7 @@ tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cu
   dim3 tb(32, 8);
   k_scale_transpose_split<<<dim3((d + 31) / 32, (h + 31) / 32), tb, 0, s>>>(static_cast<const __nv_bfloat16*>(H->W1), H->a,
                                                                             S->What_hi, S->What_lo, h, d);
-  const size_t cap = size_t(kChunk) * h;                     // floats in the score buffer
+  const size_t cap = size_t(kChunkCapture) * h;              // floats in the score buffer
   int rows_per = int(cap / d);
   rows_per = rows_per / 128 * 128;
   if (rows_per < 128) return TARDIS_ERR_UNSUPPORTED;
@@ -296,8 +299,10 @@ tardis_status_t launch_batched_forward(Handle* H, const void* xv, void* yv, int6
   const int d = H->d, h = H->h;
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(xv);
   __nv_bfloat16* y = static_cast<__nv_bfloat16*>(yv);
-  for (int64_t t0 = 0; t0 < n_total; t0 += kChunk) {
-    const int n = int(n_total - t0 < kChunk ? n_total - t0 : kChunk);
+  const bool keep_scores = H->dbg_bitmap || H->dbg_scores;
+  const int chunk = keep_scores ? kChunkCapture : kChunk;
+  for (int64_t t0 = 0; t0 < n_total; t0 += chunk) {
+    const int n = int(n_total - t0 < chunk ? n_total - t0 : chunk);
     const __nv_bfloat16* xc = x + size_t(t0) * d;
     TARDIS_CUDA_TRY(cudaMemsetAsync(S->rcount, 0, 16, s));
     k_xnorm<<<n, 256, 0, s>>>(xc, d, S->x1);
@@ -307,7 +312,6 @@ tardis_status_t launch_batched_forward(Handle* H, const void* xv, void* yv, int6
     g.A1 = xc; g.lda1 = d; g.B1 = S->What_hi; g.ldb1 = d; g.A2 = xc; g.lda2 = d; g.B2 = S->What_lo; g.ldb2 = d;
     // its epilogue turns the scores into flag words and queues the pairs too close to a range end; the scores
     // themselves are stored only for the debug capture
-    const bool keep_scores = H->dbg_bitmap || H->dbg_scores;
     g.epilogue = GEMM_EPI_FLAGS; g.out_f32 = keep_scores ? S->zhat : nullptr; g.ldo = h; g.bias = H->b1;
     g.error_word = &H->counters[CTR_ERROR];
     g.lo = H->lo; g.hi = H->hi; g.colscale = S->smaxrow; g.rowscale = S->x1; g.keps = kEps * float((1 << H->bits) - 1);

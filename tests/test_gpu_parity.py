@@ -206,8 +206,9 @@ def test_run_to_run_flags_identical():
 
 
 def test_batched_path_chunk_boundary_nan_token_and_empty_ranges():
-    """More tokens than one scratch chunk (1024) in a single call, a token holding a NaN in the middle of it,
-    and the result compared token by token with the oracle on a seeded sample."""
+    """More tokens than one scratch chunk in a single call (chunks hold 1024 tokens while the debug capture is on,
+    2048 otherwise), a token holding a NaN in the middle of it, and the result compared token by token with the
+    oracle on a seeded sample."""
     cfg = W.LayerConfig("chunks", 256, 1024, n_calib=512)
     L = _layer(cfg)
     s = L.numpy64()
@@ -225,5 +226,14 @@ def test_batched_path_chunk_boundary_nan_token_and_empty_ranges():
                          score_tol=3e-4, label="chunks")
         st = T.tardis_stats(h)
         assert st["flagged_total"] == int(F.sum()) and st["device_error"] == 0
+        # without the capture the chunks are twice as long: 2055 tokens cross that boundary too, and every token
+        # must come out as it does in the captured run (same products, same order of accumulation)
+        x2 = torch.cat([x, x[:1025]])
+        y2 = torch.empty_like(x2)
+        T.tardis_ffn_forward(h, x2, y2)
+        torch.cuda.synchronize()
+        ref2 = torch.cat([y, y[:1025]])
+        ok = (y2 == ref2) | (torch.isnan(y2) & torch.isnan(ref2))
+        assert bool(ok.all())
     finally:
         T.tardis_destroy(h)
