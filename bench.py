@@ -9,7 +9,8 @@ d_ff = 16384, bf16, about 10 % of the neurons flagged per token - run as batch-1
 "step" is 512 successive tokens, each one call of tardis_ffn_forward (predictor, flagging, folded
 product, result fixing).  Calls rotate over `--layers` independently seeded layers so that the
 state a call touches (about 80 MB) has left the 126 MB L2 by the time its layer comes round again.
-Prints ONE JSON line; see the design doc for the meaning of every key.
+Prints ONE JSON line (metric, value, roofline, cpu_baseline, e2e, clocks and context legs; the keys are
+described where they are filled in below).
 """
 from __future__ import annotations
 

@@ -38,7 +38,7 @@ typedef void* tardis_stream_t;                      /* a cudaStream_t (0 = defau
 typedef enum {
   TARDIS_OK = 0,
   TARDIS_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, negative size, bad enum */
-  TARDIS_ERR_UNSUPPORTED = 2,   /* valid request this build has no kernel for (see tardis_fold) */
+  TARDIS_ERR_UNSUPPORTED = 2,   /* valid request the library has no kernel for (see tardis_fold) */
   TARDIS_ERR_ALLOC = 3,         /* device allocation failed */
   TARDIS_ERR_CUDA = 4,          /* a CUDA call failed; text via tardis_last_error */
   TARDIS_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out */
