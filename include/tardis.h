@@ -211,6 +211,17 @@ tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, in
  * other. */
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
 
+/* Profiling aid of the fused decode kernel (the online path of Section 5.4 as one launch).  A library
+ * built with -DTARDIS_PHASE_STAMPS (python -m paper_2501_10054_b200.build --stamps) makes every CTA of that
+ * kernel record the GPU's global nanosecond timer at its phase boundaries; this call synchronises the
+ * device and copies the table of the most recent launch to `stamps`, HOST memory of max_ctas x 16 int64:
+ * per CTA, slot 0 kernel entry, 1 x loaded, 2 fixed-point x ready, 3 predictor done (first predictor
+ * warp), 4 folded product done (first streaming warp), 5 flagged list complete, 6 result fixing done,
+ * 7 CTA counted as finished, 8 y written (last CTA only, else 0), 9 the CTA's number of flagged neurons
+ * (a count, not a time); CTAs beyond the grid stay 0.  The ordinary build returns TARDIS_ERR_UNSUPPORTED
+ * and its kernel carries no stamps.  Errors: INVALID_ARG (NULL, max_ctas <= 0), UNSUPPORTED, CUDA. */
+tardis_status_t tardis_debug_phase_stamps(long long* stamps, int32_t max_ctas);
+
 /* Frees everything the handle owns (synchronises the device first). */
 tardis_status_t tardis_destroy(tardis_handle_t handle);
 

@@ -22,7 +22,7 @@ TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_calibrate",
-           "tardis_status_string", "tardis_last_error"]
+           "tardis_debug_phase_stamps", "tardis_status_string", "tardis_last_error"]
 
 
 class TardisError(RuntimeError):
@@ -75,7 +75,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_destroy.argtypes = [vp]
     lib.tardis_gemm_bf16.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, i32, vp]
     lib.tardis_calibrate.argtypes = [i32, i32, vp, i64, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp]
-    for name in EXPORTS[:10]:
+    lib.tardis_debug_phase_stamps.argtypes = [vp, i32]
+    for name in EXPORTS[:11]:
         getattr(lib, name).restype = ctypes.c_int
     lib.tardis_status_string.argtypes = [ctypes.c_int]
     lib.tardis_status_string.restype = ctypes.c_char_p
@@ -189,6 +190,15 @@ def tardis_export_folded(handle: int, Wf: Optional[torch.Tensor], bf: Optional[t
 
 def tardis_set_path(handle: int, path: int):
     _check(load_library().tardis_set_path(handle, path), "tardis_set_path")
+
+
+def tardis_debug_phase_stamps(max_ctas: int = 512):
+    """Phase stamps of the most recent fused decode launch as a numpy int64 array [max_ctas, 16] (needs a
+    library built with TARDIS_PHASE_STAMPS; the ordinary build raises UNSUPPORTED)."""
+    import numpy as np
+    buf = np.zeros((max_ctas, 16), dtype=np.int64)
+    _check(load_library().tardis_debug_phase_stamps(buf.ctypes.data, max_ctas), "tardis_debug_phase_stamps")
+    return buf
 
 
 def tardis_destroy(handle: int):

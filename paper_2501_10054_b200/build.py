@@ -10,6 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtardis.so")
+LIB_STAMPS = os.path.join(PKG, "libtardis_stamps.so")
 SOURCES = ["api.cu", "fold.cu", "generic.cu", "decode.cu", "gemm.cu", "batched.cu", "calibrate.cu"]
 
 
@@ -28,12 +29,15 @@ def needs_build() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, stamps: bool = False) -> str:
+    """Builds the library.  stamps=True builds libtardis_stamps.so instead: the same sources with
+    -DTARDIS_PHASE_STAMPS (the fused decode kernel records its phase boundaries; profiling only)."""
+    out = LIB_STAMPS if stamps else LIB
+    if not force and not stamps and not needs_build():
         return LIB
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+           "-o", out] + (["-DTARDIS_PHASE_STAMPS"] if stamps else []) + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -42,8 +46,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed:\n" + r.stdout + r.stderr)
     if verbose:
         print(r.stderr)
-    return LIB
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, stamps="--stamps" in sys.argv))

@@ -223,6 +223,11 @@ tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf
   return launch_export_folded(H, Wf, bf, s);
 }
 
+tardis_status_t tardis_debug_phase_stamps(long long* stamps, int32_t max_ctas) {
+  if (!stamps || max_ctas <= 0) return TARDIS_ERR_INVALID_ARG;
+  return decode_read_stamps(stamps, max_ctas);
+}
+
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path) {
   Handle* H = check(handle);
   if (!H || !(path == 0 || path == 1 || path == 3 || path == 4)) return TARDIS_ERR_INVALID_ARG;

@@ -72,6 +72,7 @@ tardis_status_t launch_static_forward(Handle* H, const void* x, void* y, int64_t
 tardis_status_t decode_prepare(Handle* H, cudaStream_t s);                 // builds codes_mma, pmeta, scratch
 tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
 void decode_release(Handle* H);
+tardis_status_t decode_read_stamps(long long* out, int max_ctas);   // UNSUPPORTED unless built with TARDIS_PHASE_STAMPS
 tardis_status_t batched_prepare(Handle* H);                                                   // bf16 only: allocations
 tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);    // fills the batched state
 tardis_status_t launch_batched_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);

@@ -36,9 +36,11 @@
 #include <vector>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace tardis {
 namespace dec {
+using namespace ptx;
 
 constexpr int NW = 16;            // warps per CTA
 constexpr int NWP = 8;            // of them, warps that evaluate the predictor while the others stream the folded matrix
@@ -52,7 +54,6 @@ constexpr int MAXGROUPS = 8;      // slot groups (one barrier each) of the resul
 constexpr int kBadRow = 0x40000000;   // row whose group scales do not fit the integer form: always re-evaluated
 constexpr int NREP = 4;           // replicas of the output accumulator
 constexpr int XVR = 2;            // 8-channel vectors of x per thread (padded d <= 8192)
-constexpr uint32_t SPIN_LIMIT = 1u << 21;   // spaced polls of a bounded mbarrier wait: a fraction of a second
 // control words (unsigned int) in global scratch; all zero between calls
 constexpr int CTL_TICKET = 0;     // [32] stride 32: next output tile of a channel chunk of the folded matrix
 constexpr int CTL_DONE = 1024;    // CTAs that have added all their contributions
@@ -88,83 +89,6 @@ struct Scratch {           // handle-owned device memory of the fused path
   Params base; size_t smem_bytes; size_t bytes; int grid; int vpt; const void* kernel;
 };
 
-// ---- small wrappers ---------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint64_t* b, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-               : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: false when the limit ran out (the caller records the error and goes on without the
-// data).  Polls are spaced out so that waiting warps leave the issue slots to the working ones.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity) {
-  if (mbar_test(b, parity)) return true;
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
-    __nanosleep(64);
-    if (mbar_test(b, parity)) return true;
-  }
-  return false;
-}
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {   // read-only, no L1 allocation
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-__device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// The same with a zero accumulator going in: MMAs of one warp that do not depend on each other pipeline
-// four times better than a chain through one accumulator, so each MMA of a group starts its own sum.
-__device__ __forceinline__ void mma_u8s8_z(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                           uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-               : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void red_add_f32(float* addr, float v) {
-  asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-__device__ __forceinline__ void unpack8(float (&f)[8], const uint4& w) {
-  f[0] = bf_lo(w.x); f[1] = bf_hi(w.x); f[2] = bf_lo(w.y); f[3] = bf_hi(w.y);
-  f[4] = bf_lo(w.z); f[5] = bf_hi(w.z); f[6] = bf_lo(w.w); f[7] = bf_hi(w.w);
-}
-__device__ __forceinline__ void fma8(float (&acc)[8], float s, const uint4& w) {
-  acc[0] += s * bf_lo(w.x); acc[1] += s * bf_hi(w.x);
-  acc[2] += s * bf_lo(w.y); acc[3] += s * bf_hi(w.y);
-  acc[4] += s * bf_lo(w.z); acc[5] += s * bf_hi(w.z);
-  acc[6] += s * bf_lo(w.w); acc[7] += s * bf_hi(w.w);
-}
-__device__ __forceinline__ float dot8(const uint4& w, const float (&xv)[8]) {
-  return bf_lo(w.x) * xv[0] + bf_hi(w.x) * xv[1] + bf_lo(w.y) * xv[2] + bf_hi(w.y) * xv[3] +
-         bf_lo(w.z) * xv[4] + bf_hi(w.z) * xv[5] + bf_lo(w.w) * xv[6] + bf_hi(w.w) * xv[7];
-}
-
 // ---- shared-memory carve-up (host and device agree through this) -----------------------------------
 struct SmemLayout {
   size_t pbuf_bytes, pbuf, xq, zeros, xh, sxi, zpart, wpart, score, tab, fl_j, fl_delta, rc, flagbits, wred, bars, misc, total;
@@ -195,6 +119,22 @@ struct SmemLayout {
 };
 enum { MS_NFL = 0, MS_NRC = 1, MS_ERR = 2, MS_LAST = 3, MS_WCNT = 8, MS_BUFCNT = 32 };
 
+
+// ---- phase stamps (compiled in with -DTARDIS_PHASE_STAMPS only) -----------------------------------------
+// Thread 0 of every CTA (and lane 0 of the first streaming warp) writes the global timer at the phase
+// boundaries of the last launch; tardis_debug_phase_stamps copies the table to the host.
+constexpr int kStampCtas = 512, kStampSlots = 16;
+enum { ST_START = 0, ST_X = 1, ST_LIMBS = 2, ST_PRED = 3, ST_STREAM = 4, ST_FLAGS = 5, ST_FIXED = 6, ST_COUNTED = 7,
+       ST_FINAL = 8, ST_NFL = 9 };
+#ifdef TARDIS_PHASE_STAMPS
+__device__ long long g_stamps[kStampCtas * kStampSlots];
+__device__ __forceinline__ long long global_timer() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define TARDIS_STAMP(cond, slot) do { if ((cond) && blockIdx.x < kStampCtas) g_stamps[blockIdx.x * kStampSlots + (slot)] = global_timer(); } while (0)
+#define TARDIS_STAMP_VALUE(cond, slot, v) do { if ((cond) && blockIdx.x < kStampCtas) g_stamps[blockIdx.x * kStampSlots + (slot)] = (long long)(v); } while (0)
+#else
+#define TARDIS_STAMP(cond, slot) do { } while (0)
+#define TARDIS_STAMP_VALUE(cond, slot, v) do { } while (0)
+#endif
 
 // ---- the kernel ---------------------------------------------------------------------------------------
 template <int VPT, int G>
@@ -235,6 +175,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     bulk_g2s(pbuf + size_t(b) * p.unit_bytes, p.pblocks + (size_t(plan.x + tl) * p.nkc + size_t(r) * p.cpr) * p.pbs, bytes, &full[b]);
   };
 
+  TARDIS_STAMP(tid == 0, ST_START);
   // Programmatic dependent launch: the next launch in the stream may start its own prologue (everything
   // up to its griddepcontrol.wait reads only the layer's constant state) while this one is still running.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -296,6 +237,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     if (lane == 0) { wred[warp] = amax; wred[NW + warp] = any_nf ? 1.f : 0.f; }
   }
   __syncthreads();
+  TARDIS_STAMP(tid == 0, ST_X);
   float amax_all = 0.f;
   bool tok_nonfinite = false;
 #pragma unroll
@@ -447,9 +389,11 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   // The limbs are complete once all 16 warps have passed here.  Warps 8..15 only announce their part
   // (bar.arrive) and go on to the speculative folded product, which needs nothing but x; warps 0..7 wait for
   // everybody's limbs (bar.sync) and evaluate the predictor.  Both meet again at the barrier after it.
+  TARDIS_STAMP(tid == 0, ST_LIMBS);
   if (warp >= NWP) {
     asm volatile("bar.arrive 1, %0;" ::"n"(NTH) : "memory");
     stream_c(warp - NWP, NW - NWP);
+    TARDIS_STAMP(tid == NWP * 32, ST_STREAM);
   } else {
     asm volatile("bar.sync 1, %0;" ::"n"(NTH) : "memory");
   }
@@ -545,6 +489,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       if (++r == p.nranges) { r = 0; ++tl; }
     }
   }
+  TARDIS_STAMP(tid == 0, ST_PRED);
   __syncthreads();
   // tolerance of the fast score: every rounding residual (<= 1/2 unit of 2^E) times |code - zero| <= 3 times the scale
   double tau;
@@ -648,6 +593,8 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
   __syncthreads();
   const int nfl = misc[MS_NFL];
 
+  TARDIS_STAMP(tid == 0, ST_FLAGS);
+  TARDIS_STAMP_VALUE(tid == 0, ST_NFL, nfl);
   // ---- result fixing ----
   // The predictor buffers are free now and take the rows the fixing needs, one bulk copy per row: item i < nfl
   // is the W1 row of the i-th flagged neuron, item nfl + i its W2T row.  The row slots form a ring of groups
@@ -749,12 +696,14 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
     }
   }
 
+  TARDIS_STAMP(tid == 0, ST_FIXED);
   // Any warp of any CTA may have added to any column, so the columns are complete when the last CTA is:
   // the CTAs count themselves, and the last one turns the accumulator into y.
   __threadfence();
   __syncthreads();
   if (tid == 0) misc[MS_LAST] = int(atomicAdd(&p.ctl[CTL_DONE], 1u));
   __syncthreads();
+  TARDIS_STAMP(tid == 0, ST_COUNTED);
   if (misc[MS_LAST] == int(gridDim.x) - 1) {
     __threadfence();
     for (int vec = tid; vec < p.nvec; vec += NTH) {
@@ -784,6 +733,7 @@ __global__ void __launch_bounds__(NTH, 2) k_decode(const Params p) {
       o[3] = __floats2bfloat162_rn(s1.z, s1.w);
       *reinterpret_cast<uint4*>(p.y + c0) = *reinterpret_cast<const uint4*>(o);
     }
+    TARDIS_STAMP(tid == 0, ST_FINAL);
     if (lane == 0) {
       for (int kc = warp; kc < p.nkc; kc += NW) p.ctl[CTL_TICKET + kc * 32] = 0u;
       if (warp == 0) {   // every CTA has arrived, so every CTA's flagged count is in
@@ -1019,6 +969,18 @@ tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, 
     H->launches += 1;
   }
   return TARDIS_OK;
+}
+
+tardis_status_t decode_read_stamps(long long* out, int max_ctas) {
+#ifdef TARDIS_PHASE_STAMPS
+  const int n = max_ctas < kStampCtas ? max_ctas : kStampCtas;
+  TARDIS_CUDA_TRY(cudaDeviceSynchronize());
+  TARDIS_CUDA_TRY(cudaMemcpyFromSymbol(out, g_stamps, sizeof(long long) * size_t(n) * kStampSlots));
+  return TARDIS_OK;
+#else
+  (void)out; (void)max_ctas;
+  return TARDIS_ERR_UNSUPPORTED;
+#endif
 }
 
 void decode_release(Handle* H) {
