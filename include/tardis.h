@@ -97,6 +97,8 @@ typedef struct {
   uint64_t device_error;        /* sticky device-side error word, 0 = none                 */
   uint64_t exact_rechecks;      /* predictor scores re-evaluated by the exact slow path    */
   uint64_t launches;            /* kernels launched by tardis_ffn_forward so far           */
+  uint64_t last_union;          /* neurons flagged by at least one token of the most recent
+                                   launch of the fused decode kernel (the rows it fetched)   */
 } tardis_stats_t;
 
 /* Offline part (Section 5.2 constant folding, Section 5.3 predictor set-up).

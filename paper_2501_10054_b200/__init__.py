@@ -45,7 +45,7 @@ class Stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint64) for n in
                 ("calls", "tokens", "flagged_total", "flagged_max", "last_path", "bytes_folded",
                  "bytes_predictor", "bytes_tables", "bytes_w1", "bytes_w2t", "bytes_scratch",
-                 "device_error", "exact_rechecks", "launches")]
+                 "device_error", "exact_rechecks", "launches", "last_union")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}

@@ -38,6 +38,7 @@ static tardis_status_t dev_alloc(T** p, size_t count, size_t* tally) {
 }
 
 static void free_all(Handle* H) {
+  fused_release(H);
   decode_release(H);
   batched_release(H);
   void* ptrs[] = {H->W1, H->W2T, H->C, H->bf, H->lo, H->hi, H->a, H->c, H->b1, H->codes, H->scale,
@@ -114,7 +115,8 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
     st = launch_fold_tensor(H, desc, s);
     if (st == TARDIS_ERR_UNSUPPORTED) st = launch_fold_product(H, s);   // no tensor-map support: plain kernel
   }
-  if (st == TARDIS_OK && bf16) st = decode_prepare(H, s);
+  if (st == TARDIS_OK && bf16) st = fused_prepare(H, s);
+  if (st == TARDIS_OK && bf16 && !H->fscratch) st = decode_prepare(H, s);   // wider layers: the older per-token kernel
   if (st == TARDIS_OK && bf16) st = batched_finish(H, desc, s);
   if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
   *out = reinterpret_cast<tardis_handle_t>(H);
@@ -131,11 +133,11 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   H->last_stream = s;
   tardis_status_t st;
-  const bool fused = H->path_override == 0 && H->codes_mma != nullptr && n_tokens <= kDecodeMaxTokens;
+  const bool fused = H->path_override == 0 && (H->fscratch != nullptr || H->codes_mma != nullptr) && n_tokens <= kDecodeMaxTokens;
   // (8-bit codes times a bf16 scale do not fit the exact two-term bf16 form the batched scores rely on)
   const bool batched = ((H->path_override == 0 && !fused) || H->path_override == 3) && H->bstate != nullptr && H->bits <= 4;
   if (fused) {
-    st = launch_decode_forward(H, x, y, int(n_tokens), s);
+    st = H->fscratch ? launch_fused_forward(H, x, y, int(n_tokens), s) : launch_decode_forward(H, x, y, int(n_tokens), s);
     H->last_path = 2;
   } else if (batched) {
     st = launch_batched_forward(H, x, y, n_tokens, s);
@@ -197,7 +199,7 @@ tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
   memset(out, 0, sizeof(*out));
   out->calls = H->calls; out->tokens = H->tokens; out->last_path = H->last_path;
   out->flagged_total = ctr[CTR_FLAGGED_TOTAL]; out->flagged_max = ctr[CTR_FLAGGED_MAX];
-  out->device_error = ctr[CTR_ERROR]; out->exact_rechecks = ctr[CTR_RECHECKS];
+  out->device_error = ctr[CTR_ERROR]; out->exact_rechecks = ctr[CTR_RECHECKS]; out->last_union = ctr[CTR_LAST_UNION];
   out->bytes_folded = H->bytes_folded; out->bytes_predictor = H->bytes_predictor;
   out->bytes_tables = H->bytes_tables; out->bytes_w1 = H->bytes_w1; out->bytes_w2t = H->bytes_w2t;
   out->bytes_scratch = H->bytes_scratch;
@@ -225,7 +227,8 @@ tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf
 
 tardis_status_t tardis_debug_phase_stamps(long long* stamps, int32_t max_ctas) {
   if (!stamps || max_ctas <= 0) return TARDIS_ERR_INVALID_ARG;
-  return decode_read_stamps(stamps, max_ctas);
+  // the table of the kernel that ran last is the one with the later entry stamps; both are cheap to read
+  return fused_read_stamps(stamps, max_ctas);
 }
 
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path) {

@@ -10,11 +10,11 @@ namespace tardis {
 
 constexpr uint64_t kMagic = 0x7A2D15F01DULL;
 constexpr int kGenericChunk = 256;   // tokens per pass of the generic kernels (scratch is sized for this)
-constexpr int kDecodeMaxTokens = 8;  // largest batch the fused decode kernel takes
+constexpr int kDecodeMaxTokens = 8;  // largest batch the fused decode kernels take (the newer one 4 tokens per launch)
 constexpr int kStaticMaxTokens = 64; // largest batch of the forward that keeps its scratch in the library image
 
 // device counter slots
-enum { CTR_FLAGGED_TOTAL = 0, CTR_FLAGGED_MAX = 1, CTR_ERROR = 2, CTR_RECHECKS = 3, CTR_TICKET = 4, CTR_COUNT = 8 };
+enum { CTR_FLAGGED_TOTAL = 0, CTR_FLAGGED_MAX = 1, CTR_ERROR = 2, CTR_RECHECKS = 3, CTR_TICKET = 4, CTR_LAST_UNION = 5, CTR_COUNT = 8 };
 
 struct Handle {
   uint64_t magic;
@@ -38,6 +38,7 @@ struct Handle {
   float* yacc;           // [kGenericChunk, d] fp32 accumulator
   uint32_t* bitmap;      // [kGenericChunk, h/32]
   unsigned long long* counters;  // [CTR_COUNT]
+  void* fscratch;        // fused decode state for calls of 1..4 tokens per launch (see fused.cu); null when not built
   void* dscratch;        // fused decode scratch (see decode.cu)
   size_t dscratch_bytes;
   void* bstate;          // batched / prefill state and scratch (see batched.cu); null when not built
@@ -72,7 +73,11 @@ tardis_status_t launch_static_forward(Handle* H, const void* x, void* y, int64_t
 tardis_status_t decode_prepare(Handle* H, cudaStream_t s);                 // builds codes_mma, pmeta, scratch
 tardis_status_t launch_decode_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
 void decode_release(Handle* H);
-tardis_status_t decode_read_stamps(long long* out, int max_ctas);   // UNSUPPORTED unless built with TARDIS_PHASE_STAMPS
+tardis_status_t decode_read_stamps(long long* out, int max_ctas);
+tardis_status_t fused_prepare(Handle* H, cudaStream_t s);                  // builds the state of fused.cu (bf16, d_model <= 4608)
+tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
+void fused_release(Handle* H);
+tardis_status_t fused_read_stamps(long long* out, int max_ctas);   // UNSUPPORTED unless built with TARDIS_PHASE_STAMPS
 tardis_status_t batched_prepare(Handle* H);                                                   // bf16 only: allocations
 tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);    // fills the batched state
 tardis_status_t launch_batched_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);

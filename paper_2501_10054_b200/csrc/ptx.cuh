@@ -7,8 +7,6 @@
 namespace tardis {
 namespace ptx {
 
-constexpr uint32_t SPIN_LIMIT = 1u << 21;   // spaced polls of a bounded mbarrier wait: a fraction of a second
-
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
@@ -23,14 +21,26 @@ __device__ __forceinline__ bool mbar_test(uint64_t* b, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false when the limit ran out (the caller records the error and goes on without the
-// data).  Polls are spaced out so that waiting warps leave the issue slots to the working ones.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity) {
+// data).  mbarrier.try_wait suspends the thread by itself until the phase completes or a short hardware time-out
+// passes, so the loop needs no sleep of its own; the limit is in SM clock cycles (a fraction of a second).
+constexpr long long WAIT_LIMIT_CYCLES = 400000000ll;
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, long long limit = WAIT_LIMIT_CYCLES) {
   if (mbar_test(b, parity)) return true;
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
-    __nanosleep(64);
-    if (mbar_test(b, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_test(b, parity)) return true;
+    if (clock64() - t0 > limit) return false;
   }
-  return false;
+}
+// The same for a whole warp (all 32 lanes must call it): lane 0 polls, the others learn the outcome through a shuffle,
+// which also orders their later reads of the copied data after lane 0's observation of the barrier.  (Every lane
+// polling the same barrier word serialises: with 32 warps waiting that costs more than the wait itself.)
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* b, uint32_t parity, long long limit = WAIT_LIMIT_CYCLES) {
+  int ok = 0;
+  if ((threadIdx.x & 31) == 0) ok = mbar_wait(b, parity, limit) ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -58,7 +68,7 @@ __device__ __forceinline__ void mma_u8s8_z(int (&c)[4], uint32_t a0, uint32_t a1
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }

@@ -39,7 +39,7 @@ def test_status_strings(lib):
 def test_struct_layout_matches_header():
     # 4 int32, 8 pointers, 2 int32, 3 pointers, uint32 (+ padding)
     assert ctypes.sizeof(T.FoldDesc) == 16 + 64 + 8 + 24 + 8
-    assert ctypes.sizeof(T.Stats) == 14 * 8
+    assert ctypes.sizeof(T.Stats) == 15 * 8
 
 
 def test_invalid_arguments_return_status_before_any_launch(lib):
