@@ -133,7 +133,8 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   H->last_stream = s;
   tardis_status_t st;
-  const bool fused = H->path_override == 0 && (H->fscratch != nullptr || H->codes_mma != nullptr) && n_tokens <= kDecodeMaxTokens;
+  const bool has_fused = H->fscratch != nullptr || H->codes_mma != nullptr;
+  const bool fused = has_fused && ((H->path_override == 0 && n_tokens <= (H->fscratch ? kDecodeMaxTokens : 8)) || (H->path_override == 2 && n_tokens <= 4096));
   // (8-bit codes times a bf16 scale do not fit the exact two-term bf16 form the batched scores rely on)
   const bool batched = ((H->path_override == 0 && !fused) || H->path_override == 3) && H->bstate != nullptr && H->bits <= 4;
   if (fused) {
@@ -233,7 +234,7 @@ tardis_status_t tardis_debug_phase_stamps(long long* stamps, int32_t max_ctas) {
 
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path) {
   Handle* H = check(handle);
-  if (!H || !(path == 0 || path == 1 || path == 3 || path == 4)) return TARDIS_ERR_INVALID_ARG;
+  if (!H || !(path >= 0 && path <= 4)) return TARDIS_ERR_INVALID_ARG;
   H->path_override = path;
   return TARDIS_OK;
 }

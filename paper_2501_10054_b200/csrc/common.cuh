@@ -10,7 +10,7 @@ namespace tardis {
 
 constexpr uint64_t kMagic = 0x7A2D15F01DULL;
 constexpr int kGenericChunk = 256;   // tokens per pass of the generic kernels (scratch is sized for this)
-constexpr int kDecodeMaxTokens = 8;  // largest batch the fused decode kernels take (the newer one 4 tokens per launch)
+constexpr int kDecodeMaxTokens = 12; // largest batch the fused decode kernels take (the newer one 4 tokens per launch)
 constexpr int kStaticMaxTokens = 64; // largest batch of the forward that keeps its scratch in the library image
 
 // device counter slots
