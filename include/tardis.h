@@ -73,7 +73,7 @@ typedef struct {
                                  codes per word, channel k of row j sits in word k/p, bits
                                  pred_bits*(k%p) upwards                                  */
   const void* pred_scale;     /* device [d_ff, d_model/G], type `dtype`                   */
-  const uint8_t* pred_zero;   /* device [d_ff, d_model/G], integer zero-point 0..3        */
+  const uint8_t* pred_zero;   /* device [d_ff, d_model/G], integer zero-point 0..2^pred_bits-1 */
   uint32_t flags;             /* reserved, 0                                              */
 } tardis_fold_desc_t;
 
@@ -82,12 +82,13 @@ typedef struct {
  * original weights kept for fixing (here: all of W1 and W2^T, any neuron can
  * be flagged), per-neuron tables, scratch. */
 typedef struct {
-  uint64_t calls;               /* tardis_ffn_forward calls that launched work             */
+  uint64_t calls;               /* tardis_ffn_forward / tardis_ffn_forward_static calls that launched work */
   uint64_t tokens;              /* tokens processed                                        */
   uint64_t flagged_total;       /* sum over tokens of flagged neurons                      */
   uint64_t flagged_max;         /* largest flagged count of a single token                 */
-  uint64_t last_path;           /* 0 none, 1 generic, 2 fused decode, 3 batched/prefill,
-                                   4 generic kernels on the library's built-in scratch     */
+  uint64_t last_path;           /* 0 none, 1 generic kernels, 2 fused decode kernel, 3 batched/prefill,
+                                   5 generic kernels on the library's built-in scratch
+                                   (tardis_ffn_forward_static)                              */
   uint64_t bytes_folded;        /* W_f and b_f                                             */
   uint64_t bytes_predictor;     /* codes + scales + zero-points as stored                  */
   uint64_t bytes_tables;        /* lo, hi, a, c, b1                                        */
@@ -108,7 +109,8 @@ typedef struct {
  * allocations; *out is valid on return with TARDIS_OK.
  * Errors: INVALID_ARG (NULL desc/out/required array, pointer not 16-byte
  * aligned, d_model % 8, d_model % pred_group, pred_group % 16, d_ff % 32,
- * non-positive sizes, unknown enum), UNSUPPORTED (pred_bits != 2), ALLOC, CUDA. */
+ * non-positive sizes, unknown enum, pred_bits outside 1..8), UNSUPPORTED (pred_bits of 1, 3, 5, 6 or 7), ALLOC, CUDA.
+ * Forward calls on the handle must be ordered after `stream` (same stream, or an event): the fold is asynchronous. */
 tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stream,
                             tardis_handle_t* out);
 
@@ -125,7 +127,7 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
  * Calls on one handle must be stream-ordered with respect to each other (they
  * share the handle's scratch).
  * Errors: INVALID_ARG (NULL/destroyed handle, NULL or misaligned x/y,
- * n_tokens < 0), CUDA. */
+ * n_tokens < 0, the handle's device is not the current device), CUDA. */
 tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* y,
                                    int64_t n_tokens, tardis_stream_t stream);
 
@@ -139,12 +141,15 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
  * library image (every GPU that loads the library holds those 4 MiB until the process exits).  It
  * calls no cudaMalloc, cudaFree or other allocating routine.
  * Same arguments, result and error behaviour as tardis_ffn_forward, computed by the generic
- * kernels, with these differences:
+ * kernels (the exact-range mode of tardis_set_path(handle, 4) is honoured; the other path choices do
+ * not apply), with these differences:
  *   - n_tokens <= 64 and n_tokens * (4 * d_model + d_ff / 8) <= 4 MiB (each of the two terms rounded
  *     up to 256 bytes), else TARDIS_ERR_UNSUPPORTED with the reason in tardis_last_error; the
  *     handle's device must be the current device, else TARDIS_ERR_INVALID_ARG;
  *   - the first call on a device asks the runtime for the array's device address
- *     (cudaGetSymbolAddress) and keeps it; make that first call before any stream capture starts;
+ *     (cudaGetSymbolAddress, under a lock) and keeps it; make that first call before any stream
+ *     capture starts, and do not reset the device (cudaDeviceReset) while the library is loaded:
+ *     the kept address would be stale;
  *   - the array is shared by every call and every handle in the process and keeps what the last
  *     call left in it.  A call overwrites all of the part it uses before reading it, so stale
  *     contents are harmless, but two calls that overlap in time on the GPU (different streams, or
@@ -157,7 +162,8 @@ tardis_status_t tardis_ffn_forward_static(tardis_handle_t handle, const void* x,
  * and fp32 accumulation on the tensor cores (the batched speculative product X W_f^T of Section 5.4, the
  * fold W2 (diag(a) W1) of Section 5.2 and the batched pre-activations X W1^T all have this shape).
  * A: device bf16 [M, K] row-major with leading dimension lda; B: device bf16 [N, K] row-major (ldb);
- * C: device float [M, N] (ldc), fully overwritten.  K, lda, ldb multiples of 8; A, B 16-byte aligned.
+ * C: device float [M, N] (ldc), fully overwritten.  K, lda, ldb multiples of 8; A, B and C 16-byte aligned
+ * (a view that starts at an odd column is refused).
  * Asynchronous on `stream`.  Errors: INVALID_ARG, UNSUPPORTED (driver without tensor-map support), CUDA. */
 tardis_status_t tardis_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t lda,
                                  const void* B, int32_t ldb, float* C, int32_t ldc, tardis_stream_t stream);
@@ -184,8 +190,9 @@ tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf
 /* Offline statistics of one layer: the range and the linear function of every
  * neuron from calibration pre-activations.  The paper picks, per neuron, the
  * input range that holds a given portion of the profiled activation inputs and
- * fits y = a z + c to the activation inside it by least squares (Section 3.2,
- * Insight 2; Section 4.1 step 3; Section 5.1.2 step 4).  Here the range is
+ * fits y = a z + c to the activation inside it by least squares (the procedure is
+ * described with Insight 2 in Section 4.1; steps 2 and 3 of the list in Section 5.1;
+ * Section 5.1.1 for the single range and its linear function).  Here the range is
  * the one between the quantiles q_lo and q_hi of the neuron's samples (linear
  * interpolation between the order statistics around position q (n_cal - 1),
  * evaluated in double precision, stored in single); the fit is ordinary least
@@ -204,7 +211,9 @@ tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, in
                                  tardis_stream_t stream);
 
 /* Chooses the kernel path: 0 = automatic (default), 1 = always the generic
- * kernels, 3 = the batched tensor-core path for every token count (bf16
+ * kernels, 2 = the fused decode kernel for every token count up to 4096 (in
+ * launches of at most 4 tokens; layers it does not serve fall back as in 0),
+ * 3 = the batched tensor-core path for every token count (bf16
  * layers; other layers fall back to the generic kernels), 4 = the generic
  * kernels with the range check taken on the true pre-activations
  * z = W1 x + b1 instead of the predictor's scores: the paper's third scenario

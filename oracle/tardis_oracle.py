@@ -262,7 +262,7 @@ def rel_error(y, y_ref):
 # --------------------------------------------------------------------------
 def quantile_ranges(z, q_lo, q_hi):
     """Range of every neuron: the interval that holds a chosen share of the
-    activation inputs profiled for it (Section 3.2, Insight 2), taken here as
+    activation inputs profiled for it (Section 4.1, Insight 2, describes the procedure; Section 5.1, step 2), taken here as
     the central portion between the q_lo and q_hi quantiles of the neuron's
     calibration pre-activations.  z[h, N]: row j = the N samples of
     neuron j.  The quantile at level p is the linear interpolation between the
@@ -301,7 +301,7 @@ def gelu_derivative(z, act=ACT_GELU_TANH):
 
 def least_squares_fit(z, lo, hi, act=ACT_GELU_TANH):
     """The linear function y = a z + c of every neuron: the least-squares
-    regression (Section 4.1 step 3, Section 5.1.2 step 4) of the activation
+    regression (Section 5.1, step 3; Section 4.1, Insight 2) of the activation
     sigma(z) on z over the calibration samples inside the neuron's range
     lo <= z < hi:
         a = cov(z, sigma(z)) / var(z),   c = mean(sigma(z)) - a mean(z).

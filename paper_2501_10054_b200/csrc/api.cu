@@ -23,6 +23,13 @@ static Handle* check(tardis_handle_t h) {
   return H;
 }
 
+// A handle's memory and kernels belong to the device that was current at tardis_fold: a call made with another device
+// current would launch there against this handle's pointers.
+static bool on_handle_device(const Handle* H) {
+  int cur = -1;
+  return cudaGetDevice(&cur) == cudaSuccess && cur == H->device;
+}
+
 template <typename T>
 static tardis_status_t dev_alloc(T** p, size_t count, size_t* tally) {
   *p = nullptr;
@@ -130,6 +137,7 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   if (n_tokens < 0) return TARDIS_ERR_INVALID_ARG;
   if (n_tokens == 0) return TARDIS_OK;
   if (!x || !y || !aligned16(x) || !aligned16(y)) return TARDIS_ERR_INVALID_ARG;
+  if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   H->last_stream = s;
   tardis_status_t st;
@@ -169,13 +177,14 @@ tardis_status_t tardis_ffn_forward_static(tardis_handle_t handle, const void* x,
   if (st == TARDIS_ERR_UNSUPPORTED)
     snprintf(g_last_error, sizeof(g_last_error),
              "tardis_ffn_forward_static: n_tokens * (4 d_model + d_ff / 8) exceeds the 4 MiB of built-in scratch (or d_model > 12288)");
-  if (st == TARDIS_OK) { H->last_path = 4; H->calls += 1; H->tokens += uint64_t(n_tokens); }
+  if (st == TARDIS_OK) { H->last_path = 5; H->calls += 1; H->tokens += uint64_t(n_tokens); }
   return st;
 }
 
 tardis_status_t tardis_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t lda, const void* B, int32_t ldb,
                                  float* C, int32_t ldc, tardis_stream_t stream) {
   if (!A || !B || !C || M <= 0 || N <= 0 || K <= 0 || ldc < N) return TARDIS_ERR_INVALID_ARG;
+  if (!aligned16(C)) return TARDIS_ERR_INVALID_ARG;   // the epilogue stores (and reduces) 16 bytes at a time when ldc % 4 == 0
   GemmArgs g = {};
   g.M = M; g.N = N; g.K1 = K; g.K2 = 0;
   g.A1 = A; g.B1 = B; g.lda1 = lda; g.ldb1 = ldb;
@@ -194,6 +203,7 @@ tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, in
 tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
   Handle* H = check(handle);
   if (!H || !out) return TARDIS_ERR_INVALID_ARG;
+  if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
   TARDIS_CUDA_TRY(cudaStreamSynchronize(H->last_stream));
   unsigned long long ctr[CTR_COUNT];
   TARDIS_CUDA_TRY(cudaMemcpy(ctr, H->counters, sizeof(ctr), cudaMemcpyDeviceToHost));
@@ -221,6 +231,7 @@ tardis_status_t tardis_set_debug_capture(tardis_handle_t handle, uint32_t* flag_
 tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf, tardis_stream_t stream) {
   Handle* H = check(handle);
   if (!H) return TARDIS_ERR_INVALID_ARG;
+  if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   H->last_stream = s;
   return launch_export_folded(H, Wf, bf, s);

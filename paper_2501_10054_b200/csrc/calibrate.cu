@@ -1,4 +1,4 @@
-// Offline statistics of a layer (Sections 3.2 and 5.1.2): from the calibration pre-activations of every neuron,
+// Offline statistics of a layer (Section 5.1, steps 2 and 3; the procedure is described with Insight 2 in Section 4.1): from the calibration pre-activations of every neuron,
 // the range that holds the central portion of them (quantiles q_lo, q_hi) and the least-squares line
 // y = a z + c of GELU over the samples inside that range.
 //

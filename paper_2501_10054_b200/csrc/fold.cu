@@ -2,7 +2,7 @@
 //   C[k, i] = W_f[i, k] = sum_j W2[i, j] a_j W1[j, k],   b_f = W2 (a .* b1 + c) + b2,
 // plus the W2 -> W2T[h, d] transpose that makes a neuron's output weights contiguous.
 // Accumulation is fp32 for bf16 storage and fp64 for fp32 storage; one rounding at the end
-// (the paper's precision study, Section 7.6, shows bf16 intermediates are not good enough).
+// (the paper's precision study, Section 7.7, shows bf16 intermediates are not good enough).
 #include "common.cuh"
 
 namespace tardis {

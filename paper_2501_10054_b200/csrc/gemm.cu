@@ -478,6 +478,9 @@ tardis_status_t launch_gemm(const GemmArgs& g, cudaStream_t s) {
                                          g.codes && g.scale && g.zero && g.xsrc))
     return TARDIS_ERR_INVALID_ARG;
   if (g.splits > 1 && g.epilogue != GEMM_EPI_F32) return TARDIS_ERR_INVALID_ARG;
+  // the epilogues store (or reduce) 16 bytes at a time
+  auto misaligned = [](const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15u); };
+  if (misaligned(g.out_f32) || misaligned(g.out_bf16) || misaligned(g.addend)) return TARDIS_ERR_INVALID_ARG;
   // wide tiles when they still fill the machine, narrow ones for skinny problems
   const long tiles256 = long((g.N + 255) / 256) * ((g.M + BM - 1) / BM) * (g.splits > 1 ? g.splits : 1);
   if (tiles256 >= 120) return launch_bn<256>(g, s);

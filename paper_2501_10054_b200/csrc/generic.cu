@@ -1,6 +1,8 @@
 // Generic kernels of the online path (Section 5.4) for any dtype, shape and token count:
 // exact predictor score + flag, folded product, result fixing.  They favour exactness and
 // simplicity; the fused decode kernel and the batched tensor-core path are the fast ones.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace tardis {
@@ -258,7 +260,9 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 // once per device.
 static tardis_status_t static_scratch_address(int device, unsigned char** out) {
   static unsigned char* cache[kStaticMaxDevices] = {};
+  static std::mutex guard;                       // first calls of two host threads must not race on the cache
   if (device < 0 || device >= kStaticMaxDevices) return TARDIS_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(guard);
   if (!cache[device]) {
     void* ptr = nullptr;
     TARDIS_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
@@ -271,8 +275,12 @@ static tardis_status_t static_scratch_address(int device, unsigned char** out) {
 template <typename T, typename Acc>
 static tardis_status_t static_typed(Handle* H, const T* x, T* y, int n, float* yacc, uint32_t* bitmap, cudaStream_t s) {
   const int d = H->d, h = H->h;
-  k_predictor_exact<T><<<h / 32, 1024, 0, s>>>(H->codes, static_cast<const T*>(H->scale), H->zero, H->b1, H->lo, H->hi,
-                                               x, n, d, h, H->G, H->bits, bitmap, H->dbg_bitmap, H->dbg_scores);
+  if (H->path_override == 4)                    // exact-range mode: flags from the true pre-activations, as in generic_typed
+    k_range_check_exact<T><<<h / 32, 1024, 0, s>>>(static_cast<const T*>(H->W1), H->b1, H->lo, H->hi, x, n, d, h, bitmap,
+                                                   H->dbg_bitmap, H->dbg_scores);
+  else
+    k_predictor_exact<T><<<h / 32, 1024, 0, s>>>(H->codes, static_cast<const T*>(H->scale), H->zero, H->b1, H->lo, H->hi,
+                                                 x, n, d, h, H->G, H->bits, bitmap, H->dbg_bitmap, H->dbg_scores);
   k_flag_stats<<<n, 256, 0, s>>>(bitmap, h / 32, H->counters);
   const size_t cnt = size_t(n) * d;
   k_init_yacc<<<unsigned((cnt + 255) / 256), 256, 0, s>>>(yacc, H->bf, n, d);

@@ -1,7 +1,9 @@
 """Parity at the full sizes of the five benchmark configurations, in the launch shapes bench.py times
-(batch-1 decode, batched decode, prefill chunks).  The GPU runs every token; the oracle checks a seeded
-sample of them one by one through the direct definition of the partially linear FFN (no d x d fold
-needed), which equals the folded path by the pinned identities."""
+(batch-1 decode, batched decode, prefill chunks).  The GPU runs every token.  The oracle computes the
+predictor scores and flags of EVERY token (one BLAS product per quantisation group) and compares them
+bit for bit outside the excluded band; the outputs are checked on a seeded sample of the tokens, one by
+one, through the direct definition of the partially linear FFN (no d x d fold needed), which equals the
+folded path by the pinned identities."""
 import numpy as np
 import pytest
 import torch
@@ -14,7 +16,7 @@ from tests import helpers as Hp
 pytestmark = pytest.mark.gpu
 
 
-def _check(cfg, batches, sample_per_call, seed=0, fold_rows=8):
+def _check(cfg, batches, sample_per_call, seed=0, fold_rows=8, flag_tokens=None):
     dev = torch.device("cuda", 0)
     L = W.make_layer(cfg, seed, device=dev)
     s = L.numpy64()
@@ -38,6 +40,24 @@ def _check(cfg, batches, sample_per_call, seed=0, fold_rows=8):
         st = T.tardis_stats(h)
         assert st["device_error"] == 0 and st["tokens"] == n
         assert st["flagged_total"] == int(F.sum())
+        # flags of every token (or of the first `flag_tokens` tokens of every call, where the full product would take
+        # the CPU minutes) against the oracle's scores
+        sel, t1 = [], 0
+        for b in batches:
+            sel += list(range(t1, t1 + (b if flag_tokens is None else min(b, flag_tokens))))
+            t1 += b
+        sel = np.asarray(sel)
+        band_total = 0
+        for c0 in range(0, len(sel), 512):
+            part = sel[c0:c0 + 512]
+            x64 = x[torch.as_tensor(part, device=dev)].double().cpu().numpy()
+            zhat = O.predictor_score(x64, s["codes"], s["scale"], s["zero"], s["group"], s["b1"], s["bits"])
+            F_ref = O.flags_from_score(zhat, s["lo"], s["hi"])
+            band = O.near_threshold(zhat, s["lo"], s["hi"], Hp.BAND)
+            mism = (F[part] != F_ref) & ~band
+            assert not mism.any(), "%s: %d flag mismatches outside the band over %d tokens" % (cfg.name, mism.sum(), len(part))
+            band_total += int(band.sum())
+        print("%s: flags of %d tokens compared, %d (token, neuron) pairs inside the 1e-6 band" % (cfg.name, len(sel), band_total))
         # sampled tokens of every call
         idx, t0 = [], 0
         for b in batches:
@@ -60,7 +80,7 @@ def test_decode_7b_batch1_and_batch64():
     assert 0.07 < frac < 0.13
 
 
-@pytest.mark.parametrize("q", [0, 2])
+@pytest.mark.parametrize("q", [0, 1, 2, 3])
 def test_falcon_shape_decode_batches(q):
     import dataclasses
     qlo, qhi = W.FALCON_QUANTILES[q]
@@ -69,11 +89,14 @@ def test_falcon_shape_decode_batches(q):
     assert 0.02 < frac < 0.45
 
 
-def test_prefill_layer_2048_tokens():
-    info, frac = _check(W.CONFIGS["prefill_7b"], [2048], sample_per_call=12, seed=3)
+@pytest.mark.parametrize("seed", [3, 4])
+def test_prefill_layers_4096_tokens_in_one_call(seed):
+    # two independently seeded layers of the prefill configuration; one call crosses the 2048-token chunk of the batched
+    # path (1024 while the capture is on) several times
+    info, frac = _check(W.CONFIGS["prefill_7b"], [4096], sample_per_call=12, seed=seed)
     assert 0.07 < frac < 0.13
 
 
 def test_large_8k_decode_and_prefill():
-    info, frac = _check(W.CONFIGS["large_8k"], [1, 1, 32, 1500], sample_per_call=3, fold_rows=4)
+    info, frac = _check(W.CONFIGS["large_8k"], [1, 1, 32, 4096], sample_per_call=3, fold_rows=4, flag_tokens=256)
     assert 0.07 < frac < 0.13

@@ -200,7 +200,8 @@ def test_run_to_run_flags_identical():
     h = T.fold_layer(L)
     y1, F1, S1 = Hp.gpu_forward(h, L, x, [8])
     y2, F2, S2 = Hp.gpu_forward(h, L, x, [8])
-    assert (F1 == F2).all() and np.abs(S1 - S2).max() <= 1e-4
+    # the fused kernel adds its partial scores in a fixed order: the captured scores of two runs are the same numbers
+    assert (F1 == F2).all() and (S1 == S2).all()
     assert (y1.float() - y2.float()).abs().max() <= 2e-2 * y1.float().abs().max()
     T.tardis_destroy(h)
 

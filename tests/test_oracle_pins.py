@@ -222,6 +222,50 @@ def test_unpack_convention():
     assert q[0, :4].tolist() == [1, 2, 3, 0] and q[0, 15] == 3 and q[0, 16] == 3 and q[0, 17:].sum() == 0
 
 
+def test_unpack_convention_4_and_8_bits():
+    # The packing rule of the interface: with p = 32 / bits codes per word, channel k sits in word k / p, bits
+    # bits * (k % p) upwards.  The words are written out by hand (hex digits = 4-bit codes, bytes = 8-bit codes).
+    # 4 bits: word 0 holds channels 0..7 = 1,2,3,4,5,6,7,15 -> hex digits from the low end: 0xF7654321;
+    #         word 1 holds channels 8..15 = 0,0,0,0,0,0,0,9 -> 0x90000000
+    q4 = O.unpack_codes(np.array([[0xF7654321, 0x90000000]], dtype=np.uint32), 16, bits=4)
+    assert q4[0].tolist() == [1, 2, 3, 4, 5, 6, 7, 15, 0, 0, 0, 0, 0, 0, 0, 9]
+    # 8 bits: word 0 holds channels 0..3 = 0x01, 0x80, 0xFF, 0x10 -> 0x10FF8001; word 1 channels 4..7 = 7,0,0,200 -> 0xC8000007
+    q8 = O.unpack_codes(np.array([[0x10FF8001, 0xC8000007]], dtype=np.uint32), 8, bits=8)
+    assert q8[0].tolist() == [0x01, 0x80, 0xFF, 0x10, 7, 0, 0, 200]
+    # a transposed field order (channel k in the HIGH bits first) would give other lists: check one against the wrong reading
+    assert q4[0].tolist() != [15, 7, 6, 5, 4, 3, 2, 1, 9, 0, 0, 0, 0, 0, 0, 0]
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_predictor_score_scalar_loops_4_and_8_bits(bits):
+    # scalar-loop evaluation of zhat = b1 + sum_g s (sum_k (q - zp) x) straight from hand-packed words, against the oracle
+    rng = np.random.default_rng(100 + bits)
+    per = 32 // bits
+    h, d, G = 3, 32, 16
+    q = rng.integers(0, 1 << bits, size=(h, d))
+    words = np.zeros((h, d // per), dtype=np.uint32)
+    for j in range(h):
+        for k in range(d):
+            words[j, k // per] |= np.uint32(int(q[j, k]) << (bits * (k % per)))
+    s = rng.uniform(0.01, 0.1, size=(h, d // G))
+    zp = rng.integers(0, 1 << bits, size=(h, d // G)).astype(np.uint8)
+    b1 = rng.normal(size=h)
+    x = rng.normal(size=(2, d))
+    want = np.zeros((2, h))
+    for t in range(2):
+        for j in range(h):
+            acc = b1[j]
+            for g in range(d // G):
+                inner = 0.0
+                for k in range(g * G, (g + 1) * G):
+                    inner += (int(q[j, k]) - int(zp[j, g])) * x[t, k]
+                acc += s[j, g] * inner
+            want[t, j] = acc
+    got = O.predictor_score(x, words, s, zp, G, b1, bits)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    assert O.unpack_codes(words, d, bits).tolist() == q.tolist()
+
+
 def _pack(q):
     h, d = q.shape
     w = np.zeros((h, d // 16), dtype=np.uint64)

@@ -5,8 +5,8 @@ A process that gave all device memory to its own pool at start-up, or that runs 
 callers the library offers a forward whose scratch is a fixed array inside the library image.  This
 test calls it through the C ABI twice in a row (the array is shared and keeps the previous call's
 contents, so the second call runs on a dirty array) and checks each result against the ordinary
-tardis_ffn_forward on the same inputs, under the tolerance the parity tests use; it also checks the
-size limit.  The file name makes pytest collect it after every other test.
+tardis_ffn_forward on the same inputs and against the fp64 oracle (flags bit for bit, outputs under
+the tolerance the parity tests use); it also checks the exact-range mode and the size limit.  The file name makes pytest collect it after every other test.
 """
 import pytest
 import torch
@@ -28,6 +28,7 @@ def _max_rel(y, y_ref):
 def test_static_scratch_forward_matches_regular_forward_twice(dtype):
     cfg = W.LayerConfig("noalloc_" + dtype, 512, 2048, dtype=dtype, n_calib=512)
     L = Hp.to_cuda(W.make_layer(cfg, 3))
+    s64 = L.numpy64()
     h = T.fold_layer(L)
     lib = T.load_library()
     try:
@@ -45,7 +46,24 @@ def test_static_scratch_forward_matches_regular_forward_twice(dtype):
             assert torch.cuda.mem_get_info()[0] == free_before       # nothing was taken from the device
             assert torch.isfinite(y.float()).all()
             assert _max_rel(y, y_ref) <= Hp.TOL[dtype], "call %d" % call
-            assert T.tardis_stats(h)["last_path"] == 4
+            assert T.tardis_stats(h)["last_path"] == 5
+            # and against the oracle: flags captured from the static entry, outputs of the static entry
+            bm = torch.zeros(n, cfg.d_ff // 32, dtype=torch.int32, device="cuda")
+            T.tardis_set_debug_capture(h, bm, None)
+            y2 = torch.full_like(x, float("nan"))
+            assert lib.tardis_ffn_forward_static(h, x.data_ptr(), y2.data_ptr(), n, None) == 0
+            torch.cuda.synchronize()
+            T.tardis_set_debug_capture(h, None, None)
+            Hp.assert_parity(L, s64, x, y2, Hp.unpack_bitmap(bm, cfg.d_ff), None, score_tol=None, label="static call %d" % call)
+        # exact-range mode (flags from the true pre-activations) is honoured by the static entry as by the ordinary one
+        x = W.make_tokens(cfg, 9, 21).cuda()
+        y_a, y_b = torch.empty_like(x), torch.empty_like(x)
+        T.tardis_set_path(h, 4)
+        T.tardis_ffn_forward(h, x, y_a)
+        assert lib.tardis_ffn_forward_static(h, x.data_ptr(), y_b.data_ptr(), 9, None) == 0
+        torch.cuda.synchronize()
+        assert _max_rel(y_b, y_a) <= Hp.TOL[dtype]
+        T.tardis_set_path(h, 1)
         # beyond the limits: refused with a clear message, nothing launched
         x = W.make_tokens(cfg, 65, 13).cuda()
         y = torch.empty_like(x)
