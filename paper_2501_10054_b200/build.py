@@ -36,7 +36,7 @@ def build(force: bool = False, verbose: bool = False, stamps: bool = False) -> s
     if not force and not stamps and not needs_build():
         return LIB
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+           "-Xcompiler", "-fPIC", "-shared", "-t", "8", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", out] + (["-DTARDIS_PHASE_STAMPS"] if stamps else []) + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")

@@ -51,7 +51,8 @@ constexpr int MAXRC = 64;         // exact re-checks per CTA and pass before the
 constexpr int MAXBUF = 10;        // predictor tile buffers in shared memory
 constexpr int MAXGROUPS = 4;      // slot groups (one barrier each, one buffer of partial sums each) of the result fixing
 constexpr int MAXGS = 8;          // rows per slot group (half an MMA tile: the other half of the operand is zero)
-constexpr int NREP = 4;           // replicas of the output accumulator
+constexpr int NREP = 1;           // replicas of the output accumulator (more replicas spread the reductions, but the last CTA
+                                  // reads them all: one measured fastest)
 constexpr int CTMAX = 9;          // 16-column output tiles per warp (d <= 32 * 16 * CTMAX = 4608)
 // control words (unsigned int) in global scratch; all zero between calls
 constexpr int CTL_TICKET = 0;     // next unit of the folded matrix
@@ -85,7 +86,7 @@ struct Params {
 
 struct Scratch {           // handle-owned device memory of this path
   uint8_t* pblocks; int2* plan; float* smax; float* yacc; unsigned int* ctl; uint4* Cp;
-  Params base; size_t smem_bytes; size_t bytes; int grid; const void* kernel;
+  Params base; size_t smem_bytes; size_t bytes; int grid; const void* kernels[2][2]; bool pairs_fit;
   int nbuf_n[MAXT + 1];    // tile buffers in shared memory for a call of n tokens
 };
 
@@ -173,7 +174,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------------
-template <int G, int CT>
+// G: predictor group size; CT: 16-column output tiles per warp; NTK: 1 = the call has one token (most of the token loops
+// fold away), 4 = up to four; FAST: every tile of the CTA has its own buffer and a warp has the same one or two channel
+// pairs in every tile (their x operands stay in registers), else the general loop over a ring of tile buffers.
+template <int G, int CT, int NTK, bool FAST>
 __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const SmemLayout L(p.dpad, p.ngroups, p.tiles_max, p.nbuf, p.buf_bytes, p.n, size_t(p.smem_total));
@@ -194,14 +198,14 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   volatile int* misc = reinterpret_cast<volatile int*>(smem + L.misc);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int d = p.d, n = p.n;
+  const int d = p.d, n = NTK == 1 ? 1 : p.n;
   const int TR = p.tiles_max * 16;
   const int XS = L.xstride, xq_stride = L.xq_stride;
   const int2 plan = p.plan[blockIdx.x];
   const int NU = plan.y;                           // predictor units (tiles) of this CTA
   const int NP = (n + 1) >> 1;                     // predictor passes (two tokens each)
   const int NQ = NU * NP;                          // units in the order they are consumed
-  const bool resident = NU <= p.nbuf;              // every tile has its own buffer: nothing is fetched twice
+  const bool resident = FAST || NU <= p.nbuf;      // every tile has its own buffer: nothing is fetched twice
   const int g = lane >> 2, t4 = lane & 3;
   const int nv = p.dpad >> 3;                      // 8-channel vectors per token (padded)
   const int nrow = plan.y * 16;
@@ -519,7 +523,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
         sxa = sxl[grp * 2];
         sxb = G == 64 ? sxl[(grp + 1) * 2] : 0;
       };
-      if (resident && (npairs == NWP || npairs == 2 * NWP)) {
+      if (FAST) {
         // every tile is in shared memory behind one barrier, and a warp has the same one or two pairs in every tile:
         // their x operands stay in registers
         const bool two = npairs == 2 * NWP;
@@ -676,19 +680,19 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   const int nslots = int((L.slots_end - L.pbuf) / size_t(p.slot_stride));
   const int NG = nslots >= 4 * MAXGS ? 4 : (nslots >= 12 ? 3 : 2);
   const int GS = min(MAXGS, nslots / NG);
-  // fills the group of step st; thread 0 arms the barrier, lane 0 of warp k < nwarps issues the k-th copy
-  auto fill = [&](int st, int nun, int nwarps) {
+  // fills the group of step st: warp `issuer` arms the barrier and its lanes issue one copy each
+  auto fill = [&](int st, int nun, int issuer) {
     const int nA = (nun + GS - 1) / GS;                             // steps over W1 rows (as many again over W2^T rows)
-    if (st >= 2 * nA) return;
+    if (st >= 2 * nA || warp != issuer) return;
     const bool second = st >= nA;
     const int i0 = (second ? st - nA : st) * GS, cnt = min(GS, nun - i0);
     const int gr = st % NG;
-    if (tid == 0) mbar_expect_tx(&fixbar[gr], uint32_t(cnt) * rowbytes);
-    if (lane == 0)
-      for (int k = warp; k < cnt; k += nwarps) {
-        const __nv_bfloat16* src = (second ? p.W2T : p.W1) + size_t(fl_j[i0 + k]) * d;
-        bulk_g2s(slots + size_t(gr * GS + k) * p.slot_stride, src, rowbytes, &fixbar[gr]);
-      }
+    if (lane == 0) mbar_expect_tx(&fixbar[gr], uint32_t(cnt) * rowbytes);
+    __syncwarp();
+    if (lane < cnt) {
+      const __nv_bfloat16* src = (second ? p.W2T : p.W1) + size_t(fl_j[i0 + lane]) * d;
+      bulk_g2s(slots + size_t(gr * GS + lane) * p.slot_stride, src, rowbytes, &fixbar[gr]);
+    }
   };
   auto wait_group = [&](int st) -> bool {
     const int gr = st % NG;
@@ -703,8 +707,8 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   // the predictor warps start the first copies on their own: the streaming warps may still be busy
   if (warp < NWP) {
     const int nun = misc[MS_NUN];
-    if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the region was read with ordinary loads
-    for (int st = 0; st < NG; ++st) fill(st, nun, NWP);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the region was read with ordinary loads
+    for (int st = 0; st < NG; ++st) fill(st, nun, st);
   }
   __syncthreads();
   const int nun = misc[MS_NUN];
@@ -755,8 +759,8 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
         if (2 * t4 + 1 < n) wzs[(n * g + 2 * t4 + 1) * 33 + warp] = c[1];
       }
       __syncthreads();                                              // partial sums complete; the rows are used
-      if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      for (int st = c0; st < c1; ++st) fill(st + NG, nun, NW);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      for (int st = c0; st < c1; ++st) fill(st + NG, nun, NW - 1 - (st - c0));
       // a warp adds up the 32 partial sums of a pair (a fixed tree) and turns them into delta
       const int npair = (c1 - c0) * GS * n;
       for (int pq = warp; pq < npair; pq += NW) {
@@ -814,8 +818,8 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
       }
       if (st + NG < 2 * nA) {
         __syncthreads();                                            // rows used
-        if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        fill(st + NG, nun, NW);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fill(st + NG, nun, NW - 1);
       }
     }
   }
@@ -1033,9 +1037,19 @@ tardis_status_t fused_prepare(Handle* H, cudaStream_t s) {
   k_max_scale<<<64, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(H->scale), size_t(h) * H->ngroups, S->smax);
   e = cudaGetLastError();
   const bool wide = dpad > 32 * 16 * 8;
-  S->kernel = G == 64 ? (wide ? (const void*)k_fused<64, 9> : (const void*)k_fused<64, 8>)
-                      : (wide ? (const void*)k_fused<128, 9> : (const void*)k_fused<128, 8>);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(S->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+  // kernels[one token or more][ring or fast]
+  if (G == 64 && wide) { S->kernels[0][0] = (const void*)k_fused<64, 9, 1, false>; S->kernels[0][1] = (const void*)k_fused<64, 9, 1, true>;
+                         S->kernels[1][0] = (const void*)k_fused<64, 9, 4, false>; S->kernels[1][1] = (const void*)k_fused<64, 9, 4, true>; }
+  else if (G == 64) { S->kernels[0][0] = (const void*)k_fused<64, 8, 1, false>; S->kernels[0][1] = (const void*)k_fused<64, 8, 1, true>;
+                      S->kernels[1][0] = (const void*)k_fused<64, 8, 4, false>; S->kernels[1][1] = (const void*)k_fused<64, 8, 4, true>; }
+  else if (wide) { S->kernels[0][0] = (const void*)k_fused<128, 9, 1, false>; S->kernels[0][1] = (const void*)k_fused<128, 9, 1, true>;
+                   S->kernels[1][0] = (const void*)k_fused<128, 9, 4, false>; S->kernels[1][1] = (const void*)k_fused<128, 9, 4, true>; }
+  else { S->kernels[0][0] = (const void*)k_fused<128, 8, 1, false>; S->kernels[0][1] = (const void*)k_fused<128, 8, 1, true>;
+         S->kernels[1][0] = (const void*)k_fused<128, 8, 4, false>; S->kernels[1][1] = (const void*)k_fused<128, 8, 4, true>; }
+  for (int a = 0; a < 2 && e == cudaSuccess; ++a)
+    for (int b = 0; b < 2 && e == cudaSuccess; ++b)
+      e = cudaFuncSetAttribute(S->kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+  S->pairs_fit = (p.nkc * 2 == NWP || p.nkc * 2 == 2 * NWP);
   if (e != cudaSuccess) { set_last_error(e, "fused_prepare launch"); return fail(TARDIS_ERR_CUDA); }
 
   p.pblocks = S->pblocks; p.plan = S->plan; p.smax = S->smax; p.yacc = S->yacc; p.ctl = S->ctl;
@@ -1070,7 +1084,8 @@ tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     void* args[] = {&p};
-    TARDIS_CUDA_TRY(cudaLaunchKernelExC(&cfg, S->kernel, args));
+    const bool fast = S->pairs_fit && S->nbuf_n[nt] >= p.tiles_max;
+    TARDIS_CUDA_TRY(cudaLaunchKernelExC(&cfg, S->kernels[nt == 1 ? 0 : 1][fast ? 1 : 0], args));
     H->launches += 1;
     t0 += nt;
   }
