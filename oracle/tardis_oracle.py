@@ -335,3 +335,117 @@ def least_squares_fit(z, lo, hi, act=ACT_GELU_TANH):
         a[j] = np.float32(aj)
         c[j] = np.float32(cj)
     return a, c
+
+
+# --------------------------------------------------------------------------
+# offline: the greedy range search of Algorithm 1 (Section 5.1.1, "Range Searching")
+# --------------------------------------------------------------------------
+def kde_centroid(samples):
+    """Centroid of a neuron's activation inputs by kernel density estimation (Algorithm 1, find_centroid): the
+    sample at which a Gaussian kernel density estimate of the samples is highest.  The paper names KDE but not the
+    kernel or its width; the reading taken here: Gaussian kernel, Silverman's rule-of-thumb width
+    bw = 1.06 * std * N^(-1/5) (std with N - 1 in the denominator), density evaluated at the samples themselves,
+    ties to the smallest sample.  With bw = 0 (all samples equal) or a single sample that value is the centroid."""
+    z = np.sort(_as64(samples).ravel())
+    n = z.size
+    if n == 1:
+        return float(z[0])
+    bw = 1.06 * np.std(z, ddof=1) * n ** (-0.2)
+    if not bw > 0.0:
+        return float(z[0])
+    dens = np.empty(n)
+    for i in range(n):
+        u = (z - z[i]) / bw
+        dens[i] = np.exp(-0.5 * u * u).sum()
+    return float(z[int(np.argmax(dens))])
+
+
+def approx_error(samples, lo, hi, act=ACT_GELU_TANH):
+    """Error of approximating the activation by its least-squares line over the samples inside [lo, hi)
+    (Algorithm 1, approx_error; Section 4.1 measures it as a mean squared error): the mean of the squared residuals
+    of that line.  Fewer than two samples in range, or samples that do not vary: 0 (a line fits them exactly)."""
+    z = _as64(samples).ravel()
+    zin = z[(z >= lo) & (z < hi)]
+    if zin.size < 2:
+        return 0.0
+    g = gelu(zin, act)
+    mz, mg = zin.mean(), g.mean()
+    dz, dg = zin - mz, g - mg
+    var = (dz * dz).mean()
+    if not var > 1e-30:
+        return 0.0
+    a = (dz * dg).mean() / var
+    r = dg - a * dz
+    return float((r * r).mean())
+
+
+def greedy_range_search(samples, t, step, act=ACT_GELU_TANH, return_trace=False):
+    """Range of one neuron by Algorithm 1: start from the empty range at the KDE centroid; while the share of the
+    samples inside the range is below the threshold t, form the range extended by `step` to the left and the range
+    extended by `step` to the right, measure the approximation error of each, and keep the one with the smaller
+    error (the right one on a tie).  Ranges are half-open, [lo, hi).
+
+    The printed listing builds the left candidate as (R.left - s, R.left) and the right one as (R.left, R.right + s);
+    taken literally the left candidate would drop everything found so far, so the reading is (R.left - s, R.right)
+    and (R.left, R.right + s): each candidate is the current range grown on one side.  Bounds are kept as
+    centroid - k_left * step and centroid + k_right * step with integer step counts, so that no rounding accumulates.
+    The loop also stops once the range holds every sample, and a side that has passed the outermost sample is not
+    grown any further (the other side is taken without comparing errors).
+
+    Returns (lo, hi) as Python floats (and, with return_trace, the list of 'L'/'R' choices and the smallest
+    relative margin |err_left - err_right| / max(err_left, err_right) seen, a measure of how close a decision was)."""
+    z = np.sort(_as64(samples).ravel())
+    n = z.size
+    c = kde_centroid(z)
+    kl = kr = 0
+    trace, margin = [], float("inf")
+    while True:
+        lo, hi = c - kl * step, c + kr * step
+        inside = int(((z >= lo) & (z < hi)).sum())
+        if inside >= t * n or inside == n:
+            break
+        lo_l, hi_r = c - (kl + 1) * step, c + (kr + 1) * step
+        # a side that already reaches past the outermost sample has nothing left to add: the other side is taken
+        # (as printed, the loop would grow such a side for ever whenever its error stays the smaller one)
+        if hi > z[-1]:
+            go_left = True
+        elif lo <= z[0]:
+            go_left = False
+        else:
+            e_l = approx_error(z, lo_l, hi, act)
+            e_r = approx_error(z, lo, hi_r, act)
+            m = max(e_l, e_r)
+            if m > 0.0:
+                margin = min(margin, abs(e_l - e_r) / m)
+            go_left = e_l < e_r
+        if go_left:
+            kl += 1
+            trace.append("L")
+        else:
+            kr += 1
+            trace.append("R")
+    lo, hi = c - kl * step, c + kr * step
+    if return_trace:
+        return lo, hi, trace, margin
+    return lo, hi
+
+
+def neuron_thresholds(err, t_layer, t_min, t_max):
+    """Neuron-level thresholds of Section 5.1.1: minimise sum_n E_n t_n subject to sum_n t_n = t_layer * h.  As printed
+    the problem has no bounds on t_n and is unbounded; the reading taken here adds the box t_min <= t_n <= t_max
+    (t_min <= t_layer <= t_max).  A linear objective over a box with one equality constraint is minimised greedily:
+    every neuron starts at t_min, and the remaining budget goes, up to t_max each, to the neurons in order of
+    increasing error (ties to the smaller index); at most one neuron ends strictly between the bounds."""
+    err = _as64(err).ravel()
+    h = err.size
+    if not (t_min <= t_layer <= t_max):
+        raise ValueError("need t_min <= t_layer <= t_max")
+    t = np.full(h, float(t_min))
+    budget = (t_layer - t_min) * h
+    for j in np.argsort(err, kind="stable"):
+        give = min(t_max - t_min, budget)
+        t[j] += give
+        budget -= give
+        if budget <= 0.0:
+            break
+    return t

@@ -16,13 +16,13 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
 }
 __device__ __forceinline__ bool mbar_test(uint64_t* b, uint32_t parity) {
   uint32_t ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+  asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
                : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
   return ok != 0;
 }
 // Bounded wait: false when the limit ran out (the caller records the error and goes on without the
-// data).  mbarrier.try_wait suspends the thread by itself until the phase completes or a short hardware time-out
-// passes, so the loop needs no sleep of its own; the limit is in SM clock cycles (a fraction of a second).
+// data).  The test is the non-blocking form (the potentially blocking try_wait was measured to take several hundred
+// cycles even on a completed phase); the limit is in SM clock cycles (a fraction of a second).
 constexpr long long WAIT_LIMIT_CYCLES = 400000000ll;
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, long long limit = WAIT_LIMIT_CYCLES) {
   if (mbar_test(b, parity)) return true;

@@ -427,3 +427,100 @@ def test_relu_values_and_fit_special_cases():
     a, c = O.least_squares_fit(np.array([[9.0], [9.0]]), np.array([-2.0, 1.0], np.float32), np.array([-1.0, 2.0], np.float32),
                                O.ACT_RELU)
     assert (a[0], c[0], a[1], c[1]) == (0.0, 0.0, 1.0, 0.0)
+
+
+# ------------------------------------------------------------------ Algorithm 1: range search (Section 5.1.1)
+def test_kde_centroid_against_library_kde_and_special_cases():
+    from scipy.stats import gaussian_kde
+    rng = np.random.default_rng(7)
+    z = np.concatenate([rng.normal(-1.0, 0.3, 300), rng.normal(2.0, 1.0, 100)])       # dense cluster + sparse cluster
+    c = O.kde_centroid(z)
+    # library KDE with the same kernel width (factor times the sample standard deviation), evaluated at the samples
+    kde = gaussian_kde(z, bw_method=1.06 * z.size ** -0.2)
+    zs = np.sort(z)
+    assert c == zs[int(np.argmax(kde(zs)))]
+    assert -1.6 < c < -0.4                                  # the search starts in the denser cluster
+    # shifting the samples shifts the centroid; all-equal samples and a single sample give that value
+    assert O.kde_centroid(z + 3.0) == pytest.approx(c + 3.0, abs=1e-12)
+    assert O.kde_centroid(np.full(9, 0.25)) == 0.25 and O.kde_centroid([1.5]) == 1.5
+    # symmetric samples with one centre point: the centre is the densest point
+    sym = np.concatenate([-np.arange(1, 40) ** 1.3, [0.0], np.arange(1, 40) ** 1.3]) * 0.01
+    assert O.kde_centroid(sym) == 0.0
+
+
+def test_approx_error_against_polyfit_and_exact_cases():
+    rng = np.random.default_rng(8)
+    z = rng.normal(size=400) * 1.5
+    lo, hi = -1.0, 0.7
+    zin = z[(z >= lo) & (z < hi)]
+    g = O.gelu(zin, O.ACT_GELU_TANH)
+    coef, res, *_ = np.polyfit(zin, g, 1, full=True)         # library least squares: sum of squared residuals
+    assert O.approx_error(z, lo, hi) == pytest.approx(res[0] / zin.size, rel=1e-9)
+    # ReLU is a straight line on either side of 0: no error there, some across the kink
+    assert O.approx_error(z, 0.0, 5.0, O.ACT_RELU) == pytest.approx(0.0, abs=1e-25)
+    assert O.approx_error(z, -5.0, 0.0, O.ACT_RELU) == 0.0
+    assert O.approx_error(z, -1.0, 1.0, O.ACT_RELU) > 1e-3
+    # half-open range and the fewer-than-two rule
+    assert O.approx_error([0.0, 1.0, 2.0], 0.0, 2.0) == O.approx_error([0.0, 1.0], 0.0, 2.0) == pytest.approx(0.0, abs=1e-30)
+    assert O.approx_error([0.5], 0.0, 1.0) == 0.0 and O.approx_error([3.0, 4.0], 0.0, 1.0) == 0.0
+
+
+def test_greedy_range_search_properties_and_closed_form_trace():
+    rng = np.random.default_rng(9)
+    z = np.sort(rng.standard_t(4, size=300) * 0.8 - 0.3)
+    for t, step in ((0.5, 0.05), (0.85, 0.02), (0.97, 0.1)):
+        lo, hi, trace, margin = O.greedy_range_search(z, t, step, return_trace=True)
+        c = O.kde_centroid(z)
+        inside = ((z >= lo) & (z < hi)).mean()
+        assert inside >= t                                     # the threshold is reached ...
+        kl, kr = trace.count("L"), trace.count("R")
+        assert lo == c - kl * step and hi == c + kr * step and lo <= c <= hi
+        # ... and was not reached one step earlier (the last step is undone on its side)
+        if trace[-1] == "L":
+            assert ((z >= lo + step) & (z < hi)).mean() < t
+        else:
+            assert ((z >= lo) & (z < hi - step)).mean() < t
+    # every decision re-derived from a library fit: the side with the smaller mean squared residual (right on ties)
+    lo, hi, trace, margin = O.greedy_range_search(z, 0.6, 0.05, return_trace=True)
+    c, kl, kr = O.kde_centroid(z), 0, 0
+
+    def mse(a, b):
+        zin = z[(z >= a) & (z < b)]
+        if zin.size < 2 or np.ptp(zin) == 0:
+            return 0.0
+        g = O.gelu(zin, O.ACT_GELU_TANH)
+        p = np.polyfit(zin, g, 1)
+        return float(np.mean((g - np.polyval(p, zin)) ** 2))
+    for ch in trace:
+        lo_c, hi_c = c - kl * 0.05, c + kr * 0.05
+        if hi_c > z[-1]:
+            want = "L"
+        elif lo_c <= z[0]:
+            want = "R"
+        else:
+            el, er = mse(c - (kl + 1) * 0.05, hi_c), mse(lo_c, c + (kr + 1) * 0.05)
+            want = "L" if el < er else "R"
+            if abs(el - er) <= 1e-9 * max(el, er):
+                want = ch                                  # a near-tie may go either way in another summation order
+        assert ch == want
+        kl, kr = kl + (ch == "L"), kr + (ch == "R")
+    # closed form: ReLU on positive samples has zero error on both sides at every step, ties go right, and once the range
+    # has passed the largest sample the left side is taken: R ... R L ... L
+    zp = np.linspace(1.0, 3.0, 41)
+    lo, hi, trace, _ = O.greedy_range_search(zp, 0.9, 0.25, O.ACT_RELU, return_trace=True)
+    s = "".join(trace)
+    assert s == "R" * s.count("R") + "L" * s.count("L") and s.count("R") >= 1
+    assert hi > zp[-1] and ((zp >= lo) & (zp < hi)).mean() >= 0.9
+
+
+def test_neuron_thresholds_against_library_lp():
+    from scipy.optimize import linprog
+    rng = np.random.default_rng(10)
+    err = rng.uniform(0.1, 2.0, size=12)
+    t = O.neuron_thresholds(err, 0.8, 0.6, 0.95)
+    assert t.sum() == pytest.approx(0.8 * 12) and t.min() >= 0.6 - 1e-12 and t.max() <= 0.95 + 1e-12
+    lp = linprog(err, A_eq=np.ones((1, 12)), b_eq=[0.8 * 12], bounds=[(0.6, 0.95)] * 12)
+    assert float(err @ t) == pytest.approx(lp.fun, rel=1e-9)
+    np.testing.assert_allclose(t, lp.x, atol=1e-7)
+    # the neurons with the largest error keep the lowest threshold
+    assert t[np.argmax(err)] == 0.6 and t[np.argmin(err)] == 0.95
