@@ -424,6 +424,12 @@ def main():
         msk = timed(lambda: T.tardis_calibrate(zcal, Lf.b1, cfg.q_lo, cfg.q_hi, cfg.act), 5, 1)
         out["calibrate_context"] = {"ms_per_layer": msc, "ms_ranges_and_fits": msk, "n_cal": ncal,
                                     "what": "z = W1 Xcal^T (tcgen05 GEMM) + quantile ranges + least-squares fits, 16384 neurons"}
+        # Algorithm 1's greedy range search (KDE centroid + expansion by the smaller regression error) on the same samples
+        T.tardis_range_search(zcal, Lf.b1, 0.85, 0.05, cfg.act)
+        msr = timed(lambda: T.tardis_range_search(zcal, Lf.b1, 0.85, 0.05, cfg.act), 2, 1)
+        out["range_search_context"] = {"ms_per_layer": msr, "n_cal": ncal, "threshold": 0.85, "step": 0.05,
+                                       "what": "Algorithm 1 per neuron on the GPU, %d neurons; the paper reports about 30 minutes per "
+                                               "layer for its search (Section 7.3, RTX 4090D)" % h}
         del Lf, xcal, zcal
 
         def dense_step():

@@ -210,6 +210,24 @@ tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, in
                                  double q_lo, double q_hi, int32_t act, float* lo, float* hi, float* a, float* c,
                                  tardis_stream_t stream);
 
+/* The range search of Algorithm 1 (Section 5.1.1, "Range Searching") for every neuron of one layer, from the same
+ * calibration pre-activations as tardis_calibrate: the range starts empty at the centroid of the neuron's samples (the
+ * sample with the highest Gaussian kernel density estimate; kernel width 1.06 std n_cal^(-1/5), the paper names neither
+ * kernel nor width) and grows by `step` at a time on the side whose grown range has the smaller approximation error (mean
+ * squared residual of the least-squares line over the samples inside; the right side on a tie; a side that has passed the
+ * outermost sample is not grown) until the share of the samples with lo <= z < hi reaches the neuron's threshold; then the
+ * line of the final range is fitted as in tardis_calibrate.  The listing's left candidate reads (R.left - s, R.left);
+ * it is taken as (R.left - s, R.right).  Bounds are centroid - k_left step and centroid + k_right step, evaluated in
+ * double precision and stored in single.
+ *   thresholds   device [d_ff] float, the per-neuron coverage t of Section 5.1.1's neuron-level thresholds, or NULL: then
+ *                every neuron uses `threshold`
+ *   steps_taken  device [d_ff] int32 or NULL: number of growth steps per neuron
+ * 1 <= n_cal <= 2048 (TARDIS_ERR_UNSUPPORTED beyond), step > 0, thresholds in [0, 1].  Other arguments as in
+ * tardis_calibrate.  Asynchronous on `stream`; allocates nothing; nothing is kept. */
+tardis_status_t tardis_range_search(int32_t d_ff, int32_t n_cal, const float* z, int64_t ldz, const float* b1,
+                                    const float* thresholds, double threshold, double step, int32_t act, float* lo, float* hi,
+                                    float* a, float* c, int32_t* steps_taken, tardis_stream_t stream);
+
 /* Chooses the kernel path: 0 = automatic (default), 1 = always the generic
  * kernels, 2 = the fused decode kernel for every token count up to 4096 (in
  * launches of at most 4 tokens; layers it does not serve fall back as in 0),

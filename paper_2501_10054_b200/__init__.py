@@ -22,7 +22,7 @@ TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_calibrate",
-           "tardis_debug_phase_stamps", "tardis_status_string", "tardis_last_error"]
+           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_status_string", "tardis_last_error"]
 
 
 class TardisError(RuntimeError):
@@ -76,7 +76,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_gemm_bf16.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, i32, vp]
     lib.tardis_calibrate.argtypes = [i32, i32, vp, i64, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp]
     lib.tardis_debug_phase_stamps.argtypes = [vp, i32]
-    for name in EXPORTS[:11]:
+    lib.tardis_range_search.argtypes = [i32, i32, vp, i64, vp, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp, vp]
+    for name in EXPORTS[:12]:
         getattr(lib, name).restype = ctypes.c_int
     lib.tardis_status_string.argtypes = [ctypes.c_int]
     lib.tardis_status_string.restype = ctypes.c_char_p
@@ -171,6 +172,23 @@ def tardis_calibrate(z: torch.Tensor, b1: Optional[torch.Tensor], q_lo: float, q
                                            out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), out[3].data_ptr(),
                                            _stream(stream)), "tardis_calibrate")
     return tuple(out)
+
+
+def tardis_range_search(z: torch.Tensor, b1: Optional[torch.Tensor], threshold, step: float, act: int, stream=None, want_steps=False):
+    """Algorithm 1's greedy range search per neuron from calibration pre-activations z[d_ff, n_cal] (float32, CUDA, unit
+    inner stride, n_cal <= 2048): returns (lo, hi, a, c) (and the step counts with want_steps).  `threshold` is a float
+    (one coverage for all neurons) or a float32 CUDA tensor of d_ff per-neuron thresholds."""
+    if z.dtype != torch.float32 or not z.is_cuda or z.stride(1) != 1:
+        raise TardisError(1, "z must be a float32 CUDA tensor with unit inner stride")
+    h, n = z.shape
+    out = [torch.empty(h, dtype=torch.float32, device=z.device) for _ in range(4)]
+    steps = torch.zeros(h, dtype=torch.int32, device=z.device) if want_steps else None
+    thr_t = threshold if isinstance(threshold, torch.Tensor) else None
+    _check(load_library().tardis_range_search(h, n, z.data_ptr(), z.stride(0), _ptr(b1), _ptr(thr_t),
+                                              0.0 if thr_t is not None else float(threshold), float(step), int(act),
+                                              out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), out[3].data_ptr(),
+                                              _ptr(steps), _stream(stream)), "tardis_range_search")
+    return tuple(out) + ((steps,) if want_steps else ())
 
 
 def tardis_stats(handle: int) -> dict:

@@ -200,6 +200,16 @@ tardis_status_t tardis_calibrate(int32_t d_ff, int32_t n_cal, const float* z, in
   return launch_calibrate(d_ff, n_cal, z, ldz, b1, q_lo, q_hi, act, lo, hi, a, c, reinterpret_cast<cudaStream_t>(stream));
 }
 
+tardis_status_t tardis_range_search(int32_t d_ff, int32_t n_cal, const float* z, int64_t ldz, const float* b1, const float* thresholds,
+                                    double threshold, double step, int32_t act, float* lo, float* hi, float* a, float* c,
+                                    int32_t* steps_taken, tardis_stream_t stream) {
+  if (d_ff <= 0 || n_cal <= 0 || !z || ldz < n_cal || !lo || !hi || !a || !c) return TARDIS_ERR_INVALID_ARG;
+  if (!(step > 0.0) || (!thresholds && !(threshold >= 0.0 && threshold <= 1.0))) return TARDIS_ERR_INVALID_ARG;
+  if (act != TARDIS_ACT_GELU_TANH && act != TARDIS_ACT_GELU_ERF && act != TARDIS_ACT_RELU) return TARDIS_ERR_INVALID_ARG;
+  return launch_range_search(d_ff, n_cal, z, ldz, b1, thresholds, threshold, step, act, lo, hi, a, c, steps_taken,
+                             reinterpret_cast<cudaStream_t>(stream));
+}
+
 tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
   Handle* H = check(handle);
   if (!H || !out) return TARDIS_ERR_INVALID_ARG;

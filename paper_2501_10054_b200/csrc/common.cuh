@@ -96,6 +96,9 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 tardis_status_t launch_calibrate(int h, int n, const float* z, long long ldz, const float* b1, double q_lo, double q_hi, int act,
                                  float* lo, float* hi, float* a, float* c, cudaStream_t s);
 
+tardis_status_t launch_range_search(int h, int n, const float* z, long long ldz, const float* b1, const float* thr, double t_all,
+                                    double step, int act, float* lo, float* hi, float* a, float* c, int* steps_out, cudaStream_t s);
+
 // the activation (the name is historical: ReLU is served too)
 __device__ __forceinline__ float gelu_f32(float z, int act) {
   if (act == TARDIS_ACT_RELU) return z > 0.f ? z : 0.f * z;      // 0 * z keeps NaN a NaN

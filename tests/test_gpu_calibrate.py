@@ -115,3 +115,98 @@ def test_full_size_layer_sampled_neurons():
     inside = ((zb >= lo[:, None]) & (zb < hi[:, None])).float().mean(1)
     assert bool((lo < hi).all()) and float((inside - 0.9).abs().max()) < 2e-3
     assert bool(torch.isfinite(a).all()) and bool(torch.isfinite(c).all())
+
+
+# ------------------------------------------------------------------ Algorithm 1: the greedy range search
+def _check_search(z, b1, thr, step, act, thr_tensor=None):
+    """tardis_range_search against the oracle, neuron by neuron.  The ranges must be the same float32 numbers; a neuron
+    whose search met a near-tie (the two candidate errors within 1e-7 of each other, or two samples with kernel densities
+    within 1e-9) may legitimately go the other way under a different summation order: those are counted, and for them the
+    result only has to be a valid outcome (coverage reached, not reached one step earlier)."""
+    res = T.tardis_range_search(z, b1, thr_tensor if thr_tensor is not None else thr, step, act, want_steps=True)
+    torch.cuda.synchronize()
+    lo, hi, a, c, steps = [r.cpu().numpy() for r in res]
+    zc = z.cpu().numpy()
+    if b1 is not None:
+        zc = zc + b1.cpu().numpy()[:, None]
+    h, n = zc.shape
+    ties = 0
+    for j in range(h):
+        t = float(thr_tensor[j]) if thr_tensor is not None else thr
+        lo_r, hi_r, trace, margin = O.greedy_range_search(zc[j], t, step, act, return_trace=True)
+        same = np.float32(lo_r) == lo[j] and np.float32(hi_r) == hi[j] and steps[j] == len(trace)
+        if not same:
+            zs = np.sort(zc[j].astype(np.float64))
+            bw = 1.06 * np.std(zs, ddof=1) * n ** -0.2
+            dens = np.array([np.exp(-0.5 * ((zs - v) / bw) ** 2).sum() for v in zs]) if bw > 0 else np.ones(n)
+            top = np.sort(dens)[-2:]
+            near = margin < 1e-7 or (top[1] - top[0]) <= 1e-9 * top[1]
+            assert near, "neuron %d: GPU range (%r, %r) after %d steps, oracle (%r, %r) after %d, margin %.3e" % (
+                j, lo[j], hi[j], steps[j], lo_r, hi_r, len(trace), margin)
+            ties += 1
+            inside = ((zc[j] >= lo[j]) & (zc[j] < hi[j])).mean()
+            assert inside >= t - 1e-12
+        # the line of the final range, from the float32 bounds the kernel stored
+        a_ref, c_ref = O.least_squares_fit(zc[j:j + 1], lo[j:j + 1], hi[j:j + 1], act)
+        assert abs(float(a[j]) - float(a_ref[0])) <= 2e-6 * max(1.0, abs(float(a_ref[0])))
+        assert abs(float(c[j]) - float(c_ref[0])) <= 2e-6 * max(1.0, abs(float(c_ref[0])))
+    return ties
+
+
+@pytest.mark.parametrize("act", [W.ACT_GELU_TANH, W.ACT_RELU])
+@pytest.mark.parametrize("shape", [(48, 64), (24, 257), (12, 1000)])
+def test_greedy_range_search_matches_oracle(shape, act):
+    h, n = shape
+    g = torch.Generator().manual_seed(7 * h + n)
+    z = (torch.randn(h, n, generator=g) * torch.linspace(0.3, 2.0, h)[:, None] + torch.linspace(-1, 1, h)[:, None]).cuda()
+    b1 = (0.1 * torch.randn(h, generator=g)).cuda()
+    ties = _check_search(z, b1, 0.85, 0.05, act)
+    thr = torch.linspace(0.5, 0.97, h).cuda()
+    ties += _check_search(z, None, None, 0.1, act, thr_tensor=thr)
+    print("range search %s: %d near-ties among %d searches" % (shape, ties, 2 * h))
+    assert ties <= h // 4
+
+
+def test_greedy_range_search_edge_cases_and_errors():
+    lib = T.load_library()
+    # all samples equal, a single sample, threshold 0 (empty range at the centroid) and 1 (every sample)
+    z = torch.tensor([[0.3] * 16, list(np.cumsum(np.linspace(0.1, 0.4, 16)) - 2.0)], dtype=torch.float32).cuda()   # (no symmetric ties)
+    lo, hi, a, c = T.tardis_range_search(z, None, 1.0, 0.5, W.ACT_GELU_TANH)
+    torch.cuda.synchronize()
+    zc = z.cpu().numpy()
+    for j in range(2):
+        lo_r, hi_r = O.greedy_range_search(zc[j], 1.0, 0.5)
+        assert np.float32(lo_r) == lo[j].item() and np.float32(hi_r) == hi[j].item()
+        assert ((zc[j] >= lo[j].item()) & (zc[j] < hi[j].item())).all()
+    lo0, hi0, _, _ = T.tardis_range_search(z, None, 0.0, 0.5, W.ACT_GELU_TANH)
+    assert (lo0 == hi0).all()
+    one = torch.tensor([[1.25]], dtype=torch.float32).cuda()
+    lo1, hi1, _, _ = T.tardis_range_search(one, None, 0.9, 0.25, W.ACT_RELU)
+    assert lo1.item() == 1.25 and hi1.item() == 1.5
+    big = torch.zeros(2, 4096, device="cuda")
+    with pytest.raises(T.TardisError):
+        T.tardis_range_search(big, None, 0.9, 0.1, 0)          # more than 2048 samples: unsupported
+    p = z.data_ptr()
+    assert lib.tardis_range_search(2, 16, p, 16, None, None, 0.9, 0.0, 0, p, p, p, p, None, None) == 1   # step must be positive
+    assert lib.tardis_range_search(2, 16, p, 16, None, None, 1.5, 0.1, 0, p, p, p, p, None, None) == 1   # threshold outside [0, 1]
+
+
+def test_greedy_range_search_full_layer_shape_sampled():
+    """The 7B-class shape (16384 neurons x 2048 calibration tokens) runs whole on the GPU; the oracle checks a seeded sample."""
+    cfg = W.CONFIGS["decode_7b"]
+    dev = torch.device("cuda", 0)
+    L = W.make_layer(cfg, 5, device=dev)
+    xcal = W.make_tokens(cfg, 2048, 5, device=dev, tag="calib")
+    zcal = torch.empty(cfg.d_ff, 2048, dtype=torch.float32, device=dev)
+    T.tardis_gemm_bf16(L.W1, xcal, zcal)
+    lo, hi, a, c, steps = T.tardis_range_search(zcal, L.b1, 0.85, 0.05, cfg.act, want_steps=True)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(5)
+    rows = np.sort(rng.choice(cfg.d_ff, size=6, replace=False))
+    sel = torch.as_tensor(rows, device=dev)
+    zs = zcal[sel].contiguous()
+    ties = _check_search(zs, L.b1[sel].contiguous() if L.b1 is not None else None, 0.85, 0.05, cfg.act)
+    lo_s, hi_s, _, _ = T.tardis_range_search(zs, L.b1[sel].contiguous() if L.b1 is not None else None, 0.85, 0.05, cfg.act)
+    assert torch.equal(lo_s, lo[sel]) and torch.equal(hi_s, hi[sel])
+    cov = ((zcal + L.b1[:, None] >= lo[:, None]) & (zcal + L.b1[:, None] < hi[:, None])).float().mean(dim=1)
+    assert float(cov.min()) >= 0.85 - 1e-6 and float(cov.mean()) < 0.87
