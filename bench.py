@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--graph", type=int, default=0, help="replay one step as a CUDA graph")
     ap.add_argument("--no-context", action="store_true", help="skip the dense-FFN / batch-64 / oracle context legs")
     ap.add_argument("--cpu-sample-tokens", type=int, default=16)
-    ap.add_argument("--mode", default="decode", choices=["decode", "prefill"],
+    ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "studies"],
                     help="prefill: time one prefill chunk of one layer through the batched path (a context run, not the headline)")
     ap.add_argument("--prefill-tokens", type=int, default=8192)
     return ap.parse_args()
@@ -194,6 +194,9 @@ def main():
     cfg = W.CONFIGS[args.workload]
     if args.mode == "prefill":
         run_prefill(args, cfg, T, W, torch, dev, rank, world)
+        return
+    if args.mode == "studies":
+        run_studies(args, T, W, torch, dev)
         return
     d, h, B, NT = cfg.d_model, cfg.d_ff, args.batch, args.tokens
     assert NT % B == 0
@@ -530,6 +533,73 @@ def run_prefill(args, cfg, T, W, torch, dev, rank, world):
                          "kernel": "k_gemm (4 products per chunk: scores hi+lo, folded, pre-activations, output)",
                          "flops_per_step": flops}}))
     T.tardis_destroy(hd)
+
+
+def run_studies(args, T, W, torch, dev):
+    """Two small studies on synthetic layers, after Sections 7.6 and 7.7 of the paper (context numbers, not the headline):
+    (1) predictor size: flag precision and recall of the 2-, 4- and 8-bit predictors against the flags taken on the true
+        pre-activations (the exact-range mode), on the 7B-class decode layer;
+    (2) precision of the reordered product: error of the folded matrix against the fp64 oracle for three kinds of
+        intermediate (leading bf16 term only, exact two-term bf16 split = the default, plain fp32), at two layer sizes."""
+    import dataclasses
+    import numpy as np
+    from oracle import tardis_oracle as O
+    from tests import helpers as Hp
+    out = {"mode": "studies", "data": "synthetic"}
+    base = W.CONFIGS["decode_7b"]
+    x = W.make_tokens(base, 64, seed=3, device=dev)
+    sweep = {}
+    for bits in (2, 4, 8):
+        cfg = dataclasses.replace(base, bits=bits)
+        L = W.make_layer(cfg, seed=11, device=dev)
+        hd = T.fold_layer(L)
+        y = torch.empty_like(x)
+        flags = {}
+        for name, path in (("predictor", 0), ("exact", 4)):
+            T.tardis_set_path(hd, path)
+            bm = torch.zeros(64, cfg.d_ff // 32, dtype=torch.int32, device=dev)
+            T.tardis_set_debug_capture(hd, bm, None)
+            for t in range(64):
+                T.tardis_set_debug_capture(hd, bm[t:t + 1], None)
+                T.tardis_ffn_forward(hd, x[t:t + 1], y[t:t + 1])
+            torch.cuda.synchronize()
+            T.tardis_set_debug_capture(hd, None, None)
+            flags[name] = Hp.unpack_bitmap(bm, cfg.d_ff)
+        P, E = flags["predictor"], flags["exact"]
+        tp = float((P & E).sum())
+        sweep["bits%d" % bits] = {"flagged_frac_predictor": float(P.mean()), "flagged_frac_exact": float(E.mean()),
+                                  "precision": tp / max(1.0, float(P.sum())), "recall": tp / max(1.0, float(E.sum())),
+                                  "predictor_bytes": cfg.d_ff * cfg.d_model * bits // 8}
+        T.tardis_destroy(hd)
+        del L
+        torch.cuda.empty_cache()
+    out["predictor_size"] = {"what": "flags of the quantised predictor against flags from the true pre-activations, 64 tokens, "
+                                     "decode_7b shape (ranges tuned for about 10 % flagged with the 2-bit predictor)", **sweep}
+    fold = {}
+    for name, d, h in (("x1", 2048, 8192), ("x4", 4096, 16384)):
+        cfg = W.LayerConfig("fold_" + name, d, h, n_calib=1024, group=128)
+        L = W.make_layer(cfg, seed=21, device=dev)
+        s = L.numpy64()
+        rng = np.random.default_rng(21)
+        rows = np.sort(rng.choice(d, size=16, replace=False))
+        ref = O.fold_rows(rows, s["W1"], s["W2"], s["a"])
+        scale2 = float((ref ** 2).mean())
+        res = {}
+        for mode, flag in (("bf16_intermediate", 1), ("bf16_two_terms_default", 0), ("fp32_plain", 2)):
+            hd = T.fold_layer(L, flags=flag)
+            Wf = torch.empty(d, d, dtype=torch.bfloat16, device=dev)
+            T.tardis_export_folded(hd, Wf, None)
+            torch.cuda.synchronize()
+            got = Wf[torch.as_tensor(rows, device=dev)].double().cpu().numpy()
+            res[mode] = {"mse": float(((got - ref) ** 2).mean()), "relative_mse": float(((got - ref) ** 2).mean()) / scale2}
+            T.tardis_destroy(hd)
+        rounded = torch.as_tensor(ref).to(torch.bfloat16).double().numpy()
+        res["bf16_rounding_floor"] = {"mse": float(((rounded - ref) ** 2).mean()), "relative_mse": float(((rounded - ref) ** 2).mean()) / scale2}
+        fold[name] = dict(res, d_model=d, d_ff=h)
+        del L
+        torch.cuda.empty_cache()
+    out["fold_precision"] = {"what": "mean squared error of 16 sampled rows of W_f (stored in bf16) against the fp64 oracle", **fold}
+    print(json.dumps(out))
 
 
 class _Null:

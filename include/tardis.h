@@ -74,8 +74,16 @@ typedef struct {
                                  pred_bits*(k%p) upwards                                  */
   const void* pred_scale;     /* device [d_ff, d_model/G], type `dtype`                   */
   const uint8_t* pred_zero;   /* device [d_ff, d_model/G], integer zero-point 0..2^pred_bits-1 */
-  uint32_t flags;             /* reserved, 0                                              */
+  uint32_t flags;             /* 0, or one of the TARDIS_FOLD_* study modes below          */
 } tardis_fold_desc_t;
+
+/* Study modes of the fold for bf16 layers (tardis_fold_desc_t.flags), after the paper's look at the precision of
+ * the reordered product (Section 7.7): 0 folds through the tensor cores with diag(a) W1 held as the exact sum of two
+ * bf16 matrices and fp32 accumulation (the default); TARDIS_FOLD_BF16_INTERMEDIATE keeps only the leading bf16 term
+ * of diag(a) W1 (the "bf16 intermediate" row of the paper's table); TARDIS_FOLD_FP32_PLAIN computes the product with
+ * plain fp32 arithmetic from the fp32 values of a W1 (no tensor cores).  All three round W_f to bf16 once at the end. */
+#define TARDIS_FOLD_BF16_INTERMEDIATE 1u
+#define TARDIS_FOLD_FP32_PLAIN 2u
 
 /* Counters and sizes.  Byte counts are the resident state of the handle,
  * following the paper's footprint components: folded matrix + bias, predictor,

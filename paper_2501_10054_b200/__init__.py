@@ -119,12 +119,12 @@ def _dtype_code(dt: torch.dtype) -> int:
 
 
 def tardis_fold(W1, W2, lo, hi, a, c, pred_codes, pred_scale, pred_zero, pred_group, b1=None, b2=None,
-                act=TARDIS_ACT_GELU_TANH, pred_bits=2, stream=None) -> int:
+                act=TARDIS_ACT_GELU_TANH, pred_bits=2, stream=None, flags=0) -> int:
     """tardis_fold of the C ABI.  Returns the opaque handle (an integer)."""
     lib = load_library()
     h, d = W1.shape
     desc = FoldDesc(d, h, _dtype_code(W1.dtype), act, _ptr(W1), _ptr(W2), _ptr(b1), _ptr(b2), _ptr(lo), _ptr(hi),
-                    _ptr(a), _ptr(c), pred_bits, pred_group, _ptr(pred_codes), _ptr(pred_scale), _ptr(pred_zero), 0)
+                    _ptr(a), _ptr(c), pred_bits, pred_group, _ptr(pred_codes), _ptr(pred_scale), _ptr(pred_zero), flags)
     out = ctypes.c_void_p()
     _check(lib.tardis_fold(ctypes.byref(desc), _stream(stream), ctypes.byref(out)), "tardis_fold")
     return out.value
@@ -223,9 +223,9 @@ def tardis_destroy(handle: int):
     _check(load_library().tardis_destroy(handle), "tardis_destroy")
 
 
-def fold_layer(layer, stream=None) -> int:
+def fold_layer(layer, stream=None, flags=0) -> int:
     """Convenience: tardis_fold from an object with the fields W1, W2, b1, b2, lo, hi, a, c, codes, scale,
     zero and cfg.group / cfg.act / cfg.bits (all CUDA tensors)."""
     return tardis_fold(layer.W1, layer.W2, layer.lo, layer.hi, layer.a, layer.c, layer.codes, layer.scale,
                        layer.zero, layer.cfg.group, b1=layer.b1, b2=layer.b2, act=layer.cfg.act,
-                       pred_bits=layer.cfg.bits, stream=stream)
+                       pred_bits=layer.cfg.bits, stream=stream, flags=flags)

@@ -69,7 +69,7 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   if (d <= 0 || h <= 0 || G <= 0) return TARDIS_ERR_INVALID_ARG;
   if (desc->dtype != TARDIS_F32 && desc->dtype != TARDIS_BF16) return TARDIS_ERR_INVALID_ARG;
   if (desc->act != TARDIS_ACT_GELU_TANH && desc->act != TARDIS_ACT_GELU_ERF && desc->act != TARDIS_ACT_RELU) return TARDIS_ERR_INVALID_ARG;
-  if (desc->flags != 0) return TARDIS_ERR_INVALID_ARG;
+  if (desc->flags > TARDIS_FOLD_FP32_PLAIN) return TARDIS_ERR_INVALID_ARG;
   if (d % 8 || h % 32 || G % 16 || d % G) return TARDIS_ERR_INVALID_ARG;
   if (desc->pred_bits != 2 && desc->pred_bits != 4 && desc->pred_bits != 8)
     return desc->pred_bits > 0 && desc->pred_bits <= 8 ? TARDIS_ERR_UNSUPPORTED : TARDIS_ERR_INVALID_ARG;
@@ -116,8 +116,8 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
 
   const bool bf16 = H->dtype == TARDIS_BF16;
   if (bf16) st = batched_prepare(H);                          // allocations; its buffers double as fold temporaries
-  const bool tensor_fold = st == TARDIS_OK && bf16 && H->bstate != nullptr;
-  if (st == TARDIS_OK) st = launch_fold(H, desc, s, tensor_fold);
+  const bool tensor_fold = st == TARDIS_OK && bf16 && H->bstate != nullptr && desc->flags != TARDIS_FOLD_FP32_PLAIN;
+  if (st == TARDIS_OK) st = launch_fold(H, desc, s, tensor_fold);   // (computes the product itself when tensor_fold is false)
   if (st == TARDIS_OK && tensor_fold) {
     st = launch_fold_tensor(H, desc, s);
     if (st == TARDIS_ERR_UNSUPPORTED) st = launch_fold_product(H, s);   // no tensor-map support: plain kernel

@@ -255,7 +255,7 @@ tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cu
   for (int i0 = 0; i0 < d; i0 += rows_per) {
     const int rows = d - i0 < rows_per ? d - i0 : rows_per;
     GemmArgs g = {};
-    g.M = rows; g.N = d; g.K1 = h; g.K2 = h;
+    g.M = rows; g.N = d; g.K1 = h; g.K2 = desc->flags == TARDIS_FOLD_BF16_INTERMEDIATE ? 0 : h;   // (study mode: leading term only)
     g.A1 = static_cast<const __nv_bfloat16*>(desc->W2) + size_t(i0) * h; g.lda1 = h; g.B1 = S->What_hi; g.ldb1 = h;
     g.A2 = g.A1; g.lda2 = h; g.B2 = S->What_lo; g.ldb2 = h;
     g.epilogue = GEMM_EPI_F32; g.out_f32 = S->zhat; g.ldo = d; g.error_word = &H->counters[CTR_ERROR];

@@ -66,7 +66,7 @@ def test_invalid_arguments_return_status_before_any_launch(lib):
     assert status(W1=24) == 1                 # misaligned
     assert status(pred_bits=3) == 2           # valid but not built (2, 4 and 8 are)
     assert status(pred_bits=0) == 1
-    assert status(flags=1) == 1
+    assert status(flags=7) == 1               # beyond the fold study modes
     assert out.value is None
     assert lib.tardis_ffn_forward(None, 16, 16, 1, None) == 1
     assert lib.tardis_stats(None, None) == 1
