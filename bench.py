@@ -209,7 +209,10 @@ def main():
         dense.append((L.W1, L.W2, L.b1, L.b2))
         if l == 0 and rank == 0 and not args.no_context:
             layer0_64 = L.numpy64()
-    x_all = W.make_tokens(cfg, NT, seed=rank, device=dev)
+    # every rank takes its contiguous share of one seeded token stream (tokens are independent: no exchange is needed)
+    from paper_2501_10054_b200 import sharding
+    first, count = sharding.token_shard(NT * world, world, rank)
+    x_all = W.make_tokens(cfg, NT * world, seed=0, device=dev)[first:first + count].contiguous()
     y_all = torch.empty_like(x_all)
     torch.cuda.synchronize()
     touched = algorithmic_bytes(cfg, B, int(0.1 * h))

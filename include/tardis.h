@@ -259,6 +259,15 @@ tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
  * and its kernel carries no stamps.  Errors: INVALID_ARG (NULL, max_ctas <= 0), UNSUPPORTED, CUDA. */
 tardis_status_t tardis_debug_phase_stamps(long long* stamps, int32_t max_ctas);
 
+/* Every wait inside the kernels (on a bulk copy's barrier) is bounded: when the limit runs out the kernel records it in
+ * the handle's device error word, skips the work that needed the data and returns; tardis_stats then reports
+ * TARDIS_ERR_TIMEOUT until the word is cleared.  tardis_debug_wait_timeout makes exactly that happen on purpose, for
+ * testing the reporting path without any fault: it launches one warp that waits, for at most limit_cycles SM clock
+ * cycles (0 .. 2e9), on a barrier whose bytes never arrive.  tardis_clear_error synchronises the handle's last stream and
+ * resets the error word.  (The paper has no counterpart of these two calls.)  Errors: INVALID_ARG, CUDA. */
+tardis_status_t tardis_debug_wait_timeout(tardis_handle_t handle, int64_t limit_cycles, tardis_stream_t stream);
+tardis_status_t tardis_clear_error(tardis_handle_t handle);
+
 /* Frees everything the handle owns (synchronises the device first). */
 tardis_status_t tardis_destroy(tardis_handle_t handle);
 

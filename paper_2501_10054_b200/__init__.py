@@ -22,7 +22,8 @@ TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_calibrate",
-           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_status_string", "tardis_last_error"]
+           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_debug_wait_timeout", "tardis_clear_error",
+           "tardis_status_string", "tardis_last_error"]
 
 
 class TardisError(RuntimeError):
@@ -77,7 +78,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_calibrate.argtypes = [i32, i32, vp, i64, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp]
     lib.tardis_debug_phase_stamps.argtypes = [vp, i32]
     lib.tardis_range_search.argtypes = [i32, i32, vp, i64, vp, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp, vp]
-    for name in EXPORTS[:12]:
+    lib.tardis_debug_wait_timeout.argtypes = [vp, i64, vp]
+    lib.tardis_clear_error.argtypes = [vp]
+    for name in EXPORTS[:14]:
         getattr(lib, name).restype = ctypes.c_int
     lib.tardis_status_string.argtypes = [ctypes.c_int]
     lib.tardis_status_string.restype = ctypes.c_char_p
@@ -217,6 +220,15 @@ def tardis_debug_phase_stamps(max_ctas: int = 512):
     buf = np.zeros((max_ctas, 16), dtype=np.int64)
     _check(load_library().tardis_debug_phase_stamps(buf.ctypes.data, max_ctas), "tardis_debug_phase_stamps")
     return buf
+
+
+def tardis_debug_wait_timeout(handle: int, limit_cycles: int, stream=None):
+    """Launches one warp whose bounded wait runs out after limit_cycles SM cycles (testing aid for the time-out report)."""
+    _check(load_library().tardis_debug_wait_timeout(handle, int(limit_cycles), _stream(stream)), "tardis_debug_wait_timeout")
+
+
+def tardis_clear_error(handle: int):
+    _check(load_library().tardis_clear_error(handle), "tardis_clear_error")
 
 
 def tardis_destroy(handle: int):

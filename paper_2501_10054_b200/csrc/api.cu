@@ -253,6 +253,24 @@ tardis_status_t tardis_debug_phase_stamps(long long* stamps, int32_t max_ctas) {
   return fused_read_stamps(stamps, max_ctas);
 }
 
+tardis_status_t tardis_debug_wait_timeout(tardis_handle_t handle, int64_t limit_cycles, tardis_stream_t stream) {
+  Handle* H = check(handle);
+  if (!H || limit_cycles < 0 || limit_cycles > 2000000000ll) return TARDIS_ERR_INVALID_ARG;
+  if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  H->last_stream = s;
+  return launch_wait_that_runs_out(H, limit_cycles, s);
+}
+
+tardis_status_t tardis_clear_error(tardis_handle_t handle) {
+  Handle* H = check(handle);
+  if (!H) return TARDIS_ERR_INVALID_ARG;
+  if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
+  TARDIS_CUDA_TRY(cudaStreamSynchronize(H->last_stream));
+  TARDIS_CUDA_TRY(cudaMemset(H->counters + CTR_ERROR, 0, sizeof(unsigned long long)));
+  return TARDIS_OK;
+}
+
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path) {
   Handle* H = check(handle);
   if (!H || !(path >= 0 && path <= 4)) return TARDIS_ERR_INVALID_ARG;

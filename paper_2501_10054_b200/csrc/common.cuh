@@ -77,7 +77,8 @@ tardis_status_t decode_read_stamps(long long* out, int max_ctas);
 tardis_status_t fused_prepare(Handle* H, cudaStream_t s);                  // builds the state of fused.cu (bf16, d_model <= 4608)
 tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
 void fused_release(Handle* H);
-tardis_status_t fused_read_stamps(long long* out, int max_ctas);   // UNSUPPORTED unless built with TARDIS_PHASE_STAMPS
+tardis_status_t fused_read_stamps(long long* out, int max_ctas);
+tardis_status_t launch_wait_that_runs_out(Handle* H, long long limit_cycles, cudaStream_t s);   // UNSUPPORTED unless built with TARDIS_PHASE_STAMPS
 tardis_status_t batched_prepare(Handle* H);                                                   // bf16 only: allocations
 tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);    // fills the batched state
 tardis_status_t launch_batched_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);

@@ -1092,6 +1092,26 @@ tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, c
   return TARDIS_OK;
 }
 
+// A bounded wait that runs out, on purpose and without any fault: one warp arms a barrier for bytes that no copy will ever
+// deliver, waits with the given limit, and records the time-out in the handle's error word exactly as the kernels do.
+__global__ void k_wait_that_runs_out(long long limit_cycles, unsigned long long* counters) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    fz::mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fz::mbar_expect_tx(&bar, 16u);
+  }
+  __syncwarp();
+  const bool landed = fz::mbar_wait_warp(&bar, 0u, limit_cycles);
+  if (!landed && threadIdx.x == 0) atomicExch(&counters[CTR_ERROR], 1ull);
+}
+
+tardis_status_t launch_wait_that_runs_out(Handle* H, long long limit_cycles, cudaStream_t s) {
+  k_wait_that_runs_out<<<1, 32, 0, s>>>(limit_cycles, H->counters);
+  TARDIS_CUDA_TRY(cudaGetLastError());
+  return TARDIS_OK;
+}
+
 tardis_status_t fused_read_stamps(long long* out, int max_ctas) {
 #ifdef TARDIS_PHASE_STAMPS
   const int n = max_ctas < kStampCtas ? max_ctas : kStampCtas;

@@ -1,6 +1,8 @@
 """GPU parity: the CUDA library (through its C ABI) against the fp64 oracle on the same seeded
 inputs.  Flags bit-exact outside the 1e-6 score band; outputs within 1e-5 (fp32) / 2e-2 (bf16)
 max relative error |dy| / max(|y_ref|, rms(y_ref[t,:]))."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -238,3 +240,26 @@ def test_batched_path_chunk_boundary_nan_token_and_empty_ranges():
         assert bool(ok.all())
     finally:
         T.tardis_destroy(h)
+
+
+def test_bounded_wait_runs_out_is_reported_and_cleared():
+    """A device-side wait whose data never arrives ends by its limit, sets the error word (no trap, no hang: the kernel
+    returns normally), tardis_stats reports the time-out, and after tardis_clear_error the handle works as before."""
+    cfg = W.LayerConfig("timeout", 256, 1024, n_calib=256)
+    L = _layer(cfg)
+    s = L.numpy64()
+    x = W.make_tokens(cfg, 3, 4).cuda()
+    h = T.fold_layer(L)
+    lib = T.load_library()
+    y0, F0, _ = Hp.gpu_forward(h, L, x, [3])
+    assert lib.tardis_debug_wait_timeout(h, 200000, None) == 0          # about 0.1 ms of waiting
+    st = T.Stats()
+    assert lib.tardis_stats(h, ctypes.byref(st)) == 5                   # TARDIS_ERR_TIMEOUT
+    assert st.device_error == 1
+    assert lib.tardis_clear_error(h) == 0
+    assert lib.tardis_stats(h, ctypes.byref(st)) == 0 and st.device_error == 0
+    y1, F1, _ = Hp.gpu_forward(h, L, x, [3])
+    assert (F0 == F1).all()
+    Hp.assert_parity(L, s, x, y1, F1, None, score_tol=None, label="after a cleared time-out")
+    assert lib.tardis_debug_wait_timeout(h, -1, None) == 1
+    T.tardis_destroy(h)
