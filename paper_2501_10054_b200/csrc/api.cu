@@ -249,8 +249,20 @@ tardis_status_t tardis_export_folded(tardis_handle_t handle, void* Wf, float* bf
 
 tardis_status_t tardis_debug_phase_stamps(long long* stamps, int32_t max_ctas) {
   if (!stamps || max_ctas <= 0) return TARDIS_ERR_INVALID_ARG;
-  // the table of the kernel that ran last is the one with the later entry stamps; both are cheap to read
-  return fused_read_stamps(stamps, max_ctas);
+  // both fused kernels keep a table; the one whose kernel ran last holds the later entry stamps
+  tardis_status_t st = fused_read_stamps(stamps, max_ctas);
+  if (st != TARDIS_OK) return st;
+  const size_t count = size_t(max_ctas < 512 ? max_ctas : 512) * 16;
+  long long* other = new (std::nothrow) long long[count];
+  if (!other) return TARDIS_ERR_ALLOC;
+  st = decode_read_stamps(other, max_ctas);
+  if (st == TARDIS_OK) {
+    long long ma = 0, mb = 0;
+    for (size_t i = 0; i < count; i += 16) { if (stamps[i] > ma) ma = stamps[i]; if (other[i] > mb) mb = other[i]; }
+    if (mb > ma) memcpy(stamps, other, count * sizeof(long long));
+  }
+  delete[] other;
+  return st;
 }
 
 tardis_status_t tardis_debug_wait_timeout(tardis_handle_t handle, int64_t limit_cycles, tardis_stream_t stream) {

@@ -599,8 +599,10 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
           const int e = atomicAdd(const_cast<int*>(&misc[MS_NRC]), 1);
           if (e < MAXRC) { rc[e] = (tl << 16) | r; f = -1; }
           else {                                        // list full: this thread re-evaluates its neuron alone
-            zhat = b1 + (resident ? exact_from_blocks(pbuf + size_t(tile) * p.buf_bytes, p.pbs, G, rr, xh + t * XS, d, 0, 1)
-                                  : exact_score_single(p.codes, p.scale, p.zero, xh + t * XS, j, d, G, 2));
+            const int qu = pass * NU + tile;            // the tile's blocks are still in shared memory unless its buffer was refilled
+            const bool here = resident || qu + p.nbuf >= NQ;
+            zhat = b1 + (here ? exact_from_blocks(pbuf + size_t(resident ? tile : qu % p.nbuf) * p.buf_bytes, p.pbs, G, rr, xh + t * XS, d, 0, 1)
+                              : exact_score_single(p.codes, p.scale, p.zero, xh + t * XS, j, d, G, 2));
             f = ((lo <= zhat) && (zhat < hi)) ? 0 : 1;
           }
         }
@@ -615,8 +617,9 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
           const int tl = rc[e] >> 16, r = rc[e] & 0xffff, t = t0 + tl;
           const int j = plan.x * 16 + r;
           double ex;
-          if (resident) {                       // the tile's blocks are still in shared memory
-            ex = exact_from_blocks(pbuf + size_t(r >> 4) * p.buf_bytes, p.pbs, G, r & 15, xh + t * XS, d, lane, 32);
+          const int qu = pass * NU + (r >> 4);
+          if (resident || qu + p.nbuf >= NQ) {  // the tile's blocks are still in shared memory (its buffer was not refilled)
+            ex = exact_from_blocks(pbuf + size_t(resident ? (r >> 4) : qu % p.nbuf) * p.buf_bytes, p.pbs, G, r & 15, xh + t * XS, d, lane, 32);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) ex += __shfl_xor_sync(0xffffffffu, ex, o);
           } else {
