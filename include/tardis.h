@@ -259,6 +259,19 @@ tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
  * and its kernel carries no stamps.  Errors: INVALID_ARG (NULL, max_ctas <= 0), UNSUPPORTED, CUDA. */
 tardis_status_t tardis_debug_phase_stamps(long long* stamps, int32_t max_ctas);
 
+/* A handle's state in a binary file and back (Section 6: the offline component writes the folded matrix and the
+ * predictor to a binary file that the runtime loads).  tardis_save synchronises the handle's last stream and writes, to
+ * the HOST path `path`: a 64-byte header (magic "TARDIS01", d_model, d_ff, dtype, act, pred_group, pred_bits), then W1,
+ * W2^T, the folded matrix (as stored: [channel][output]), b_f, lo, hi, a, c, b1, the predictor codes, scales and
+ * zero-points as raw little-endian arrays, then a 64-bit FNV-1a checksum of the array bytes.  tardis_load reads such a
+ * file, allocates a handle on the current device, uploads the arrays and derives the kernel-specific copies as
+ * tardis_fold does; no fold is recomputed, so the loaded handle gives bit-identical flags and scores, and outputs equal
+ * to those of the saved handle up to the order of floating-point reductions.  *out is valid on return with TARDIS_OK;
+ * work is enqueued on `stream`.  Errors: INVALID_ARG (NULL, file cannot be opened or written), CORRUPT (bad magic,
+ * implausible header, truncated file, checksum mismatch), ALLOC, CUDA. */
+tardis_status_t tardis_save(tardis_handle_t handle, const char* path);
+tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_handle_t* out);
+
 /* Every wait inside the kernels (on a bulk copy's barrier) is bounded: when the limit runs out the kernel records it in
  * the handle's device error word, skips the work that needed the data and returns; tardis_stats then reports
  * TARDIS_ERR_TIMEOUT until the word is cleared.  tardis_debug_wait_timeout makes exactly that happen on purpose, for

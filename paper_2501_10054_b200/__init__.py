@@ -23,7 +23,7 @@ TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_calibrate",
            "tardis_debug_phase_stamps", "tardis_range_search", "tardis_debug_wait_timeout", "tardis_clear_error",
-           "tardis_status_string", "tardis_last_error"]
+           "tardis_save", "tardis_load", "tardis_status_string", "tardis_last_error"]
 
 
 class TardisError(RuntimeError):
@@ -80,7 +80,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_range_search.argtypes = [i32, i32, vp, i64, vp, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp, vp]
     lib.tardis_debug_wait_timeout.argtypes = [vp, i64, vp]
     lib.tardis_clear_error.argtypes = [vp]
-    for name in EXPORTS[:14]:
+    lib.tardis_save.argtypes = [vp, ctypes.c_char_p]
+    lib.tardis_load.argtypes = [ctypes.c_char_p, vp, ctypes.POINTER(vp)]
+    for name in EXPORTS[:16]:
         getattr(lib, name).restype = ctypes.c_int
     lib.tardis_status_string.argtypes = [ctypes.c_int]
     lib.tardis_status_string.restype = ctypes.c_char_p
@@ -229,6 +231,18 @@ def tardis_debug_wait_timeout(handle: int, limit_cycles: int, stream=None):
 
 def tardis_clear_error(handle: int):
     _check(load_library().tardis_clear_error(handle), "tardis_clear_error")
+
+
+def tardis_save(handle: int, path: str):
+    """Writes the handle's state (folded matrix, predictor, original weights, tables) to a binary file."""
+    _check(load_library().tardis_save(handle, os.fsencode(path)), "tardis_save")
+
+
+def tardis_load(path: str, stream=None) -> int:
+    """Reads a file written by tardis_save and returns a new handle on the current device."""
+    out = ctypes.c_void_p()
+    _check(load_library().tardis_load(os.fsencode(path), _stream(stream), ctypes.byref(out)), "tardis_load")
+    return out.value
 
 
 def tardis_destroy(handle: int):

@@ -1,5 +1,6 @@
 // C ABI of libtardis: argument validation, handle life cycle, dispatch.
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -56,6 +57,43 @@ static void free_all(Handle* H) {
   delete H;
 }
 
+// Allocates a handle and its device arrays for a layer of the given shape (nothing is filled in yet).
+static tardis_status_t new_handle(int d, int h, int dtype, int act, int G, int bits, cudaStream_t s, Handle** out) {
+  *out = nullptr;
+  Handle* H = new (std::nothrow) Handle();
+  if (!H) return TARDIS_ERR_ALLOC;
+  memset(H, 0, sizeof(*H));
+  H->magic = kMagic;
+  H->d = d; H->h = h; H->dtype = dtype; H->act = act; H->G = G; H->ngroups = d / G;
+  H->bits = bits;
+  H->esize = dtype == TARDIS_F32 ? 4 : 2;
+  H->last_stream = s;
+  cudaError_t e = cudaGetDevice(&H->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&H->num_sms, cudaDevAttrMultiProcessorCount, H->device);
+  if (e != cudaSuccess) { set_last_error(e, "device query"); delete H; return TARDIS_ERR_CUDA; }
+  const size_t hd = size_t(h) * d;
+  tardis_status_t st = TARDIS_OK;
+  auto A = [&](auto** p, size_t count, size_t* tally) { if (st == TARDIS_OK) st = dev_alloc(p, count, tally); };
+  A(reinterpret_cast<char**>(&H->W1), hd * H->esize, &H->bytes_w1);
+  A(reinterpret_cast<char**>(&H->W2T), hd * H->esize, &H->bytes_w2t);
+  A(reinterpret_cast<char**>(&H->C), size_t(d) * d * H->esize, &H->bytes_folded);
+  A(&H->bf, size_t(d), &H->bytes_folded);
+  A(&H->lo, size_t(h), &H->bytes_tables);
+  A(&H->hi, size_t(h), &H->bytes_tables);
+  A(&H->a, size_t(h), &H->bytes_tables);
+  A(&H->c, size_t(h), &H->bytes_tables);
+  A(&H->b1, size_t(h), &H->bytes_tables);
+  A(&H->codes, hd * H->bits / 32, &H->bytes_predictor);
+  A(reinterpret_cast<char**>(&H->scale), size_t(h) * H->ngroups * H->esize, &H->bytes_predictor);
+  A(&H->zero, size_t(h) * H->ngroups, &H->bytes_predictor);
+  A(&H->yacc, size_t(kGenericChunk) * d, &H->bytes_scratch);
+  A(&H->bitmap, size_t(kGenericChunk) * (h / 32), &H->bytes_scratch);
+  A(&H->counters, size_t(CTR_COUNT), &H->bytes_scratch);
+  if (st != TARDIS_OK) { free_all(H); return st; }
+  *out = H;
+  return TARDIS_OK;
+}
+
 }  // namespace tardis
 
 using namespace tardis;
@@ -81,38 +119,10 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   for (const void* p : al)
     if (!aligned16(p)) return TARDIS_ERR_INVALID_ARG;
 
-  Handle* H = new (std::nothrow) Handle();
-  if (!H) return TARDIS_ERR_ALLOC;
-  memset(H, 0, sizeof(*H));
-  H->magic = kMagic;
-  H->d = d; H->h = h; H->dtype = desc->dtype; H->act = desc->act; H->G = G; H->ngroups = d / G;
-  H->bits = desc->pred_bits;
-  H->esize = desc->dtype == TARDIS_F32 ? 4 : 2;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  H->last_stream = s;
-  cudaError_t e = cudaGetDevice(&H->device);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&H->num_sms, cudaDevAttrMultiProcessorCount, H->device);
-  if (e != cudaSuccess) { set_last_error(e, "device query"); delete H; return TARDIS_ERR_CUDA; }
-
-  const size_t hd = size_t(h) * d;
-  tardis_status_t st = TARDIS_OK;
-  auto A = [&](auto** p, size_t count, size_t* tally) { if (st == TARDIS_OK) st = dev_alloc(p, count, tally); };
-  A(reinterpret_cast<char**>(&H->W1), hd * H->esize, &H->bytes_w1);
-  A(reinterpret_cast<char**>(&H->W2T), hd * H->esize, &H->bytes_w2t);
-  A(reinterpret_cast<char**>(&H->C), size_t(d) * d * H->esize, &H->bytes_folded);
-  A(&H->bf, size_t(d), &H->bytes_folded);
-  A(&H->lo, size_t(h), &H->bytes_tables);
-  A(&H->hi, size_t(h), &H->bytes_tables);
-  A(&H->a, size_t(h), &H->bytes_tables);
-  A(&H->c, size_t(h), &H->bytes_tables);
-  A(&H->b1, size_t(h), &H->bytes_tables);
-  A(&H->codes, hd * H->bits / 32, &H->bytes_predictor);
-  A(reinterpret_cast<char**>(&H->scale), size_t(h) * H->ngroups * H->esize, &H->bytes_predictor);
-  A(&H->zero, size_t(h) * H->ngroups, &H->bytes_predictor);
-  A(&H->yacc, size_t(kGenericChunk) * d, &H->bytes_scratch);
-  A(&H->bitmap, size_t(kGenericChunk) * (h / 32), &H->bytes_scratch);
-  A(&H->counters, size_t(CTR_COUNT), &H->bytes_scratch);
-  if (st != TARDIS_OK) { free_all(H); return st; }
+  Handle* H = nullptr;
+  tardis_status_t st = new_handle(d, h, desc->dtype, desc->act, G, desc->pred_bits, s, &H);
+  if (st != TARDIS_OK) return st;
 
   const bool bf16 = H->dtype == TARDIS_BF16;
   if (bf16) st = batched_prepare(H);                          // allocations; its buffers double as fold temporaries
@@ -124,7 +134,7 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   }
   if (st == TARDIS_OK && bf16) st = fused_prepare(H, s);
   if (st == TARDIS_OK && bf16 && !H->fscratch) st = decode_prepare(H, s);   // wider layers: the older per-token kernel
-  if (st == TARDIS_OK && bf16) st = batched_finish(H, desc, s);
+  if (st == TARDIS_OK && bf16) st = batched_finish(H, desc->W2, s);
   if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
   *out = reinterpret_cast<tardis_handle_t>(H);
   return TARDIS_OK;
@@ -280,6 +290,114 @@ tardis_status_t tardis_clear_error(tardis_handle_t handle) {
   if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
   TARDIS_CUDA_TRY(cudaStreamSynchronize(H->last_stream));
   TARDIS_CUDA_TRY(cudaMemset(H->counters + CTR_ERROR, 0, sizeof(unsigned long long)));
+  return TARDIS_OK;
+}
+
+// ---- a handle's state in a file (Section 6: the offline part writes the folded matrix and the predictor to a binary file)
+// Layout: 64-byte header {8-byte magic, d, h, dtype, act, G, bits as int32, rest zero}, then the arrays in the order of
+// `parts` below as raw bytes, then a 64-bit FNV-1a checksum of all array bytes.
+static const char kFileMagic[8] = {'T', 'A', 'R', 'D', 'I', 'S', '0', '1'};
+
+struct FilePart { void* dev; size_t bytes; };
+static int file_parts(Handle* H, FilePart* parts) {
+  const size_t hd = size_t(H->h) * H->d, h = H->h, d = H->d;
+  int n = 0;
+  parts[n++] = {H->W1, hd * H->esize};
+  parts[n++] = {H->W2T, hd * H->esize};
+  parts[n++] = {H->C, d * d * H->esize};
+  parts[n++] = {H->bf, d * 4};
+  parts[n++] = {H->lo, h * 4}; parts[n++] = {H->hi, h * 4}; parts[n++] = {H->a, h * 4}; parts[n++] = {H->c, h * 4};
+  parts[n++] = {H->b1, h * 4};
+  parts[n++] = {H->codes, hd / 8 * H->bits};
+  parts[n++] = {H->scale, h * size_t(H->ngroups) * H->esize};
+  parts[n++] = {H->zero, h * size_t(H->ngroups)};
+  return n;
+}
+static uint64_t fnv1a(uint64_t hsh, const unsigned char* p, size_t n) {
+  for (size_t i = 0; i < n; ++i) { hsh ^= p[i]; hsh *= 1099511628211ull; }
+  return hsh;
+}
+
+tardis_status_t tardis_save(tardis_handle_t handle, const char* path) {
+  Handle* H = check(handle);
+  if (!H || !path) return TARDIS_ERR_INVALID_ARG;
+  if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
+  TARDIS_CUDA_TRY(cudaStreamSynchronize(H->last_stream));
+  FILE* f = fopen(path, "wb");
+  if (!f) { snprintf(g_last_error, sizeof(g_last_error), "tardis_save: cannot open %s", path); return TARDIS_ERR_INVALID_ARG; }
+  unsigned char header[64] = {};
+  memcpy(header, kFileMagic, 8);
+  const int32_t dims[6] = {H->d, H->h, H->dtype, H->act, H->G, H->bits};
+  memcpy(header + 8, dims, sizeof(dims));
+  bool ok = fwrite(header, 1, 64, f) == 64;
+  const size_t chunk = size_t(8) << 20;
+  unsigned char* buf = static_cast<unsigned char*>(malloc(chunk));
+  if (!buf) { fclose(f); return TARDIS_ERR_ALLOC; }
+  FilePart parts[16];
+  const int np = file_parts(H, parts);
+  uint64_t sum = 14695981039346656037ull;
+  cudaError_t e = cudaSuccess;
+  for (int i = 0; i < np && ok && e == cudaSuccess; ++i)
+    for (size_t o = 0; o < parts[i].bytes && ok && e == cudaSuccess; o += chunk) {
+      const size_t nb = parts[i].bytes - o < chunk ? parts[i].bytes - o : chunk;
+      e = cudaMemcpy(buf, static_cast<const unsigned char*>(parts[i].dev) + o, nb, cudaMemcpyDeviceToHost);
+      if (e == cudaSuccess) { sum = fnv1a(sum, buf, nb); ok = fwrite(buf, 1, nb, f) == nb; }
+    }
+  if (ok && e == cudaSuccess) ok = fwrite(&sum, 1, 8, f) == 8;
+  free(buf);
+  ok = (fclose(f) == 0) && ok;
+  if (e != cudaSuccess) { set_last_error(e, "tardis_save"); return TARDIS_ERR_CUDA; }
+  if (!ok) { snprintf(g_last_error, sizeof(g_last_error), "tardis_save: write to %s failed", path); return TARDIS_ERR_INVALID_ARG; }
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_handle_t* out) {
+  if (!path || !out) return TARDIS_ERR_INVALID_ARG;
+  *out = nullptr;
+  FILE* f = fopen(path, "rb");
+  if (!f) { snprintf(g_last_error, sizeof(g_last_error), "tardis_load: cannot open %s", path); return TARDIS_ERR_INVALID_ARG; }
+  unsigned char header[64];
+  int32_t dims[6];
+  if (fread(header, 1, 64, f) != 64 || memcmp(header, kFileMagic, 8) != 0) { fclose(f); return TARDIS_ERR_CORRUPT; }
+  memcpy(dims, header + 8, sizeof(dims));
+  const int d = dims[0], h = dims[1], dtype = dims[2], act = dims[3], G = dims[4], bits = dims[5];
+  const bool sane = d > 0 && h > 0 && G > 0 && d <= (1 << 20) && h <= (1 << 24) && (dtype == TARDIS_F32 || dtype == TARDIS_BF16) &&
+                    act >= 0 && act <= TARDIS_ACT_RELU && !(d % 8) && !(h % 32) && !(G % 16) && !(d % G) &&
+                    (bits == 2 || bits == 4 || bits == 8);
+  if (!sane) { fclose(f); return TARDIS_ERR_CORRUPT; }
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  Handle* H = nullptr;
+  tardis_status_t st = new_handle(d, h, dtype, act, G, bits, s, &H);
+  if (st != TARDIS_OK) { fclose(f); return st; }
+  const size_t chunk = size_t(8) << 20;
+  unsigned char* buf = static_cast<unsigned char*>(malloc(chunk));
+  if (!buf) { fclose(f); free_all(H); return TARDIS_ERR_ALLOC; }
+  FilePart parts[16];
+  const int np = file_parts(H, parts);
+  uint64_t sum = 14695981039346656037ull, stored = 0;
+  bool ok = true;
+  cudaError_t e = cudaSuccess;
+  for (int i = 0; i < np && ok && e == cudaSuccess; ++i)
+    for (size_t o = 0; o < parts[i].bytes && ok && e == cudaSuccess; o += chunk) {
+      const size_t nb = parts[i].bytes - o < chunk ? parts[i].bytes - o : chunk;
+      ok = fread(buf, 1, nb, f) == nb;
+      if (ok) { sum = fnv1a(sum, buf, nb); e = cudaMemcpy(static_cast<unsigned char*>(parts[i].dev) + o, buf, nb, cudaMemcpyHostToDevice); }
+    }
+  if (ok) ok = fread(&stored, 1, 8, f) == 8 && stored == sum;
+  free(buf);
+  fclose(f);
+  if (e != cudaSuccess) { set_last_error(e, "tardis_load"); free_all(H); return TARDIS_ERR_CUDA; }
+  if (!ok) { free_all(H); return TARDIS_ERR_CORRUPT; }          // truncated file or checksum mismatch
+  e = cudaMemsetAsync(H->counters, 0, CTR_COUNT * sizeof(unsigned long long), s);
+  if (e != cudaSuccess) { set_last_error(e, "tardis_load"); free_all(H); return TARDIS_ERR_CUDA; }
+  // the kernel-specific copies are derived from the stored arrays exactly as tardis_fold derives them
+  const bool bf16 = H->dtype == TARDIS_BF16;
+  if (bf16) st = batched_prepare(H);
+  if (st == TARDIS_OK && bf16) st = fused_prepare(H, s);
+  if (st == TARDIS_OK && bf16 && !H->fscratch) st = decode_prepare(H, s);
+  if (st == TARDIS_OK && bf16) st = batched_finish(H, nullptr, s);
+  if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
+  *out = reinterpret_cast<tardis_handle_t>(H);
   return TARDIS_OK;
 }
 

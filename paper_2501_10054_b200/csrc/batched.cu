@@ -267,7 +267,7 @@ tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cu
   return TARDIS_OK;
 }
 
-tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s) {
+tardis_status_t batched_finish(Handle* H, const void* W2, cudaStream_t s) {
   State* S = static_cast<State*>(H->bstate);
   if (!S) return TARDIS_OK;
   const int d = H->d, h = H->h;
@@ -275,7 +275,9 @@ tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaSt
   dim3 tb(32, 8);
   // W_f[i][k] row-major (the GEMMs want the channel index contiguous in both operands): transpose of C
   k_transpose_b<__nv_bfloat16><<<dim3((d + 31) / 32, (d + 31) / 32), tb, 0, s>>>(static_cast<const __nv_bfloat16*>(H->C), S->Wf, d, d);
-  TARDIS_CUDA_TRY(cudaMemcpyAsync(S->W2, desc->W2, hd * 2, cudaMemcpyDeviceToDevice, s));
+  if (W2) TARDIS_CUDA_TRY(cudaMemcpyAsync(S->W2, W2, hd * 2, cudaMemcpyDeviceToDevice, s));
+  else      // (a handle read back from a file has only the transposed copy)
+    k_transpose_b<__nv_bfloat16><<<dim3((d + 31) / 32, (h + 31) / 32), tb, 0, s>>>(static_cast<const __nv_bfloat16*>(H->W2T), S->W2, h, d);
   if (H->bits <= 4)   // (8-bit codes: the batched path is not used, see the dispatch)
     k_dequant_split<<<h, 256, 0, s>>>(H->codes, static_cast<const __nv_bfloat16*>(H->scale), H->zero, S->What_hi, S->What_lo,
                                     S->smaxrow, d, H->G, H->bits);

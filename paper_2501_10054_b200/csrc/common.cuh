@@ -80,7 +80,7 @@ void fused_release(Handle* H);
 tardis_status_t fused_read_stamps(long long* out, int max_ctas);
 tardis_status_t launch_wait_that_runs_out(Handle* H, long long limit_cycles, cudaStream_t s);   // UNSUPPORTED unless built with TARDIS_PHASE_STAMPS
 tardis_status_t batched_prepare(Handle* H);                                                   // bf16 only: allocations
-tardis_status_t batched_finish(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);    // fills the batched state
+tardis_status_t batched_finish(Handle* H, const void* W2, cudaStream_t s);   // fills the batched state (W2 null: from W2T)
 tardis_status_t launch_batched_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
 void batched_release(Handle* H);
 tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);  // bf16 fold on the tensor cores

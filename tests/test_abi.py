@@ -76,6 +76,9 @@ def test_invalid_arguments_return_status_before_any_launch(lib):
     assert lib.tardis_gemm_bf16(8, 8, 8, 16, 8, 16, 8, 20, 8, None) == 1
     assert lib.tardis_gemm_bf16(8, 8, 8, 16, 8, 16, 8, None, 8, None) == 1
     assert lib.tardis_debug_phase_stamps(None, 4) == 1
+    assert lib.tardis_save(None, b"/tmp/x") == 1 and lib.tardis_load(None, None, None) == 1
+    out2 = ctypes.c_void_p()
+    assert lib.tardis_load(b"/nonexistent/dir/file", None, ctypes.byref(out2)) == 1 and out2.value is None
 
 
 def test_binding_fails_loudly_without_library(tmp_path):

@@ -263,3 +263,43 @@ def test_bounded_wait_runs_out_is_reported_and_cleared():
     Hp.assert_parity(L, s, x, y1, F1, None, score_tol=None, label="after a cleared time-out")
     assert lib.tardis_debug_wait_timeout(h, -1, None) == 1
     T.tardis_destroy(h)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_save_and_load_round_trip(tmp_path, dtype):
+    """A handle written to a file and read back gives the same flags and scores bit for bit, outputs within the parity
+    tolerance of the oracle, and the same footprint; a damaged file is refused."""
+    cfg = W.LayerConfig("saveload_" + dtype, 512, 2048, dtype=dtype, n_calib=512)
+    L = _layer(cfg)
+    s = L.numpy64()
+    x = W.make_tokens(cfg, 21, 6).cuda()
+    h = T.fold_layer(L)
+    path = str(tmp_path / "layer.tardis")
+    T.tardis_save(h, path)
+    h2 = T.tardis_load(path)
+    calls = [1, 4, 16]
+    y1, F1, S1 = Hp.gpu_forward(h, L, x, calls)
+    y2, F2, S2 = Hp.gpu_forward(h2, L, x, calls)
+    assert (F1 == F2).all() and np.array_equal(S1, S2, equal_nan=True)
+    Hp.assert_parity(L, s, x, y2, F2, None, score_tol=None, label="loaded handle")
+    st1, st2 = T.tardis_stats(h), T.tardis_stats(h2)
+    for k in ("bytes_folded", "bytes_predictor", "bytes_tables", "bytes_w1", "bytes_w2t"):
+        assert st1[k] == st2[k]
+    Wf1 = torch.empty(cfg.d_model, cfg.d_model, dtype=x.dtype, device="cuda")
+    Wf2 = torch.empty_like(Wf1)
+    T.tardis_export_folded(h, Wf1, None)
+    T.tardis_export_folded(h2, Wf2, None)
+    torch.cuda.synchronize()
+    assert torch.equal(Wf1, Wf2)
+    T.tardis_destroy(h)
+    T.tardis_destroy(h2)
+    # one flipped byte in the middle, and a truncated file: TARDIS_ERR_CORRUPT (6), no handle
+    raw = bytearray(open(path, "rb").read())
+    raw[len(raw) // 2] ^= 0x40
+    bad = str(tmp_path / "bad.tardis")
+    open(bad, "wb").write(raw)
+    lib = T.load_library()
+    out = ctypes.c_void_p()
+    assert lib.tardis_load(bad.encode(), None, ctypes.byref(out)) == 6 and out.value is None
+    open(bad, "wb").write(raw[:len(raw) // 3])
+    assert lib.tardis_load(bad.encode(), None, ctypes.byref(out)) == 6 and out.value is None
