@@ -91,9 +91,9 @@ struct Scratch {           // handle-owned device memory of this path
 };
 
 // ---- shared-memory carve-up (host and device agree through this) -----------------------------------
-// Small tables first, then what depends on the number of tokens of the call (x, partial pre-activations), then the
-// predictor buffers, the limbs and the partial scores.  Everything from pbuf to the end of the CTA's shared memory
-// becomes the row slots of the result fixing.
+// Small tables first, then x of the call's tokens, then the predictor buffers, the limbs and the partial scores.
+// Everything from pbuf to the partial pre-activations at the end of the CTA's shared memory becomes the row slots of
+// the result fixing.
 struct SmemLayout {
   size_t zeros, sx2, tab, fl_j, fl_mask, fl_delta, rc, flagbits, red, bars, misc, xh, wz, pbuf, xq, zpart, pred_end, slots_end;
   int xstride, xq_stride;
@@ -115,12 +115,16 @@ struct SmemLayout {
     bars = take(size_t(MAXBUF + MAXGROUPS) * sizeof(uint64_t), 8);
     misc = take(64 * sizeof(int), 8);
     xh = take(size_t(ntok) * xstride * 2, 16);
-    wz = take(size_t(MAXGROUPS) * MAXGS * ntok * 33 * sizeof(float), 16);   // one buffer per slot group
     pbuf = take(size_t(nbuf) * buf_bytes, 128);
     xq = take(size_t(2) * 4 * xq_stride, 128);             // limbs of two tokens
     zpart = take(size_t(tiles_max) * NWP * 2 * 16 * sizeof(float), 16);
     pred_end = o;
-    slots_end = total_bytes > o ? total_bytes : o;
+    // the partial pre-activations of the result fixing (one buffer per slot group) sit at the very end: they are not needed
+    // while the predictor runs, so they do not compete with its buffers for room
+    const size_t wzbytes = size_t(MAXGROUPS) * MAXGS * ntok * 33 * sizeof(float);
+    const size_t end = total_bytes > o + wzbytes ? total_bytes : o + wzbytes;
+    wz = (end - wzbytes) / 16 * 16;
+    slots_end = wz;
   }
 };
 enum { MS_NRC = 1, MS_ERR = 2, MS_LAST = 3, MS_NUN = 4, MS_AMAX = 8, MS_NONFIN = 12, MS_TOKCNT = 16, MS_WCNT = 24, MS_BUFCNT = 32 };
@@ -1000,7 +1004,7 @@ tardis_status_t fused_prepare(Handle* H, cudaStream_t s) {
     S->nbuf_n[nt] = 0;
     for (int nbuf = tiles_max < MAXBUF ? tiles_max : MAXBUF; nbuf >= 1; --nbuf) {
       const SmemLayout L(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes, nt, size_t(max_smem));
-      if (L.pred_end <= size_t(max_smem) && L.slots_end - L.pbuf >= need_slots) { S->nbuf_n[nt] = nbuf; break; }
+      if (L.pred_end <= size_t(max_smem) && L.slots_end <= size_t(max_smem) && L.slots_end - L.pbuf >= need_slots) { S->nbuf_n[nt] = nbuf; break; }
     }
     if (S->nbuf_n[nt] == 0) { delete S; return TARDIS_OK; }
   }
