@@ -100,3 +100,42 @@ def test_prefill_layers_4096_tokens_in_one_call(seed):
 def test_large_8k_decode_and_prefill():
     info, frac = _check(W.CONFIGS["large_8k"], [1, 1, 32, 4096], sample_per_call=3, fold_rows=4, flag_tokens=256)
     assert 0.07 < frac < 0.13
+
+
+@pytest.mark.parametrize("cfgname", ["large_8k", "decode_7b"])
+@pytest.mark.parametrize("path", [0, 3])
+def test_adversarial_tokens_one_huge_channel_many_tiny(path, cfgname):
+    """Tokens built to stress the fast scores: one channel thousands of times larger than the rest, the rest tiny with
+    alternating signs, at d_model = 8192 (the longest accumulation) and at the headline shape.  The flags of every such token
+    must still equal the oracle's, on the fused kernels and on the batched tensor-core path (whose allowance for its fp32 accumulation is an
+    assumed bound: this is the search for a violation)."""
+    cfg = W.CONFIGS[cfgname]
+    dev = torch.device("cuda", 0)
+    L = W.make_layer(cfg, 2, device=dev)
+    s = L.numpy64()
+    d = cfg.d_model
+    g = torch.Generator().manual_seed(99)
+    n = 24
+    x = torch.empty(n, d)
+    sign = torch.tensor([1.0, -1.0]).repeat(d // 2)
+    for t in range(n):
+        tiny = (10.0 ** -(1 + t % 4)) * (0.5 + torch.rand(d, generator=g)) * sign
+        x[t] = tiny
+        x[t, int(torch.randint(0, d, (1,), generator=g))] = float(2.0 ** (3 + t % 9)) * (1 if t % 2 else -1)
+    x = x.to(torch.bfloat16).to(dev)
+    h = T.fold_layer(L)
+    try:
+        T.tardis_set_path(h, path)
+        y, F, S = Hp.gpu_forward(h, L, x, [n] if path == 3 else [1] * n, capture=True)
+        x64 = x.double().cpu().numpy()
+        zhat = O.predictor_score(x64, s["codes"], s["scale"], s["zero"], s["group"], s["b1"], s["bits"])
+        F_ref = O.flags_from_score(zhat, s["lo"], s["hi"])
+        band = O.near_threshold(zhat, s["lo"], s["hi"], Hp.BAND)
+        mism = (F != F_ref) & ~band
+        assert not mism.any(), "%d flag mismatches on adversarial tokens (path %d)" % (mism.sum(), path)
+        err = np.abs(S - zhat)
+        print("adversarial tokens, " + cfgname + ", path %d: largest score error %.3e (score magnitudes up to %.1f), %d pairs in the band"
+              % (path, float(np.nanmax(err)), float(np.abs(zhat).max()), int(band.sum())))
+        assert T.tardis_stats(h)["device_error"] == 0
+    finally:
+        T.tardis_destroy(h)
