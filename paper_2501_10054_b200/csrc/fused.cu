@@ -95,8 +95,8 @@ struct Scratch {           // handle-owned device memory of this path
 // Everything from pbuf to the partial pre-activations at the end of the CTA's shared memory becomes the row slots of
 // the result fixing.
 struct SmemLayout {
-  size_t zeros, sx2, tab, fl_j, fl_mask, fl_delta, rc, flagbits, red, bars, misc, xh, wz, pbuf, xq, zpart, pred_end, slots_end;
-  int xstride, xq_stride;
+  size_t zeros, sx2, tab, fl_j, fl_mask, fl_delta, rc, flagbits, red, bars, misc, xh, wz, wz_end, pbuf, xq, zpart, pred_end, slots_end;
+  int xstride, xq_stride, wz_groups;
   __host__ __device__ SmemLayout(int dpad, int ngroups, int tiles_max, int nbuf, int buf_bytes, int ntok, size_t total_bytes) {
     size_t o = 0;
     auto take = [&](size_t bytes, size_t align) { o = (o + align - 1) / align * align; size_t r = o; o += bytes; return r; };
@@ -119,11 +119,17 @@ struct SmemLayout {
     xq = take(size_t(2) * 4 * xq_stride, 128);             // limbs of two tokens
     zpart = take(size_t(tiles_max) * NWP * 2 * 16 * sizeof(float), 16);
     pred_end = o;
-    // the partial pre-activations of the result fixing (one buffer per slot group) sit at the very end: they are not needed
-    // while the predictor runs, so they do not compete with its buffers for room
-    const size_t wzbytes = size_t(MAXGROUPS) * MAXGS * ntok * 33 * sizeof(float);
+    // the partial pre-activations of the result fixing sit at the very end: they are not needed while the predictor runs,
+    // so they do not compete with its buffers for room.  One buffer per step of MAXGS neurons; as many buffers as fit behind
+    // the predictor's state, MAXGROUPS at most (one at least: wz_end tells the caller whether that one fits)
+    const size_t per = size_t(MAXGS) * ntok * 33 * sizeof(float);
+    size_t nb = total_bytes > o ? (total_bytes - o) / per : 0;
+    nb = nb > size_t(MAXGROUPS) ? size_t(MAXGROUPS) : (nb < 1 ? 1 : nb);
+    wz_groups = int(nb);
+    const size_t wzbytes = nb * per;
     const size_t end = total_bytes > o + wzbytes ? total_bytes : o + wzbytes;
     wz = (end - wzbytes) / 16 * 16;
+    wz_end = wz + wzbytes;
     slots_end = wz;
   }
 };
@@ -741,8 +747,9 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
       }
     }
     const int wzstride = MAXGS * n * 33;                            // floats per buffer of partial sums
-    for (int c0 = 0; c0 < nA; c0 += NG) {
-      const int c1 = min(nA, c0 + NG);
+    const int NCH = min(NG, L.wz_groups);                           // steps summed up together
+    for (int c0 = 0; c0 < nA; c0 += NCH) {
+      const int c1 = min(nA, c0 + NCH);
       for (int st = c0; st < c1; ++st) {
         const int nw1 = min(GS, nun - st * GS);
         const bool landed = wait_group(st);
@@ -1004,7 +1011,7 @@ tardis_status_t fused_prepare(Handle* H, cudaStream_t s) {
     S->nbuf_n[nt] = 0;
     for (int nbuf = tiles_max < MAXBUF ? tiles_max : MAXBUF; nbuf >= 1; --nbuf) {
       const SmemLayout L(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes, nt, size_t(max_smem));
-      if (L.pred_end <= size_t(max_smem) && L.slots_end <= size_t(max_smem) && L.slots_end - L.pbuf >= need_slots) { S->nbuf_n[nt] = nbuf; break; }
+      if (L.pred_end <= size_t(max_smem) && L.wz_end <= size_t(max_smem) && L.slots_end - L.pbuf >= need_slots) { S->nbuf_n[nt] = nbuf; break; }
     }
     if (S->nbuf_n[nt] == 0) { delete S; return TARDIS_OK; }
   }
