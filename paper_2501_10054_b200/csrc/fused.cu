@@ -717,15 +717,22 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
     }
     return landed;
   };
-  // the predictor warps start the first copies on their own: the streaming warps may still be busy
+  // the predictor warps start the first copies on their own: the streaming warps may still be busy.  Only W1 rows
+  // go out here: the pre-activations are needed first, and W2^T rows asked for at the same moment would share the
+  // memory system with them
   if (warp < NWP) {
     const int nun = misc[MS_NUN];
+    const int nA0 = (nun + GS - 1) / GS;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the region was read with ordinary loads
-    for (int st = 0; st < NG; ++st) fill(st, nun, st);
+    for (int st = 0; st < NG && st < nA0; ++st) fill(st, nun, st);
   }
   __syncthreads();
   const int nun = misc[MS_NUN];
   const int nA = (nun + GS - 1) / GS;
+  if (nA < NG) {                                                    // slot groups left over: the first W2^T rows follow
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    for (int st = nA; st < NG; ++st) fill(st, nun, NW - 1 - st);
+  }
   const int nks = d >> 4;                                           // 16-channel steps of a row (= 16-column tiles of an output)
   FZ_STAMP_VALUE(tid == 0, ST_NFL, nun);
   // -- pre-activations and deltas: steps over the W1 rows, NG steps at a time --
