@@ -248,6 +248,25 @@ tardis_status_t tardis_range_search(int32_t d_ff, int32_t n_cal, const float* z,
  * other. */
 tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
 
+/* Deterministic accumulation, on (1) or off (0, the default).  The paper does not
+ * say in which order the speculative product and the corrections of Section 5.4
+ * are added up; by default this library adds partial sums to y in the order in
+ * which the CTAs finish (floating-point atomics), so the last bits of y may differ
+ * between two runs on the same input.  With the mode on, every partial sum is
+ * written to a place of its own and added in one fixed order (the fused decode
+ * kernel keeps [d_model / 256 + CTAs][4][d_model] fp32 partial outputs, allocated
+ * by this call the first time, and a second small kernel sums them; the batched
+ * products no longer split their channel range): y is then the same bits from run
+ * to run for the same handle, input and token count.  Flags do not depend on the
+ * mode.  Cost: one more launch per 4 tokens on the fused path, and products of
+ * few tokens run on fewer CTAs on the batched path.
+ * Returns TARDIS_ERR_UNSUPPORTED when the layer is served only by kernels that
+ * add with atomics (fp32 layers, 8-bit codes, wider bf16 layers on the per-token
+ * kernel); a later tardis_ffn_forward on a handle in this mode returns
+ * TARDIS_ERR_UNSUPPORTED too where its path choice (tardis_set_path 1 or 4) leads
+ * to such kernels.  tardis_ffn_forward_static does not look at the mode. */
+tardis_status_t tardis_set_deterministic(tardis_handle_t handle, int32_t on);
+
 /* Profiling aid of the fused decode kernel (the online path of Section 5.4 as one launch).  A library
  * built with -DTARDIS_PHASE_STAMPS (python -m paper_2501_10054_b200.build --stamps) makes every CTA of that
  * kernel record the GPU's global nanosecond timer at its phase boundaries; this call synchronises the

@@ -21,7 +21,7 @@ TARDIS_F32, TARDIS_BF16 = 0, 1
 TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
-           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_destroy", "tardis_calibrate",
+           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_set_deterministic", "tardis_destroy", "tardis_calibrate",
            "tardis_debug_phase_stamps", "tardis_range_search", "tardis_debug_wait_timeout", "tardis_clear_error",
            "tardis_save", "tardis_load", "tardis_status_string", "tardis_last_error"]
 
@@ -73,6 +73,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_set_debug_capture.argtypes = [vp, vp, vp]
     lib.tardis_export_folded.argtypes = [vp, vp, vp, vp]
     lib.tardis_set_path.argtypes = [vp, i32]
+    lib.tardis_set_deterministic.argtypes = [vp, i32]
     lib.tardis_destroy.argtypes = [vp]
     lib.tardis_gemm_bf16.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, i32, vp]
     lib.tardis_calibrate.argtypes = [i32, i32, vp, i64, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp]
@@ -213,6 +214,10 @@ def tardis_export_folded(handle: int, Wf: Optional[torch.Tensor], bf: Optional[t
 
 def tardis_set_path(handle: int, path: int):
     _check(load_library().tardis_set_path(handle, path), "tardis_set_path")
+
+
+def tardis_set_deterministic(handle: int, on: bool):
+    _check(load_library().tardis_set_deterministic(handle, 1 if on else 0), "tardis_set_deterministic")
 
 
 def tardis_debug_phase_stamps(max_ctas: int = 512):

@@ -151,10 +151,12 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   H->last_stream = s;
   tardis_status_t st;
-  const bool has_fused = H->fscratch != nullptr || H->codes_mma != nullptr;
+  // (deterministic mode: only the kernels of fused.cu and the tensor-core products without a split channel range qualify)
+  const bool has_fused = H->fscratch != nullptr || (H->codes_mma != nullptr && !H->deterministic);
   const bool fused = has_fused && ((H->path_override == 0 && n_tokens <= (H->fscratch ? kDecodeMaxTokens : 8)) || (H->path_override == 2 && n_tokens <= 4096));
   // (8-bit codes times a bf16 scale do not fit the exact two-term bf16 form the batched scores rely on)
   const bool batched = ((H->path_override == 0 && !fused) || H->path_override == 3) && H->bstate != nullptr && H->bits <= 4;
+  if (H->deterministic && !fused && !batched) return TARDIS_ERR_UNSUPPORTED;
   if (fused) {
     st = H->fscratch ? launch_fused_forward(H, x, y, int(n_tokens), s) : launch_decode_forward(H, x, y, int(n_tokens), s);
     H->last_path = 2;
@@ -398,6 +400,19 @@ tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_han
   if (st == TARDIS_OK && bf16) st = batched_finish(H, nullptr, s);
   if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
   *out = reinterpret_cast<tardis_handle_t>(H);
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_set_deterministic(tardis_handle_t handle, int32_t on) {
+  Handle* H = check(handle);
+  if (!H || !(on == 0 || on == 1)) return TARDIS_ERR_INVALID_ARG;
+  if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
+  if (on && !H->fscratch && !(H->bstate != nullptr && H->bits <= 4)) return TARDIS_ERR_UNSUPPORTED;
+  if (on) {
+    const tardis_status_t st = fused_set_deterministic(H, true);
+    if (st != TARDIS_OK) return st;
+  }
+  H->deterministic = on != 0;
   return TARDIS_OK;
 }
 

@@ -332,7 +332,8 @@ tardis_status_t launch_batched_forward(Handle* H, const void* xv, void* yv, int6
     }
     // A batch of one tile of tokens is bound by weight traffic and its products over d outputs have few
     // tiles: those split their channel range over several CTAs, which add into the fp32 accumulator.
-    const int splits = (n <= 128 && d <= 8192) ? 4 : 1;
+    // (not in deterministic mode: the order of those additions is not fixed)
+    const int splits = (n <= 128 && d <= 8192 && !H->deterministic) ? 4 : 1;
     // 2. speculative folded product
     GemmArgs f = {};
     f.M = n; f.N = d; f.K1 = d; f.A1 = xc; f.lda1 = d; f.B1 = S->Wf; f.ldb1 = d;

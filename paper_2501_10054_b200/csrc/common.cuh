@@ -49,6 +49,7 @@ struct Handle {
   uint64_t calls, tokens, last_path, launches;
   cudaStream_t last_stream;
   int path_override;
+  bool deterministic;    // y must not depend on the order in which partial sums arrive (tardis_set_deterministic)
   size_t bytes_folded, bytes_predictor, bytes_tables, bytes_w1, bytes_w2t, bytes_scratch;
   int num_sms;
 };
@@ -77,6 +78,7 @@ tardis_status_t decode_read_stamps(long long* out, int max_ctas);
 tardis_status_t fused_prepare(Handle* H, cudaStream_t s);                  // builds the state of fused.cu (bf16, d_model <= 4608)
 tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s);
 void fused_release(Handle* H);
+tardis_status_t fused_set_deterministic(Handle* H, bool on);               // allocates the partial-output buffer of the mode
 tardis_status_t fused_read_stamps(long long* out, int max_ctas);
 tardis_status_t launch_wait_that_runs_out(Handle* H, long long limit_cycles, cudaStream_t s);   // UNSUPPORTED unless built with TARDIS_PHASE_STAMPS
 tardis_status_t batched_prepare(Handle* H);                                                   // bf16 only: allocations

@@ -72,6 +72,7 @@ struct Params {
   const int2* plan;        // per CTA: first tile, tile count
   const __nv_bfloat16* x; __nv_bfloat16* y;
   float* yacc;             // [NREP][MAXT][dacc] fp32
+  float* dpart;            // deterministic mode: [nkc + grid][MAXT][dacc] partial outputs, each written by one owner; else null
   unsigned int* ctl; unsigned long long* counters;
   uint32_t* dbg_bitmap; double* dbg_scores;
   int n;                   // tokens of this call (1..MAXT)
@@ -87,6 +88,7 @@ struct Params {
 struct Scratch {           // handle-owned device memory of this path
   uint8_t* pblocks; int2* plan; float* smax; float* yacc; unsigned int* ctl; uint4* Cp;
   Params base; size_t smem_bytes; size_t bytes; int grid; const void* kernels[2][2]; bool pairs_fit;
+  float* dpart;            // partial outputs of the deterministic mode (allocated when the mode is first switched on)
   int nbuf_n[MAXT + 1];    // tile buffers in shared memory for a call of n tokens
 };
 
@@ -439,13 +441,19 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
       raw = more ? issue() : 0xffffffffu;
       if (nx >= 0) load(ba, nx, 0);
       multiply(c, bb, xp, 3);
-      if (2 * t4 < n) {
-        red_add_f32(rep + (2 * t4) * p.dacc + it * 16 + g, c[0][0] + c[1][0]);
-        red_add_f32(rep + (2 * t4) * p.dacc + it * 16 + g + 8, c[0][2] + c[1][2]);
-      }
-      if (2 * t4 + 1 < n) {
-        red_add_f32(rep + (2 * t4 + 1) * p.dacc + it * 16 + g, c[0][1] + c[1][1]);
-        red_add_f32(rep + (2 * t4 + 1) * p.dacc + it * 16 + g + 8, c[0][3] + c[1][3]);
+      if (p.dpart) {                                    // deterministic mode: the unit's sums have a place of their own
+        float* const o = p.dpart + size_t(kc) * MAXT * p.dacc + it * 16 + g;
+        if (2 * t4 < n) { o[(2 * t4) * p.dacc] = c[0][0] + c[1][0]; o[(2 * t4) * p.dacc + 8] = c[0][2] + c[1][2]; }
+        if (2 * t4 + 1 < n) { o[(2 * t4 + 1) * p.dacc] = c[0][1] + c[1][1]; o[(2 * t4 + 1) * p.dacc + 8] = c[0][3] + c[1][3]; }
+      } else {
+        if (2 * t4 < n) {
+          red_add_f32(rep + (2 * t4) * p.dacc + it * 16 + g, c[0][0] + c[1][0]);
+          red_add_f32(rep + (2 * t4) * p.dacc + it * 16 + g + 8, c[0][2] + c[1][2]);
+        }
+        if (2 * t4 + 1 < n) {
+          red_add_f32(rep + (2 * t4 + 1) * p.dacc + it * 16 + g, c[0][1] + c[1][1]);
+          red_add_f32(rep + (2 * t4 + 1) * p.dacc + it * 16 + g + 8, c[0][3] + c[1][3]);
+        }
       }
       u = nx;
     }
@@ -846,7 +854,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   }
   // The accumulators hold 16 output columns x (leading | remaining term of 4 tokens) per tile: add the two terms,
   // stage the sums in shared memory (the row slots are free) and add them to this CTA's replica with 128-bit reductions.
-  if (nun > 0) {
+  if (nun > 0 || p.dpart) {                                         // (deterministic mode: every CTA writes its part, zeros too)
     __syncthreads();
     float* const yst = reinterpret_cast<float*>(slots);           // [n][dpad]
 #pragma unroll
@@ -865,7 +873,8 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
     for (int i = tid; i < n * nq; i += NTH) {
       const int t = i / nq, v4 = i - t * nq;
       const float4 s = *reinterpret_cast<const float4*>(yst + t * p.dpad + v4 * 4);
-      red_add_v4(rep + t * p.dacc + v4 * 4, s.x, s.y, s.z, s.w);
+      if (p.dpart) *reinterpret_cast<float4*>(p.dpart + (size_t(p.nkc + blockIdx.x) * MAXT + t) * p.dacc + v4 * 4) = s;
+      else red_add_v4(rep + t * p.dacc + v4 * 4, s.x, s.y, s.z, s.w);
     }
   }
   FZ_STAMP(tid == 0, ST_FIXED);
@@ -879,7 +888,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   FZ_STAMP(tid == 0, ST_COUNTED);
   if (misc[MS_LAST] == int(gridDim.x) - 1) {
     __threadfence();
-    for (int i = tid; i < n * p.nvec; i += NTH) {
+    for (int i = tid; i < (p.dpart ? 0 : n * p.nvec); i += NTH) {    // (deterministic mode: k_ordered_sum writes y)
       const int t = i / p.nvec, c0 = (i - t * p.nvec) * 8;
       float4 a0[NREP + 1], a1[NREP + 1];
       a0[NREP] = *reinterpret_cast<const float4*>(p.bf + c0);
@@ -1085,8 +1094,48 @@ tardis_status_t fused_prepare(Handle* H, cudaStream_t s) {
   return TARDIS_OK;
 }
 
+// Deterministic mode: y[t][i] = b_f[i] + the partial outputs of the channel chunks and of the CTAs (parts 0 .. nparts - 1).
+// A warp takes four columns of one token: lane l adds parts l, l + 32, ... in ascending order, the 32 lane sums meet
+// in a fixed tree.  The same bits whenever the inputs are the same.
+__global__ void k_ordered_sum(const float* __restrict__ dpart, const float* __restrict__ bf, __nv_bfloat16* __restrict__ y,
+                              int n, int d, int dacc, int nparts) {
+  const int nq = d >> 2;
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (i >= n * nq) return;                              // (the same for the whole warp)
+  const int t = i / nq, q = i - t * nq;
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+  for (int part = lane; part < nparts; part += 32) {
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(dpart + (size_t(part) * fz::MAXT + t) * dacc + q * 4));
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    s.x += __shfl_xor_sync(0xffffffffu, s.x, o); s.y += __shfl_xor_sync(0xffffffffu, s.y, o);
+    s.z += __shfl_xor_sync(0xffffffffu, s.z, o); s.w += __shfl_xor_sync(0xffffffffu, s.w, o);
+  }
+  if (lane == 0) {
+    const float4 b = *reinterpret_cast<const float4*>(bf + q * 4);
+    __nv_bfloat162 o[2] = {__floats2bfloat162_rn(s.x + b.x, s.y + b.y), __floats2bfloat162_rn(s.z + b.z, s.w + b.w)};
+    *reinterpret_cast<uint2*>(y + size_t(t) * d + q * 4) = *reinterpret_cast<const uint2*>(o);
+  }
+}
+
+// Switches the order-independent accumulation of this path on or off; the partial-output buffer is allocated the first time.
+tardis_status_t fused_set_deterministic(Handle* H, bool on) {
+  Scratch* S = static_cast<Scratch*>(H->fscratch);
+  if (!S) return TARDIS_OK;
+  if (on && !S->dpart) {
+    const size_t bytes = size_t(S->base.nkc + S->grid) * MAXT * S->base.dacc * sizeof(float);
+    TARDIS_CUDA_TRY(cudaMalloc(&S->dpart, bytes));
+    H->bytes_scratch += bytes;
+  }
+  return TARDIS_OK;
+}
+
 tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, cudaStream_t s) {
   Scratch* S = static_cast<Scratch*>(H->fscratch);
+  const bool det = H->deterministic && S->dpart;
   for (int t0 = 0; t0 < n;) {
     // calls of 5 to 8 tokens go as two launches of about equal size
     const int left = n - t0;
@@ -1098,6 +1147,7 @@ tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, c
     p.y = static_cast<__nv_bfloat16*>(y) + size_t(t0) * H->d;
     p.dbg_bitmap = H->dbg_bitmap ? H->dbg_bitmap + size_t(t0) * (H->h / 32) : nullptr;
     p.dbg_scores = H->dbg_scores ? H->dbg_scores + size_t(t0) * H->h : nullptr;
+    p.dpart = det ? S->dpart : nullptr;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S->grid); cfg.blockDim = dim3(NTH); cfg.dynamicSmemBytes = S->smem_bytes; cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -1108,6 +1158,12 @@ tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, c
     const bool fast = S->pairs_fit && S->nbuf_n[nt] >= p.tiles_max;
     TARDIS_CUDA_TRY(cudaLaunchKernelExC(&cfg, S->kernels[nt == 1 ? 0 : 1][fast ? 1 : 0], args));
     H->launches += 1;
+    if (det) {
+      const int work = nt * (H->d >> 2);                    // warps
+      k_ordered_sum<<<(work + 3) / 4, 128, 0, s>>>(S->dpart, H->bf, p.y, nt, H->d, p.dacc, p.nkc + S->grid);
+      TARDIS_CUDA_TRY(cudaGetLastError());
+      H->launches += 1;
+    }
     t0 += nt;
   }
   return TARDIS_OK;
@@ -1148,7 +1204,7 @@ tardis_status_t fused_read_stamps(long long* out, int max_ctas) {
 void fused_release(Handle* H) {
   Scratch* S = static_cast<Scratch*>(H->fscratch);
   if (!S) return;
-  void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl, S->Cp};
+  void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl, S->Cp, S->dpart};
   for (void* q : ptrs)
     if (q) cudaFree(q);
   delete S;

@@ -208,6 +208,62 @@ def test_run_to_run_flags_identical():
     T.tardis_destroy(h)
 
 
+@pytest.mark.parametrize("d,h,G", [(512, 2048, 64), (4096, 16384, 128)])
+def test_deterministic_mode_same_bits_run_to_run(d, h, G):
+    """With tardis_set_deterministic on, y of repeated calls is the same bits (fused path at 1, 3, 4 and 9 tokens, batched
+    path at 40 tokens), still agrees with the oracle, and other work in between (a call in the default mode, a call on
+    another handle) does not change it."""
+    cfg = W.LayerConfig("det", d, h, n_calib=512, group=G)
+    L = _layer(cfg)
+    s = L.numpy64()
+    other = T.fold_layer(L)                                  # a second handle of the same layer, left in the default mode
+    hd = T.fold_layer(L)
+    try:
+        T.tardis_set_deterministic(hd, True)
+        for n in (1, 3, 4, 9, 40):
+            x = W.make_tokens(cfg, n, 7 + n).cuda()
+            outs = []
+            for rep in range(4):
+                y = torch.empty_like(x)
+                T.tardis_ffn_forward(hd, x, y)
+                torch.cuda.synchronize()
+                outs.append(y.clone())
+                yo = torch.empty_like(x)
+                T.tardis_ffn_forward(other, x, yo)            # unrelated work between the repetitions
+            for y in outs[1:]:
+                assert torch.equal(y.view(torch.int16), outs[0].view(torch.int16)), "n = %d" % n
+            assert T.tardis_stats(hd)["last_path"] == (2 if n <= 12 else 3)
+            yg, F, S = Hp.gpu_forward(hd, L, x, [n])
+            assert torch.equal(yg.view(torch.int16), outs[0].view(torch.int16))
+            keep = np.arange(n)[: 6]
+            ix = torch.as_tensor(keep).cuda()
+            Hp.assert_parity(L, s, x[ix], yg[ix], F[keep], S[keep], score_tol=3e-4, label="det n=%d" % n)
+        # switching the mode off again gives the default kernels back (same flags, y within the usual tolerance)
+        T.tardis_set_deterministic(hd, False)
+        x = W.make_tokens(cfg, 4, 99).cuda()
+        y0 = torch.empty_like(x); y1 = torch.empty_like(x)
+        T.tardis_ffn_forward(hd, x, y0)
+        T.tardis_ffn_forward(other, x, y1)
+        torch.cuda.synchronize()
+        assert (y0.float() - y1.float()).abs().max() <= 2e-2 * y1.float().abs().max()
+        assert T.tardis_stats(hd)["device_error"] == 0
+    finally:
+        T.tardis_destroy(hd)
+        T.tardis_destroy(other)
+
+
+def test_deterministic_mode_refused_where_only_atomic_kernels_serve():
+    cfg = W.LayerConfig("detf32", 256, 1024, n_calib=512, dtype="f32")
+    L = _layer(cfg)
+    h = T.fold_layer(L)
+    try:
+        with pytest.raises(T.TardisError) as e:
+            T.tardis_set_deterministic(h, True)
+        assert e.value.status == 2
+    finally:
+        T.tardis_destroy(h)
+
+
 def test_batched_path_chunk_boundary_nan_token_and_empty_ranges():
     """More tokens than one scratch chunk in a single call (chunks hold 1024 tokens while the debug capture is on,
     2048 otherwise), a token holding a NaN in the middle of it, and the result compared token by token with the
