@@ -438,6 +438,24 @@ def main():
                                                "layer for its search (Section 7.3, RTX 4090D)" % h}
         del Lf, xcal, zcal
 
+        # a chain of 32 layers on one residual stream (layer normalisation, forward, addition per layer): the bench's
+        # layers four times over, batch 1, once as plain launches and once replayed from a CUDA graph
+        chain = (handles * ((32 + len(handles) - 1) // len(handles)))[:32]
+        xs1, ys1 = x_all[:1].clone(), torch.empty_like(x_all[:1])
+        wk = torch.empty(2, 1, d, dtype=x_all.dtype, device=dev)
+
+        def stack_step():
+            T.tardis_stack_forward(chain, xs1, ys1, None, None, 1e-5, True, True, work=wk)
+        ms_s = timed(stack_step, max(3, args.steps // 2), 3)
+        try:
+            ms_g = timed(stack_step, max(3, args.steps // 2), 3, graph=True)
+        except Exception as e:      # capture refused: reported, not fatal
+            ms_g = None
+            out.setdefault("notes", []).append("stack graph capture failed: %s" % str(e)[:120])
+        out["stack_context"] = {"layers": 32, "batch": 1, "us_per_layer": ms_s * 1e3 / 32,
+                                "us_per_layer_graph": None if ms_g is None else ms_g * 1e3 / 32,
+                                "what": "tardis_stack_forward: per layer k_layernorm, the fused kernel, k_stream_update"}
+
         def dense_step():
             for i in range(NT // B):
                 W1, W2, b1, b2 = dense[i % len(dense)]

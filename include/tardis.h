@@ -267,6 +267,36 @@ tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
  * to such kernels.  tardis_ffn_forward_static does not look at the mode. */
 tardis_status_t tardis_set_deterministic(tardis_handle_t handle, int32_t on);
 
+/* A chain of layers on one residual stream.  The paper replaces the FFN block inside an existing
+ * model (Section 6) and has no call of this kind; this is the shape in which a decoder hands the
+ * FFN blocks of consecutive layers to the library, attention left out:
+ *     s_0 = x;   u_l = normalise ? LayerNorm_l(s_l) : s_l;   f_l = FFN_l(u_l)  (tardis_ffn_forward);
+ *     s_{l+1} = residual ? s_l + f_l : f_l;   y = s_{n_layers}.
+ * LayerNorm_l(v)[i] = (v[i] - mean(v)) / sqrt(var(v) + ln_eps) * gamma_l[i] + beta_l[i], mean and
+ * variance (divisor d_model) over the token's row, computed in fp32 and rounded to the layers' dtype;
+ * s_l + f_l is added in fp32 and rounded to the dtype once per layer.
+ *   layers    host array of n_layers handles of the same d_model, dtype and device (each keeps its own
+ *             path choice, capture and accumulation mode);
+ *   ln_gamma, ln_beta   host arrays of n_layers device pointers to [d_model] fp32, or NULL (1 and 0);
+ *   x, y      device [n_tokens, d_model] in the layers' dtype, 16-byte aligned; y may be x (in place);
+ *   work      device scratch of at least 2 n_tokens d_model elements, caller-owned (the call allocates
+ *             nothing); ignored when keep is given;
+ *   keep      NULL, or device [n_layers][2][n_tokens, d_model]: u_l and f_l of every layer stay there
+ *             for the caller to look at (tests compare each layer with the oracle on that layer's input).
+ * Everything is enqueued on `stream`; d_model up to 12288.  Errors: INVALID_ARG for a bad descriptor,
+ * mismatched layers, a missing or small buffer; otherwise what tardis_ffn_forward returns. */
+typedef struct {
+  int32_t n_layers;
+  const tardis_handle_t* layers;
+  int32_t normalise;               /* 1: layer normalisation before every layer */
+  const float* const* ln_gamma;
+  const float* const* ln_beta;
+  float ln_eps;
+  int32_t residual;                /* 1: s_{l+1} = s_l + f_l; 0: s_{l+1} = f_l */
+} tardis_stack_desc_t;
+tardis_status_t tardis_stack_forward(const tardis_stack_desc_t* desc, const void* x, void* y, void* work, size_t work_bytes,
+                                     void* keep, size_t keep_bytes, int64_t n_tokens, tardis_stream_t stream);
+
 /* Profiling aid of the fused decode kernel (the online path of Section 5.4 as one launch).  A library
  * built with -DTARDIS_PHASE_STAMPS (python -m paper_2501_10054_b200.build --stamps) makes every CTA of that
  * kernel record the GPU's global nanosecond timer at its phase boundaries; this call synchronises the

@@ -449,3 +449,35 @@ def neuron_thresholds(err, t_layer, t_min, t_max):
         if budget <= 0.0:
             break
     return t
+
+
+# ---- a chain of layers on one residual stream (no counterpart in the paper: the stack call of the library) ----
+def layer_norm(v, gamma=None, beta=None, eps=1e-5):
+    """Layer normalisation of every row of v[n, d] by its definition: subtract the row's mean, divide by the square
+    root of the row's variance (divisor d) plus eps, multiply by gamma[d] and add beta[d] (1 and 0 when absent)."""
+    v = _as64(v)
+    d = v.shape[-1]
+    out = np.empty_like(v)
+    for t in range(v.shape[0]):
+        mean = v[t].sum() / d
+        var = ((v[t] - mean) ** 2).sum() / d
+        out[t] = (v[t] - mean) / math.sqrt(var + eps)
+    if gamma is not None:
+        out = out * _as64(gamma)[None, :]
+    if beta is not None:
+        out = out + _as64(beta)[None, :]
+    return out
+
+
+def stack_forward(x, ffns, gammas=None, betas=None, eps=1e-5, normalise=True, residual=True):
+    """s_0 = x; u_l = layer_norm(s_l) or s_l; f_l = ffns[l](u_l); s_{l+1} = s_l + f_l or f_l.  Returns s_L and the
+    lists of u_l and f_l.  `ffns` are callables [n, d] -> [n, d] (a layer's partially linear forward)."""
+    s = _as64(x)
+    us, fs = [], []
+    for l, ffn in enumerate(ffns):
+        u = layer_norm(s, None if gammas is None else gammas[l], None if betas is None else betas[l], eps) if normalise else s
+        f = _as64(ffn(u))
+        us.append(u)
+        fs.append(f)
+        s = s + f if residual else f
+    return s, us, fs

@@ -21,7 +21,7 @@ TARDIS_F32, TARDIS_BF16 = 0, 1
 TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
-           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_set_deterministic", "tardis_destroy", "tardis_calibrate",
+           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_set_deterministic", "tardis_stack_forward", "tardis_destroy", "tardis_calibrate",
            "tardis_debug_phase_stamps", "tardis_range_search", "tardis_debug_wait_timeout", "tardis_clear_error",
            "tardis_save", "tardis_load", "tardis_status_string", "tardis_last_error"]
 
@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_export_folded.argtypes = [vp, vp, vp, vp]
     lib.tardis_set_path.argtypes = [vp, i32]
     lib.tardis_set_deterministic.argtypes = [vp, i32]
+    lib.tardis_stack_forward.argtypes = [vp, vp, vp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, ctypes.c_int64, vp]
     lib.tardis_destroy.argtypes = [vp]
     lib.tardis_gemm_bf16.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, i32, vp]
     lib.tardis_calibrate.argtypes = [i32, i32, vp, i64, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp]
@@ -83,7 +84,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_clear_error.argtypes = [vp]
     lib.tardis_save.argtypes = [vp, ctypes.c_char_p]
     lib.tardis_load.argtypes = [ctypes.c_char_p, vp, ctypes.POINTER(vp)]
-    for name in EXPORTS[:16]:
+    for name in EXPORTS[:-2]:
         getattr(lib, name).restype = ctypes.c_int
     lib.tardis_status_string.argtypes = [ctypes.c_int]
     lib.tardis_status_string.restype = ctypes.c_char_p
@@ -236,6 +237,32 @@ def tardis_debug_wait_timeout(handle: int, limit_cycles: int, stream=None):
 
 def tardis_clear_error(handle: int):
     _check(load_library().tardis_clear_error(handle), "tardis_clear_error")
+
+
+class StackDesc(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("layers", ctypes.POINTER(ctypes.c_void_p)), ("normalise", ctypes.c_int32),
+                ("ln_gamma", ctypes.POINTER(ctypes.c_void_p)), ("ln_beta", ctypes.POINTER(ctypes.c_void_p)),
+                ("ln_eps", ctypes.c_float), ("residual", ctypes.c_int32)]
+
+
+def tardis_stack_forward(handles, x: torch.Tensor, y: torch.Tensor, gammas=None, betas=None, eps: float = 1e-5,
+                         normalise: bool = True, residual: bool = True, work: Optional[torch.Tensor] = None,
+                         keep: Optional[torch.Tensor] = None, stream=None):
+    """The layers `handles` chained on one residual stream (see tardis_stack_forward in tardis.h).  `work` is scratch of
+    2 n d elements in x's dtype (made here when neither it nor `keep` is given: the C call itself allocates nothing);
+    `keep` [n_layers, 2, n, d] receives every layer's input and output."""
+    L = len(handles)
+    arr = (ctypes.c_void_p * L)(*handles)
+    ga = (ctypes.c_void_p * L)(*[_ptr(g) for g in gammas]) if gammas is not None else None
+    be = (ctypes.c_void_p * L)(*[_ptr(b) for b in betas]) if betas is not None else None
+    desc = StackDesc(L, arr, 1 if normalise else 0, ga, be, eps, 1 if residual else 0)
+    n = x.shape[0]
+    if work is None and keep is None:
+        work = torch.empty(2, *x.shape, dtype=x.dtype, device=x.device)
+    wb = work.numel() * work.element_size() if work is not None else 0
+    kb = keep.numel() * keep.element_size() if keep is not None else 0
+    _check(load_library().tardis_stack_forward(ctypes.byref(desc), _ptr(x), _ptr(y), _ptr(work), wb, _ptr(keep), kb, n,
+                                               _stream(stream)), "tardis_stack_forward")
 
 
 def tardis_save(handle: int, path: str):

@@ -403,6 +403,29 @@ tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_han
   return TARDIS_OK;
 }
 
+tardis_status_t tardis_stack_forward(const tardis_stack_desc_t* desc, const void* x, void* y, void* work, size_t work_bytes,
+                                     void* keep, size_t keep_bytes, int64_t n_tokens, tardis_stream_t stream) {
+  if (!desc || desc->n_layers < 1 || !desc->layers || n_tokens < 0) return TARDIS_ERR_INVALID_ARG;
+  if (!(desc->residual == 0 || desc->residual == 1) || !(desc->normalise == 0 || desc->normalise == 1)) return TARDIS_ERR_INVALID_ARG;
+  if (desc->normalise && !(desc->ln_eps >= 0.f)) return TARDIS_ERR_INVALID_ARG;
+  Handle* H0 = check(desc->layers[0]);
+  if (!H0 || !on_handle_device(H0)) return TARDIS_ERR_INVALID_ARG;
+  for (int l = 0; l < desc->n_layers; ++l) {
+    Handle* H = check(desc->layers[l]);
+    if (!H || H->d != H0->d || H->dtype != H0->dtype || H->device != H0->device) return TARDIS_ERR_INVALID_ARG;
+    if (desc->normalise && ((desc->ln_gamma && !desc->ln_gamma[l]) || (desc->ln_beta && !desc->ln_beta[l]))) return TARDIS_ERR_INVALID_ARG;
+  }
+  if (n_tokens == 0) return TARDIS_OK;
+  if (!x || !y || !aligned16(x) || !aligned16(y)) return TARDIS_ERR_INVALID_ARG;
+  const size_t count = size_t(n_tokens) * H0->d * H0->esize;
+  if (keep) {
+    if (!aligned16(keep) || keep_bytes < size_t(2) * desc->n_layers * count) return TARDIS_ERR_INVALID_ARG;
+  } else if (!work || !aligned16(work) || work_bytes < 2 * count) {
+    return TARDIS_ERR_INVALID_ARG;
+  }
+  return launch_stack_forward(desc, x, y, work, keep, n_tokens, reinterpret_cast<cudaStream_t>(stream));
+}
+
 tardis_status_t tardis_set_deterministic(tardis_handle_t handle, int32_t on) {
   Handle* H = check(handle);
   if (!H || !(on == 0 || on == 1)) return TARDIS_ERR_INVALID_ARG;

@@ -85,6 +85,8 @@ tardis_status_t batched_prepare(Handle* H);                                     
 tardis_status_t batched_finish(Handle* H, const void* W2, cudaStream_t s);   // fills the batched state (W2 null: from W2T)
 tardis_status_t launch_batched_forward(Handle* H, const void* x, void* y, int64_t n, cudaStream_t s);
 void batched_release(Handle* H);
+tardis_status_t launch_stack_forward(const tardis_stack_desc_t* desc, const void* x, void* y, void* work, void* keep, int64_t n,
+                                     cudaStream_t s);   // stack.cu; arguments checked by the caller
 tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);  // bf16 fold on the tensor cores
 
 // ---- small device helpers ----

@@ -264,6 +264,64 @@ def test_deterministic_mode_refused_where_only_atomic_kernels_serve():
         T.tardis_destroy(h)
 
 
+@pytest.mark.parametrize("n,normalise,residual", [(1, True, True), (5, True, True), (40, True, True), (3, False, True), (4, True, False)])
+def test_stack_forward_layer_by_layer_against_the_oracle(n, normalise, residual):
+    """Three independently seeded layers chained on one stream.  With `keep`, every layer's input u_l and output f_l
+    are read back: u_l against the oracle's layer normalisation of the stream the GPU itself had (rebuilt from the
+    kept outputs, so that a flag that flips downstream of a bf16 rounding does not hide a layer's error), f_l against
+    the oracle's forward on exactly u_l (flags and scores captured per layer), the final stream against the rounded
+    sums.  The same call without `keep` (two work buffers in turns) gives the same y."""
+    cfg = W.LayerConfig("stack", 512, 2048, n_calib=512)
+    Ls = [_layer(cfg, seed=10 + l) for l in range(3)]
+    hs = [T.fold_layer(L) for L in Ls]
+    g = torch.Generator().manual_seed(3)
+    gammas = [(1.0 + 0.1 * torch.randn(512, generator=g)).cuda() for _ in Ls]
+    betas = [(0.1 * torch.randn(512, generator=g)).cuda() for _ in Ls]
+    x = W.make_tokens(cfg, n, 21).cuda()
+    try:
+        caps = []
+        for h in hs:
+            bm = torch.zeros(n, 2048 // 32, dtype=torch.int32, device="cuda")
+            sc = torch.full((n, 2048), float("nan"), dtype=torch.float64, device="cuda")
+            T.tardis_set_debug_capture(h, bm, sc)
+            caps.append((bm, sc))
+        keep = torch.full((3, 2, n, 512), float("nan"), dtype=x.dtype, device="cuda")
+        y = torch.empty_like(x)
+        T.tardis_stack_forward(hs, x, y, gammas, betas, 1e-5, normalise, residual, keep=keep)
+        torch.cuda.synchronize()
+        for h in hs:
+            T.tardis_set_debug_capture(h, None, None)
+        stream = x.clone()
+        for l, L in enumerate(Ls):
+            u, f = keep[l, 0], keep[l, 1]
+            if normalise:
+                ref_u = O.layer_norm(stream.double().cpu().numpy(), gammas[l].double().cpu().numpy(), betas[l].double().cpu().numpy(), 1e-5)
+                err = np.abs(u.double().cpu().numpy() - ref_u)
+                assert (err <= 2.0 ** -8 * np.abs(ref_u) + 1e-6).all(), "layer %d: normalisation off by %.3e" % (l, err.max())
+            else:
+                assert torch.equal(u, stream)
+            F = Hp.unpack_bitmap(caps[l][0], 2048)
+            S = caps[l][1].cpu().numpy()
+            Hp.assert_parity(L, L.numpy64(), u, f, F, S, score_tol=3e-4, label="stack layer %d" % l)
+            stream = (stream.float() + f.float()).to(x.dtype) if residual else f.clone()
+        assert torch.equal(y, stream)
+        # without keep: same result from the two work buffers; in place as well
+        y2 = torch.empty_like(x)
+        T.tardis_stack_forward(hs, x, y2, gammas, betas, 1e-5, normalise, residual)
+        x3 = x.clone()
+        T.tardis_stack_forward(hs, x3, x3, gammas, betas, 1e-5, normalise, residual)
+        torch.cuda.synchronize()
+        tol = 2e-2 * float(y.float().abs().max())
+        assert float((y2.float() - y.float()).abs().max()) <= tol and float((x3.float() - y.float()).abs().max()) <= tol
+        # a buffer that is too small is refused
+        with pytest.raises(T.TardisError) as e:
+            T.tardis_stack_forward(hs, x, y2, gammas, betas, 1e-5, normalise, residual, work=torch.empty(n * 512, dtype=x.dtype, device="cuda"))
+        assert e.value.status == 1
+    finally:
+        for h in hs:
+            T.tardis_destroy(h)
+
+
 def test_batched_path_chunk_boundary_nan_token_and_empty_ranges():
     """More tokens than one scratch chunk in a single call (chunks hold 1024 tokens while the debug capture is on,
     2048 otherwise), a token holding a NaN in the middle of it, and the result compared token by token with the

@@ -524,3 +524,44 @@ def test_neuron_thresholds_against_library_lp():
     np.testing.assert_allclose(t, lp.x, atol=1e-7)
     # the neurons with the largest error keep the lowest threshold
     assert t[np.argmax(err)] == 0.6 and t[np.argmin(err)] == 0.95
+
+
+def test_layer_norm_and_stack_against_library_and_closed_forms():
+    """layer_norm: the library routine of torch on the same rows (another implementation), rows of known statistics
+    (a row a + b k normalises to the standardised ramp whatever a and b > 0 are; a constant row gives beta), invariance
+    under shift and positive scaling of the input (eps = 0), mean 0 / variance 1 of the output.  stack_forward: linear
+    stand-in layers give a closed form (residual: product of (I + M_l); none: product of M_l), and the kept inputs and
+    outputs are consistent with the final stream."""
+    import torch
+    rng = np.random.default_rng(5)
+    v = rng.standard_normal((7, 48)) * 3 + 1.5
+    g, b = rng.standard_normal(48), rng.standard_normal(48)
+    ref = torch.nn.functional.layer_norm(torch.from_numpy(v), (48,), torch.from_numpy(g), torch.from_numpy(b), 1e-5).numpy()
+    np.testing.assert_allclose(O.layer_norm(v, g, b, 1e-5), ref, rtol=1e-12, atol=1e-12)
+    out = O.layer_norm(v, None, None, 0.0)
+    np.testing.assert_allclose(out.mean(axis=1), 0.0, atol=1e-13)
+    np.testing.assert_allclose((out ** 2).mean(axis=1), 1.0, rtol=1e-12)
+    np.testing.assert_allclose(O.layer_norm(4.0 * v - 9.0, None, None, 0.0), out, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(O.layer_norm(-v, None, None, 0.0), -out, rtol=1e-12, atol=1e-13)   # a sign error in the centring shows here
+    k = np.arange(9.0)
+    ramp = (k - 4.0) / math.sqrt(60.0 / 9.0)                       # mean 4, variance (sum (k-4)^2)/9 = 60/9
+    np.testing.assert_allclose(O.layer_norm((2.0 + 0.5 * k)[None, :], None, None, 0.0)[0], ramp, rtol=1e-12)
+    np.testing.assert_allclose(O.layer_norm(np.full((1, 9), 3.0), g[:9], b[:9], 1e-5)[0], b[:9], atol=1e-12)
+    # eps enters under the root: variance 60/9, eps 1 -> divisor sqrt(60/9 + 1)
+    np.testing.assert_allclose(O.layer_norm(k[None, :], None, None, 1.0)[0], (k - 4.0) / math.sqrt(60.0 / 9.0 + 1.0), rtol=1e-12)
+
+    Ms = [rng.standard_normal((6, 6)) * 0.3 for _ in range(3)]
+    ffns = [lambda u, M=M: u @ M.T for M in Ms]
+    x = rng.standard_normal((4, 6))
+    y, us, fs = O.stack_forward(x, ffns, normalise=False, residual=True)
+    P = np.eye(6)
+    for M in Ms:
+        P = (np.eye(6) + M) @ P
+    np.testing.assert_allclose(y, x @ P.T, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(y, x + fs[0] + fs[1] + fs[2], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(us[1], x + fs[0], rtol=1e-12, atol=1e-12)
+    y2, _, _ = O.stack_forward(x, ffns, normalise=False, residual=False)
+    np.testing.assert_allclose(y2, x @ (Ms[2] @ Ms[1] @ Ms[0]).T, rtol=1e-12, atol=1e-12)
+    y3, us3, fs3 = O.stack_forward(x, ffns, gammas=[g[:6]] * 3, betas=[b[:6]] * 3, eps=1e-5, normalise=True, residual=True)
+    np.testing.assert_allclose(us3[2], O.layer_norm(x + fs3[0] + fs3[1], g[:6], b[:6], 1e-5), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(fs3[2], us3[2] @ Ms[2].T, rtol=1e-12, atol=1e-12)
