@@ -481,3 +481,69 @@ def stack_forward(x, ffns, gammas=None, betas=None, eps=1e-5, normalise=True, re
         fs.append(f)
         s = s + f if residual else f
     return s, us, fs
+
+
+# ---- building the predictor: quantisation of W1 with error compensation (Section 6: "GPTQ with 2-bit precision") ----
+def round_to_storage(v, dtype):
+    """The value a float64 number takes when stored as `dtype` ("f32" or "bf16"): rounded to nearest-even to float32, and
+    for bf16 rounded once more, to nearest-even, to the upper 16 bits of the float32 word (finite values)."""
+    f = np.asarray(v, dtype=np.float64).astype(np.float32)
+    if dtype == "f32":
+        return f.astype(np.float64)
+    u = f.view(np.uint32).astype(np.uint64)
+    u = (u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))) & np.uint64(0xFFFF0000)
+    return u.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def group_grid(wg, bits, dtype):
+    """Asymmetric uniform grid of one group of weights wg[..., G]: the range [min, max] widened to contain 0, the scale
+    (max - min) / (2^bits - 1) rounded to its storage type before anything else uses it (1 if that is 0), the zero-point
+    round(-min / scale) clamped to the code range.  Returns (scale, zero)."""
+    levels = (1 << bits) - 1
+    wmin = np.minimum(wg.min(axis=-1), 0.0)
+    wmax = np.maximum(wg.max(axis=-1), 0.0)
+    scale = round_to_storage((wmax - wmin) / levels, dtype)
+    scale = np.where(scale > 0.0, scale, 1.0)
+    zero = np.clip(np.rint(-wmin / scale), 0, levels)
+    return scale, zero
+
+
+def gptq_quantise(W1, U, group, bits=2, dtype="bf16"):
+    """Quantisation of W1[h, d] with the error of every rounded channel spread over the channels not yet rounded (the
+    GPTQ procedure the paper uses for its predictor).  U[d, d] is the upper Cholesky factor of the inverse Hessian of the
+    layer's inputs (U^T U = H^-1); U = None stands for the identity, which leaves plain rounding to nearest.
+
+    Channels go in ascending order.  When channel k opens a group, the group's grid comes from the weights as they are at
+    that moment (earlier errors already spread into them).  Then q_k = clip(rint(w_k / s + z)), the error
+    e_k = (w_k - s (q_k - z)) / U[k, k], and every later channel j > k takes w_j <- w_j - e_k U[k, j].
+    Returns (q uint8 [h, d], scale [h, d/G], zero [h, d/G], E [h, d] the errors e_k)."""
+    W = _as64(W1).copy()
+    h, d = W.shape
+    levels = (1 << bits) - 1
+    q = np.empty((h, d), dtype=np.uint8)
+    E = np.empty((h, d))
+    scale = np.empty((h, d // group))
+    zero = np.empty((h, d // group))
+    for k in range(d):
+        g = k // group
+        if k % group == 0:
+            scale[:, g], zero[:, g] = group_grid(W[:, k:k + group], bits, dtype)
+        qk = np.clip(np.rint(W[:, k] / scale[:, g] + zero[:, g]), 0, levels)
+        q[:, k] = qk.astype(np.uint8)
+        ukk = 1.0 if U is None else U[k, k]
+        E[:, k] = (W[:, k] - scale[:, g] * (qk - zero[:, g])) / ukk
+        if U is not None and k + 1 < d:
+            W[:, k + 1:] -= E[:, k][:, None] * U[k, k + 1:][None, :]
+    return q, scale, zero, E
+
+
+def pack_codes(q, bits=2):
+    """The inverse of unpack_codes: [h, d] codes into [h, d bits / 32] 32-bit words, channel order ascending, lowest bits
+    first."""
+    q = np.asarray(q, dtype=np.uint64)
+    per = 32 // bits
+    h, d = q.shape
+    words = np.zeros((h, d // per), dtype=np.uint64)
+    for p in range(per):
+        words |= q[:, p::per] << np.uint64(bits * p)
+    return words.astype(np.uint32)

@@ -565,3 +565,58 @@ def test_layer_norm_and_stack_against_library_and_closed_forms():
     y3, us3, fs3 = O.stack_forward(x, ffns, gammas=[g[:6]] * 3, betas=[b[:6]] * 3, eps=1e-5, normalise=True, residual=True)
     np.testing.assert_allclose(us3[2], O.layer_norm(x + fs3[0] + fs3[1], g[:6], b[:6], 1e-5), rtol=1e-12, atol=1e-12)
     np.testing.assert_allclose(fs3[2], us3[2] @ Ms[2].T, rtol=1e-12, atol=1e-12)
+
+
+def test_gptq_quantise_identities_and_special_cases():
+    """round_to_storage against torch's conversions (another implementation of the same format); group_grid on a hand
+    example; gptq_quantise: with U = identity it is rounding to nearest on the group's grid (and the errors are the plain
+    residuals); with a general U the recorded errors reproduce the result exactly through W - E U = dequantised codes
+    (the defining recurrence unrolled: a wrong sign, a wrong row of U or an off-by-one in `later channels` breaks it);
+    a two-channel case worked by hand; on correlated inputs the output error ||X (W - What)^T|| is smaller than with
+    plain rounding (what the procedure is for); pack_codes inverts unpack_codes."""
+    import torch
+    rng = np.random.default_rng(11)
+    v = np.concatenate([rng.standard_normal(4000) * 10.0 ** rng.integers(-6, 6, 4000), [0.0, 1.0, -2.5, 3.0e-39]])
+    np.testing.assert_array_equal(O.round_to_storage(v, "bf16"), torch.from_numpy(v).float().bfloat16().double().numpy())
+    np.testing.assert_array_equal(O.round_to_storage(v, "f32"), torch.from_numpy(v).float().double().numpy())
+    # grid by hand: weights -1 .. 2, 2 bits: scale 1, zero 1; all positive 0.5 .. 2: range widened to 0: scale 2/3 -> bf16
+    s, z = O.group_grid(np.array([[-1.0, 0.25, 2.0, 1.0]]), 2, "f32")
+    assert s[0] == 1.0 and z[0] == 1.0
+    s, z = O.group_grid(np.array([[0.5, 2.0, 1.0, 1.5]]), 2, "bf16")
+    assert s[0] == 0.66796875 and z[0] == 0.0                       # 2/3 in bf16 = 171 / 256
+    s, z = O.group_grid(np.zeros((1, 4)), 2, "bf16")
+    assert s[0] == 1.0 and z[0] == 0.0
+
+    h, d, G = 6, 32, 16
+    W = rng.standard_normal((h, d))
+    q, sc, zp, E = O.gptq_quantise(W, None, G, 2, "f32")
+    for j in range(h):
+        for g in range(d // G):
+            wg = W[j, g * G:(g + 1) * G]
+            s_, z_ = O.group_grid(wg[None, :], 2, "f32")
+            np.testing.assert_array_equal(q[j, g * G:(g + 1) * G], np.clip(np.rint(wg / s_[0] + z_[0]), 0, 3))
+    deq = (q.reshape(h, d // G, G) - zp[:, :, None]) * sc[:, :, None]
+    np.testing.assert_allclose(E, W - deq.reshape(h, d), rtol=0, atol=1e-15)
+
+    X = rng.standard_normal((200, d)) @ (np.eye(d) + 0.6 * rng.standard_normal((d, d)))      # correlated channels
+    H = 2.0 / 200 * X.T @ X + 0.01 * np.mean(np.diag(2.0 / 200 * X.T @ X)) * np.eye(d)
+    U = np.linalg.cholesky(np.linalg.inv(H)).T                                                   # upper: U^T U = H^-1
+    np.testing.assert_allclose(U.T @ U, np.linalg.inv(H), rtol=1e-9, atol=1e-12)
+    q2, sc2, zp2, E2 = O.gptq_quantise(W, U, G, 2, "f32")
+    deq2 = ((q2.reshape(h, d // G, G) - zp2[:, :, None]) * sc2[:, :, None]).reshape(h, d)
+    np.testing.assert_allclose(W - E2 @ np.triu(U), deq2, rtol=1e-10, atol=1e-10)
+    err_rtn = np.linalg.norm(X @ (W - deq.reshape(h, d)).T)
+    err_gptq = np.linalg.norm(X @ (W - deq2).T)
+    assert err_gptq < 0.9 * err_rtn, (err_gptq, err_rtn)
+    # two channels, one group, by hand: w = (0.9, 1.4), 2 bits, range [0, 1.4] -> scale 1.4/3, zero 0;
+    # q0 = rint(0.9 / s) = 2, e0 = (0.9 - 2 s) / u00, w1 <- 1.4 - e0 u01, q1 = rint(w1 / s)
+    U2 = np.array([[2.0, 0.5], [0.0, 1.0]])
+    qh, sh, zh, Eh = O.gptq_quantise(np.array([[0.9, 1.4]]), U2, 2, 2, "f32")
+    s_ = float(np.float32(1.4 / 3))
+    e0 = (0.9 - 2 * s_) / 2.0
+    w1 = 1.4 - e0 * 0.5
+    assert sh[0, 0] == s_ and zh[0, 0] == 0 and qh[0, 0] == 2 and qh[0, 1] == int(np.rint(w1 / s_))
+    np.testing.assert_allclose(Eh[0], [e0, (w1 - s_ * qh[0, 1]) / 1.0], rtol=1e-15)
+    for bits in (2, 4, 8):
+        qq = rng.integers(0, 1 << bits, (5, 64)).astype(np.uint8)
+        np.testing.assert_array_equal(O.unpack_codes(O.pack_codes(qq, bits), 64, bits), qq)
