@@ -436,7 +436,17 @@ def main():
         out["range_search_context"] = {"ms_per_layer": msr, "n_cal": ncal, "threshold": 0.85, "step": 0.05,
                                        "what": "Algorithm 1 per neuron on the GPU, %d neurons; the paper reports about 30 minutes per "
                                                "layer for its search (Section 7.3, RTX 4090D)" % h}
-        del Lf, xcal, zcal
+        # the predictor by error-compensated quantisation (GPTQ, Section 6): Hessian and its Cholesky factors by torch's
+        # routines (the caller's side), the channel-by-channel rounding of all neurons by tardis_build_predictor
+        Xd = xcal.double()
+        Hm = 2.0 / ncal * Xd.t() @ Xd
+        Hm += 0.01 * torch.mean(torch.diagonal(Hm)) * torch.eye(d, dtype=torch.float64, device=dev)
+        Um = torch.linalg.cholesky(torch.cholesky_inverse(torch.linalg.cholesky(Hm)), upper=True).contiguous()
+        msb = timed(lambda: T.tardis_build_predictor(Lf.W1, Um, cfg.bits, cfg.group), 2, 1)
+        out["predictor_build_context"] = {"ms_per_layer": msb, "bits": cfg.bits, "group": cfg.group,
+                                          "what": "tardis_build_predictor on %d x %d weights, double precision, scratch allocation "
+                                                  "and release included; the Hessian's factor is an input" % (h, d)}
+        del Lf, xcal, zcal, Xd, Hm, Um
 
         # a chain of 32 layers on one residual stream (layer normalisation, forward, addition per layer): the bench's
         # layers four times over, batch 1, once as plain launches and once replayed from a CUDA graph

@@ -267,6 +267,27 @@ tardis_status_t tardis_set_path(tardis_handle_t handle, int32_t path);
  * to such kernels.  tardis_ffn_forward_static does not look at the mode. */
 tardis_status_t tardis_set_deterministic(tardis_handle_t handle, int32_t on);
 
+/* Offline: the predictor of a layer, built on the GPU.  The paper obtains its predictor by GPTQ with 2-bit precision
+ * (Section 6; Section 5.3 for what the predictor is, Section 7.6 for other widths).  Per neuron, channels in ascending
+ * order: when channel k opens a group, the group's grid is taken from the weights as they are then (range widened to
+ * contain 0; scale = (max - min) / (2^bits - 1) rounded to `dtype`, 1 if that is 0; zero-point = round(-min / scale)
+ * clamped to the code range); q_k = clip(round(w_k / scale + zero)); e_k = (w_k - scale (q_k - zero)) / U[k][k]; every
+ * later channel takes w_j <- w_j - e_k U[k][j].  Rounding is to nearest-even, all arithmetic is double precision with
+ * separately rounded products and differences, so the codes are those of a plain double-precision implementation.
+ *   W1     device [d_ff, d_model] row-major in `dtype`;
+ *   U      device double [d_model, d_model] row-major, the upper Cholesky factor of the inverse Hessian of the layer's
+ *          inputs (U^T U = H^-1, H = (2/N) X^T X plus damping: made by the caller, e.g. with a library Cholesky), only
+ *          its upper triangle is read; NULL = identity, which gives plain rounding to nearest;
+ *   bits   2, 4 or 8; group a multiple of 64 that divides d_model;
+ *   codes  out, device [d_ff, d_model bits / 32] (channel order ascending, lowest bits first);
+ *   scale  out, device [d_ff, d_model / group] in `dtype`; zero out, device bytes of the same shape.
+ * The outputs are what tardis_fold_desc_t takes as pred_codes, pred_scale, pred_zero.  The call allocates its scratch
+ * (8 d_ff d_model bytes and a little more), runs on `stream` and returns after the stream has finished the work.
+ * Errors: INVALID_ARG, ALLOC, CUDA. */
+tardis_status_t tardis_build_predictor(int32_t d_ff, int32_t d_model, tardis_dtype_t dtype, const void* W1, const double* U,
+                                       int32_t bits, int32_t group, uint32_t* codes, void* scale, uint8_t* zero,
+                                       tardis_stream_t stream);
+
 /* A chain of layers on one residual stream.  The paper replaces the FFN block inside an existing
  * model (Section 6) and has no call of this kind; this is the shape in which a decoder hands the
  * FFN blocks of consecutive layers to the library, attention left out:

@@ -21,7 +21,7 @@ TARDIS_F32, TARDIS_BF16 = 0, 1
 TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
-           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_set_deterministic", "tardis_stack_forward", "tardis_destroy", "tardis_calibrate",
+           "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_set_deterministic", "tardis_stack_forward", "tardis_build_predictor", "tardis_destroy", "tardis_calibrate",
            "tardis_debug_phase_stamps", "tardis_range_search", "tardis_debug_wait_timeout", "tardis_clear_error",
            "tardis_save", "tardis_load", "tardis_status_string", "tardis_last_error"]
 
@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_export_folded.argtypes = [vp, vp, vp, vp]
     lib.tardis_set_path.argtypes = [vp, i32]
     lib.tardis_set_deterministic.argtypes = [vp, i32]
+    lib.tardis_build_predictor.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.tardis_stack_forward.argtypes = [vp, vp, vp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, ctypes.c_int64, vp]
     lib.tardis_destroy.argtypes = [vp]
     lib.tardis_gemm_bf16.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, i32, vp]
@@ -237,6 +238,21 @@ def tardis_debug_wait_timeout(handle: int, limit_cycles: int, stream=None):
 
 def tardis_clear_error(handle: int):
     _check(load_library().tardis_clear_error(handle), "tardis_clear_error")
+
+
+def tardis_build_predictor(W1: torch.Tensor, U: Optional[torch.Tensor], bits: int, group: int, stream=None):
+    """Predictor of a layer by error-compensated quantisation on the GPU (see tardis_build_predictor in tardis.h).
+    W1 [h, d] float32 or bfloat16, U [d, d] float64 upper Cholesky factor of the inverse Hessian (None: round to nearest).
+    Returns (codes int32 [h, d bits / 32], scale [h, d / group] in W1's dtype, zero uint8 [h, d / group])."""
+    h, d = W1.shape
+    if not W1.is_contiguous() or (U is not None and (U.dtype != torch.float64 or not U.is_contiguous() or tuple(U.shape) != (d, d))):
+        raise TardisError(1, "W1 must be contiguous and U a contiguous float64 [d, d] tensor")
+    codes = torch.empty(h, d * bits // 32, dtype=torch.int32, device=W1.device)
+    scale = torch.empty(h, d // group, dtype=W1.dtype, device=W1.device)
+    zero = torch.empty(h, d // group, dtype=torch.uint8, device=W1.device)
+    _check(load_library().tardis_build_predictor(h, d, _dtype_code(W1.dtype), _ptr(W1), _ptr(U), bits, group, _ptr(codes),
+                                                 _ptr(scale), _ptr(zero), _stream(stream)), "tardis_build_predictor")
+    return codes, scale, zero
 
 
 class StackDesc(ctypes.Structure):

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtardis.so")
 LIB_STAMPS = os.path.join(PKG, "libtardis_stamps.so")
-SOURCES = ["api.cu", "fold.cu", "generic.cu", "decode.cu", "fused.cu", "gemm.cu", "batched.cu", "calibrate.cu", "stack.cu"]
+SOURCES = ["api.cu", "fold.cu", "generic.cu", "decode.cu", "fused.cu", "gemm.cu", "batched.cu", "calibrate.cu", "stack.cu", "gptq.cu"]
 
 
 def nvcc_path() -> str:

@@ -403,6 +403,14 @@ tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_han
   return TARDIS_OK;
 }
 
+tardis_status_t tardis_build_predictor(int32_t d_ff, int32_t d_model, tardis_dtype_t dtype, const void* W1, const double* U,
+                                       int32_t bits, int32_t group, uint32_t* codes, void* scale, uint8_t* zero, tardis_stream_t stream) {
+  if (d_ff < 1 || d_model < 1 || !W1 || !codes || !scale || !zero) return TARDIS_ERR_INVALID_ARG;
+  if (!(dtype == TARDIS_F32 || dtype == TARDIS_BF16) || !(bits == 2 || bits == 4 || bits == 8)) return TARDIS_ERR_INVALID_ARG;
+  if (group < 64 || group % 64 || d_model % group) return TARDIS_ERR_INVALID_ARG;
+  return launch_build_predictor(d_ff, d_model, dtype, W1, U, bits, group, codes, scale, zero, reinterpret_cast<cudaStream_t>(stream));
+}
+
 tardis_status_t tardis_stack_forward(const tardis_stack_desc_t* desc, const void* x, void* y, void* work, size_t work_bytes,
                                      void* keep, size_t keep_bytes, int64_t n_tokens, tardis_stream_t stream) {
   if (!desc || desc->n_layers < 1 || !desc->layers || n_tokens < 0) return TARDIS_ERR_INVALID_ARG;

@@ -87,6 +87,8 @@ tardis_status_t launch_batched_forward(Handle* H, const void* x, void* y, int64_
 void batched_release(Handle* H);
 tardis_status_t launch_stack_forward(const tardis_stack_desc_t* desc, const void* x, void* y, void* work, void* keep, int64_t n,
                                      cudaStream_t s);   // stack.cu; arguments checked by the caller
+tardis_status_t launch_build_predictor(int h, int d, int dtype, const void* W1, const double* U, int bits, int G, uint32_t* codes,
+                                       void* scale, uint8_t* zero, cudaStream_t s);   // gptq.cu; arguments checked by the caller
 tardis_status_t launch_fold_tensor(Handle* H, const tardis_fold_desc_t* desc, cudaStream_t s);  // bf16 fold on the tensor cores
 
 // ---- small device helpers ----

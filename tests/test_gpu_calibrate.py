@@ -210,3 +210,84 @@ def test_greedy_range_search_full_layer_shape_sampled():
     assert torch.equal(lo_s, lo[sel]) and torch.equal(hi_s, hi[sel])
     cov = ((zcal + L.b1[:, None] >= lo[:, None]) & (zcal + L.b1[:, None] < hi[:, None])).float().mean(dim=1)
     assert float(cov.min()) >= 0.85 - 1e-6 and float(cov.mean()) < 0.87
+
+
+# ---- the predictor built on the GPU (tardis_build_predictor) ----
+def _upper_factor(X, damp=0.01):
+    """Upper Cholesky factor of the inverse of H = (2/N) X^T X + damp mean(diag H) I, by numpy's routines in float64."""
+    X = np.asarray(X, dtype=np.float64)
+    H = 2.0 / X.shape[0] * X.T @ X
+    H += damp * np.mean(np.diag(H)) * np.eye(H.shape[0])
+    return np.ascontiguousarray(np.linalg.cholesky(np.linalg.inv(H)).T)
+
+
+def _build_and_compare(W1, U, bits, G, rows=None):
+    """GPU builder against the oracle on the same W1 and U: codes, zero-points and scales must be identical (every rounding
+    decision is taken in double precision with the same sequence of rounded operations on both sides)."""
+    dtype = "f32" if W1.dtype == torch.float32 else "bf16"
+    Ud = None if U is None else torch.from_numpy(U).cuda()
+    codes, scale, zero = T.tardis_build_predictor(W1, Ud, bits, G)
+    torch.cuda.synchronize()
+    h, d = W1.shape
+    rows = np.arange(h) if rows is None else rows
+    q_ref, s_ref, z_ref, _ = O.gptq_quantise(W1[torch.as_tensor(rows).cuda()].double().cpu().numpy(), U, G, bits, dtype)
+    q_gpu = O.unpack_codes(codes.cpu().numpy().view(np.uint32)[rows], d, bits)
+    bad = int((q_gpu != q_ref).sum())
+    assert bad == 0, "%d of %d codes differ" % (bad, q_ref.size)
+    assert np.array_equal(zero.cpu().numpy()[rows].astype(np.float64), z_ref)
+    assert np.array_equal(scale.double().cpu().numpy()[rows], s_ref)
+    return codes, scale, zero
+
+
+@pytest.mark.parametrize("dt", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("h,d,G,bits", [(400, 512, 64, 2), (130, 512, 128, 2), (64, 256, 128, 4), (70, 384, 64, 8), (1, 64, 64, 2)])
+def test_build_predictor_matches_oracle(h, d, G, bits, dt):
+    g = torch.Generator().manual_seed(h * 7 + d + bits)
+    W1 = (torch.randn(h, d, generator=g) * 0.05).to(dt).cuda()
+    mix = torch.eye(d) + 0.5 * torch.randn(d, d, generator=g) / d ** 0.5
+    X = (torch.randn(3 * d, d, generator=g) @ mix).numpy()
+    _build_and_compare(W1, _upper_factor(X), bits, G)
+    _build_and_compare(W1, None, bits, G)                       # no U: plain rounding to nearest
+    W0 = W1.clone()
+    W0[0] = 0                                                   # a neuron of zeros: scale 1, every code = zero-point 0
+    _build_and_compare(W0, _upper_factor(X), bits, G)
+
+
+def test_build_predictor_full_size_sampled_rows_and_use_in_a_layer():
+    """The 7B-class layer (16384 x 4096, groups of 128, 2 bits): sampled neurons against the oracle (neurons are independent
+    given U), then the built predictor goes into tardis_fold and a forward is compared with the oracle run on those codes."""
+    cfg = W.CONFIGS["decode_7b"]
+    L = W.make_layer(cfg, seed=4, device=torch.device("cuda", 0))
+    xcal = W.make_tokens(cfg, 1024, 4, device=torch.device("cuda", 0), tag="calibration").double()
+    H = 2.0 / xcal.shape[0] * xcal.t() @ xcal
+    H += 0.01 * torch.mean(torch.diagonal(H)) * torch.eye(cfg.d_model, dtype=torch.float64, device=H.device)
+    U = torch.linalg.cholesky(torch.cholesky_inverse(torch.linalg.cholesky(H)), upper=True).contiguous()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    codes, scale, zero = T.tardis_build_predictor(L.W1, U, 2, 128)
+    e1.record()
+    torch.cuda.synchronize()
+    print("tardis_build_predictor, 16384 x 4096: %.1f ms" % e0.elapsed_time(e1))
+    rows = np.array([0, 1, 63, 64, 4097, 8191, 12345, 16383])
+    Un = U.cpu().numpy()
+    q_ref, s_ref, z_ref, _ = O.gptq_quantise(L.W1[torch.as_tensor(rows).cuda()].double().cpu().numpy(), Un, 128, 2, "bf16")
+    q_gpu = O.unpack_codes(codes.cpu().numpy().view(np.uint32)[rows], cfg.d_model, 2)
+    assert np.array_equal(q_gpu, q_ref) and np.array_equal(zero.cpu().numpy()[rows].astype(np.float64), z_ref)
+    assert np.array_equal(scale.double().cpu().numpy()[rows], s_ref)
+    # the output error on the calibration inputs is below that of plain rounding for these neurons
+    r_codes, r_scale, r_zero = T.tardis_build_predictor(L.W1, None, 2, 128)
+    def out_err(c, s_, z_):
+        qq = O.unpack_codes(c.cpu().numpy().view(np.uint32)[rows], cfg.d_model, 2).astype(np.float64).reshape(len(rows), -1, 128)
+        deq = ((qq - z_.cpu().numpy()[rows].astype(np.float64)[:, :, None]) * s_.double().cpu().numpy()[rows][:, :, None]).reshape(len(rows), -1)
+        return np.linalg.norm(xcal.cpu().numpy() @ (L.W1[torch.as_tensor(rows).cuda()].double().cpu().numpy() - deq).T)
+    assert out_err(codes, scale, zero) < 0.9 * out_err(r_codes, r_scale, r_zero)
+    import dataclasses
+    from tests import helpers as Hp
+    L2 = dataclasses.replace(L, codes=codes, scale=scale, zero=zero)
+    h = T.fold_layer(L2)
+    try:
+        x = W.make_tokens(cfg, 3, 9, device=torch.device("cuda", 0))
+        y, F, S = Hp.gpu_forward(h, L2, x, [1, 2])
+        Hp.assert_parity(L2, L2.numpy64(), x, y, F, S, score_tol=3e-4, label="built predictor")
+    finally:
+        T.tardis_destroy(h)
