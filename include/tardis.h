@@ -351,6 +351,12 @@ tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_han
 tardis_status_t tardis_debug_wait_timeout(tardis_handle_t handle, int64_t limit_cycles, tardis_stream_t stream);
 tardis_status_t tardis_clear_error(tardis_handle_t handle);
 
+/* For testing what the library does when the device allocator says no, without exhausting a GPU: after this call the next
+ * `nth` device allocations of the library (process-wide, any thread) succeed and the one after them fails once, as
+ * cudaMalloc would with no memory left; nth < 0 switches the injection off.  The entry point that hits the failure
+ * returns TARDIS_ERR_ALLOC and must leave nothing allocated behind.  (The paper has no counterpart of this call.) */
+tardis_status_t tardis_debug_fail_alloc(int32_t nth);
+
 /* Frees everything the handle owns (synchronises the device first). */
 tardis_status_t tardis_destroy(tardis_handle_t handle);
 

@@ -22,7 +22,7 @@ TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_set_deterministic", "tardis_stack_forward", "tardis_build_predictor", "tardis_destroy", "tardis_calibrate",
-           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_debug_wait_timeout", "tardis_clear_error",
+           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_debug_wait_timeout", "tardis_clear_error", "tardis_debug_fail_alloc",
            "tardis_save", "tardis_load", "tardis_status_string", "tardis_last_error"]
 
 
@@ -83,6 +83,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_range_search.argtypes = [i32, i32, vp, i64, vp, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp, vp]
     lib.tardis_debug_wait_timeout.argtypes = [vp, i64, vp]
     lib.tardis_clear_error.argtypes = [vp]
+    lib.tardis_debug_fail_alloc.argtypes = [i32]
     lib.tardis_save.argtypes = [vp, ctypes.c_char_p]
     lib.tardis_load.argtypes = [ctypes.c_char_p, vp, ctypes.POINTER(vp)]
     for name in EXPORTS[:-2]:
@@ -279,6 +280,11 @@ def tardis_stack_forward(handles, x: torch.Tensor, y: torch.Tensor, gammas=None,
     kb = keep.numel() * keep.element_size() if keep is not None else 0
     _check(load_library().tardis_stack_forward(ctypes.byref(desc), _ptr(x), _ptr(y), _ptr(work), wb, _ptr(keep), kb, n,
                                                _stream(stream)), "tardis_stack_forward")
+
+
+def tardis_debug_fail_alloc(nth: int):
+    """The library's (nth + 1)-th device allocation from now fails once; nth < 0 switches the injection off."""
+    _check(load_library().tardis_debug_fail_alloc(nth), "tardis_debug_fail_alloc")
 
 
 def tardis_save(handle: int, path: str):

@@ -5,6 +5,7 @@
 
 #include <new>
 
+#include <atomic>
 #include "common.cuh"
 #include "gemm.cuh"
 
@@ -26,6 +27,16 @@ static Handle* check(tardis_handle_t h) {
 
 // A handle's memory and kernels belong to the device that was current at tardis_fold: a call made with another device
 // current would launch there against this handle's pointers.
+static std::atomic<int> g_fail_alloc{-1};   // >= 0: that many allocations still succeed, the next one fails (once)
+
+cudaError_t dev_malloc_raw(void** p, size_t bytes) {
+  if (g_fail_alloc.load() >= 0 && g_fail_alloc.fetch_sub(1) == 0) {
+    *p = nullptr;
+    return cudaErrorMemoryAllocation;
+  }
+  return cudaMalloc(p, bytes);
+}
+
 static bool on_handle_device(const Handle* H) {
   int cur = -1;
   return cudaGetDevice(&cur) == cudaSuccess && cur == H->device;
@@ -35,7 +46,7 @@ template <typename T>
 static tardis_status_t dev_alloc(T** p, size_t count, size_t* tally) {
   *p = nullptr;
   size_t bytes = count * sizeof(T);
-  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes ? bytes : 16);
+  cudaError_t e = dev_malloc(reinterpret_cast<void**>(p), bytes ? bytes : 16);
   if (e != cudaSuccess) {
     set_last_error(e, "cudaMalloc");
     cudaGetLastError();
@@ -400,6 +411,11 @@ tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_han
   if (st == TARDIS_OK && bf16) st = batched_finish(H, nullptr, s);
   if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
   *out = reinterpret_cast<tardis_handle_t>(H);
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_debug_fail_alloc(int32_t nth) {
+  g_fail_alloc.store(nth < 0 ? -1 : nth);
   return TARDIS_OK;
 }
 

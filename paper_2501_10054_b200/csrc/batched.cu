@@ -191,7 +191,7 @@ tardis_status_t batched_prepare(Handle* H) {
       {reinterpret_cast<void**>(&S->bitmap), size_t(kChunk) * (h / 32) * 4, true},
       {reinterpret_cast<void**>(&S->rlist), size_t(kMaxRecheck) * 8, true}, {reinterpret_cast<void**>(&S->rcount), 16, true}};
   for (const Req& r : reqs) {
-    cudaError_t e = cudaMalloc(r.p, r.bytes);
+    cudaError_t e = dev_malloc(r.p, r.bytes);
     if (e != cudaSuccess) { set_last_error(e, "cudaMalloc"); cudaGetLastError(); batched_release(H); return TARDIS_ERR_ALLOC; }
     (r.scratch ? S->bytes_scratch : S->bytes_state) += r.bytes;
   }

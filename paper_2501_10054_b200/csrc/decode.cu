@@ -900,14 +900,14 @@ tardis_status_t decode_prepare(Handle* H, cudaStream_t s) {
   size_t tally = 0;
   const size_t pb_bytes = size_t(NT) * p.nkc * p.pbs;
   const size_t yacc_bytes = sizeof(float) * NREP * p.dacc;
-  cudaError_t e = cudaMalloc(&S->pblocks, pb_bytes); tally += pb_bytes;
-  if (e == cudaSuccess) { e = cudaMalloc(&S->plan, sizeof(int2) * grid); tally += sizeof(int2) * grid; }
-  if (e == cudaSuccess) { e = cudaMalloc(&S->smax, 16); tally += 16; }
-  if (e == cudaSuccess) { e = cudaMalloc(&S->rowexp, sizeof(int) * h); tally += sizeof(int) * h; }
+  cudaError_t e = dev_malloc(&S->pblocks, pb_bytes); tally += pb_bytes;
+  if (e == cudaSuccess) { e = dev_malloc(&S->plan, sizeof(int2) * grid); tally += sizeof(int2) * grid; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->smax, 16); tally += 16; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->rowexp, sizeof(int) * h); tally += sizeof(int) * h; }
   const size_t cp_bytes = size_t(p.nunits) * 8192;
-  if (e == cudaSuccess) { e = cudaMalloc(&S->Cp, cp_bytes); tally += cp_bytes; }
-  if (e == cudaSuccess) { e = cudaMalloc(&S->yacc, yacc_bytes); tally += yacc_bytes; }
-  if (e == cudaSuccess) { e = cudaMalloc(&S->ctl, sizeof(unsigned int) * CTL_WORDS); tally += sizeof(unsigned int) * CTL_WORDS; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->Cp, cp_bytes); tally += cp_bytes; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->yacc, yacc_bytes); tally += yacc_bytes; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->ctl, sizeof(unsigned int) * CTL_WORDS); tally += sizeof(unsigned int) * CTL_WORDS; }
   if (e != cudaSuccess) { set_last_error(e, "cudaMalloc"); cudaGetLastError(); return fail(TARDIS_ERR_ALLOC); }
   S->bytes = tally;
 

@@ -1038,12 +1038,12 @@ tardis_status_t fused_prepare(Handle* H, cudaStream_t s) {
   const size_t pb_bytes = size_t(NT) * p.nkc * p.pbs;
   const size_t yacc_bytes = sizeof(float) * NREP * MAXT * p.dacc;
   const size_t cp_bytes = size_t(p.nunits) * 8192;
-  cudaError_t e = cudaMalloc(&S->pblocks, pb_bytes); tally += pb_bytes;
-  if (e == cudaSuccess) { e = cudaMalloc(&S->plan, sizeof(int2) * grid); tally += sizeof(int2) * grid; }
-  if (e == cudaSuccess) { e = cudaMalloc(&S->smax, 16); tally += 16; }
-  if (e == cudaSuccess) { e = cudaMalloc(&S->Cp, cp_bytes); tally += cp_bytes; }
-  if (e == cudaSuccess) { e = cudaMalloc(&S->yacc, yacc_bytes); tally += yacc_bytes; }
-  if (e == cudaSuccess) { e = cudaMalloc(&S->ctl, sizeof(unsigned int) * CTL_WORDS); tally += sizeof(unsigned int) * CTL_WORDS; }
+  cudaError_t e = dev_malloc(&S->pblocks, pb_bytes); tally += pb_bytes;
+  if (e == cudaSuccess) { e = dev_malloc(&S->plan, sizeof(int2) * grid); tally += sizeof(int2) * grid; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->smax, 16); tally += 16; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->Cp, cp_bytes); tally += cp_bytes; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->yacc, yacc_bytes); tally += yacc_bytes; }
+  if (e == cudaSuccess) { e = dev_malloc(&S->ctl, sizeof(unsigned int) * CTL_WORDS); tally += sizeof(unsigned int) * CTL_WORDS; }
   if (e != cudaSuccess) { set_last_error(e, "cudaMalloc"); cudaGetLastError(); return fail(TARDIS_ERR_ALLOC); }
   S->bytes = tally;
 
@@ -1127,7 +1127,8 @@ tardis_status_t fused_set_deterministic(Handle* H, bool on) {
   if (!S) return TARDIS_OK;
   if (on && !S->dpart) {
     const size_t bytes = size_t(S->base.nkc + S->grid) * MAXT * S->base.dacc * sizeof(float);
-    TARDIS_CUDA_TRY(cudaMalloc(&S->dpart, bytes));
+    const cudaError_t e = dev_malloc(&S->dpart, bytes);
+    if (e != cudaSuccess) { S->dpart = nullptr; set_last_error(e, "cudaMalloc"); cudaGetLastError(); return TARDIS_ERR_ALLOC; }
     H->bytes_scratch += bytes;
   }
   return TARDIS_OK;

@@ -144,11 +144,11 @@ tardis_status_t launch_build_predictor(int h, int d, int dtype, const void* W1, 
   auto release = [&]() {
     cudaFree(Wd); cudaFree(Eb); cudaFree(scale64); cudaFree(zero64); cudaFree(q);
   };
-  cudaError_t e = cudaMalloc(&Wd, size_t(h) * d * sizeof(double));
-  if (e == cudaSuccess) e = cudaMalloc(&Eb, size_t(h) * QB * sizeof(double));
-  if (e == cudaSuccess) e = cudaMalloc(&scale64, size_t(h) * ng * sizeof(double));
-  if (e == cudaSuccess) e = cudaMalloc(&zero64, size_t(h) * ng * sizeof(double));
-  if (e == cudaSuccess) e = cudaMalloc(&q, size_t(h) * d);
+  cudaError_t e = dev_malloc(&Wd, size_t(h) * d * sizeof(double));
+  if (e == cudaSuccess) e = dev_malloc(&Eb, size_t(h) * QB * sizeof(double));
+  if (e == cudaSuccess) e = dev_malloc(&scale64, size_t(h) * ng * sizeof(double));
+  if (e == cudaSuccess) e = dev_malloc(&zero64, size_t(h) * ng * sizeof(double));
+  if (e == cudaSuccess) e = dev_malloc(&q, size_t(h) * d);
   if (e != cudaSuccess) { release(); cudaGetLastError(); return TARDIS_ERR_ALLOC; }
   const size_t count = size_t(h) * d;
   if (dtype == TARDIS_F32) k_widen<float><<<2048, 256, 0, s>>>(static_cast<const float*>(W1), Wd, count);

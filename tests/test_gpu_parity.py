@@ -322,6 +322,73 @@ def test_stack_forward_layer_by_layer_against_the_oracle(n, normalise, residual)
             T.tardis_destroy(h)
 
 
+@pytest.mark.parametrize("dtype,d,h", [("bf16", 512, 2048), ("f32", 256, 1024)])
+def test_allocation_failures_return_a_status_and_leak_nothing(dtype, d, h):
+    """Every device allocation of tardis_fold (and of what it prepares for the kernels) fails once in turn, injected through
+    tardis_debug_fail_alloc: the call returns TARDIS_ERR_ALLOC, frees what it had, and a later fold of the same layer works
+    and gives correct results.  The same for the buffers of the deterministic mode, the predictor builder and tardis_load."""
+    import tempfile, os
+    cfg = W.LayerConfig("allocfail", d, h, n_calib=512, dtype=dtype)
+    L = _layer(cfg)
+    torch.cuda.synchronize()
+    hd = T.fold_layer(L)
+    T.tardis_destroy(hd)                                     # (first use: one-off allocations of the CUDA runtime settle)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    failed = 0
+    try:
+        for nth in range(200):
+            T.tardis_debug_fail_alloc(nth)
+            try:
+                hd = T.fold_layer(L)
+            except T.TardisError as e:
+                assert e.status == 3, e.status
+                failed += 1
+                torch.cuda.synchronize()
+                assert torch.cuda.mem_get_info()[0] >= free0, "allocation %d: %d bytes left behind" % (nth, free0 - torch.cuda.mem_get_info()[0])
+                continue
+            break                                            # nth is past the last allocation of a fold: it went through
+        else:
+            raise AssertionError("fold never succeeded")
+        T.tardis_debug_fail_alloc(-1)
+        assert failed >= 10, failed
+        x = W.make_tokens(cfg, 3, 1).cuda()
+        y, F, S = Hp.gpu_forward(hd, L, x, [3])
+        Hp.assert_parity(L, L.numpy64(), x, y, F, S, score_tol=3e-4, label="after failures")
+        if dtype == "bf16":
+            T.tardis_debug_fail_alloc(0)
+            with pytest.raises(T.TardisError):
+                T.tardis_set_deterministic(hd, True)
+            T.tardis_debug_fail_alloc(-1)
+            T.tardis_set_deterministic(hd, True)
+            T.tardis_set_deterministic(hd, False)
+        path = os.path.join(tempfile.mkdtemp(), "layer.bin")
+        T.tardis_save(hd, path)
+        T.tardis_destroy(hd)
+        hd = None
+        torch.cuda.synchronize()
+        free1 = torch.cuda.mem_get_info()[0]
+        for nth in (0, 3, 9):
+            T.tardis_debug_fail_alloc(nth)
+            with pytest.raises(T.TardisError) as e:
+                T.tardis_load(path)
+            assert e.value.status == 3
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] >= free1
+        for nth in range(5):
+            T.tardis_debug_fail_alloc(nth)
+            with pytest.raises(T.TardisError) as e:
+                T.tardis_build_predictor(L.W1, None, 2, 64)
+            assert e.value.status == 3
+        T.tardis_debug_fail_alloc(-1)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] >= free1
+    finally:
+        T.tardis_debug_fail_alloc(-1)
+        if hd:
+            T.tardis_destroy(hd)
+
+
 def test_batched_path_chunk_boundary_nan_token_and_empty_ranges():
     """More tokens than one scratch chunk in a single call (chunks hold 1024 tokens while the debug capture is on,
     2048 otherwise), a token holding a NaN in the middle of it, and the result compared token by token with the
