@@ -236,6 +236,21 @@ tardis_status_t tardis_range_search(int32_t d_ff, int32_t n_cal, const float* z,
                                     const float* thresholds, double threshold, double step, int32_t act, float* lo, float* hi,
                                     float* a, float* c, int32_t* steps_taken, tardis_stream_t stream);
 
+/* The neuron-level thresholds of Section 5.1.1: within a layer, the layer's threshold t_layer is distributed over the
+ * neurons by minimising sum_j E_j t_j subject to sum_j t_j = t_layer d_ff, where E_j is the error contribution of neuron j.
+ * As printed the problem has no bounds on t_j and no minimum; it is read with the box t_min <= t_j <= t_max, whose solution
+ * is: every neuron gets t_min, and the remaining budget (t_layer - t_min) d_ff goes, t_max - t_min each, to the neurons in
+ * order of increasing E_j (the smaller index first among equal errors); at most one neuron ends between the bounds.  E_j is
+ * measured as Algorithm 1's approx_error does: the mean squared residual of the least-squares line over the neuron's
+ * calibration samples inside its range [lo_j, hi_j) (0 with fewer than two samples inside), in double precision, stored in
+ * single; the order is taken on the stored values.
+ *   z, ldz, b1, n_cal   as in tardis_range_search (n_cal <= 2048);  lo, hi   device [d_ff], e.g. a search at t_layer;
+ *   err         out, device [d_ff]: E_j;   thresholds   out, device [d_ff]: t_j, what tardis_range_search takes next.
+ * 0 <= t_min <= t_layer <= t_max <= 1.  Asynchronous on `stream`; allocates nothing; nothing is kept. */
+tardis_status_t tardis_neuron_thresholds(int32_t d_ff, int32_t n_cal, const float* z, int64_t ldz, const float* b1,
+                                         const float* lo, const float* hi, int32_t act, double t_layer, double t_min,
+                                         double t_max, float* err, float* thresholds, tardis_stream_t stream);
+
 /* Chooses the kernel path: 0 = automatic (default), 1 = always the generic
  * kernels, 2 = the fused decode kernel for every token count up to 4096 (in
  * launches of at most 4 tokens; layers it does not serve fall back as in 0),

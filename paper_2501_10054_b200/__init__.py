@@ -22,7 +22,7 @@ TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_set_deterministic", "tardis_stack_forward", "tardis_build_predictor", "tardis_destroy", "tardis_calibrate",
-           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_debug_wait_timeout", "tardis_clear_error", "tardis_debug_fail_alloc",
+           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_neuron_thresholds", "tardis_debug_wait_timeout", "tardis_clear_error", "tardis_debug_fail_alloc",
            "tardis_save", "tardis_load", "tardis_status_string", "tardis_last_error"]
 
 
@@ -82,6 +82,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_debug_phase_stamps.argtypes = [vp, i32]
     lib.tardis_range_search.argtypes = [i32, i32, vp, i64, vp, vp, ctypes.c_double, ctypes.c_double, i32, vp, vp, vp, vp, vp, vp]
     lib.tardis_debug_wait_timeout.argtypes = [vp, i64, vp]
+    lib.tardis_neuron_thresholds.argtypes = [i32, i32, vp, i64, vp, vp, vp, i32, ctypes.c_double, ctypes.c_double, ctypes.c_double, vp, vp, vp]
     lib.tardis_clear_error.argtypes = [vp]
     lib.tardis_debug_fail_alloc.argtypes = [i32]
     lib.tardis_save.argtypes = [vp, ctypes.c_char_p]
@@ -198,6 +199,21 @@ def tardis_range_search(z: torch.Tensor, b1: Optional[torch.Tensor], threshold, 
                                               out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), out[3].data_ptr(),
                                               _ptr(steps), _stream(stream)), "tardis_range_search")
     return tuple(out) + ((steps,) if want_steps else ())
+
+
+def tardis_neuron_thresholds(z: torch.Tensor, b1: Optional[torch.Tensor], lo: torch.Tensor, hi: torch.Tensor, act: int,
+                             t_layer: float, t_min: float, t_max: float, stream=None):
+    """Per-neuron coverage thresholds of Section 5.1.1 from the neurons' approximation errors inside [lo, hi): returns
+    (err, thresholds), float32 tensors of d_ff elements (see tardis_neuron_thresholds in tardis.h)."""
+    if z.dtype != torch.float32 or not z.is_cuda or z.stride(1) != 1:
+        raise TardisError(1, "z must be a float32 CUDA tensor with unit inner stride")
+    h, n = z.shape
+    err = torch.empty(h, dtype=torch.float32, device=z.device)
+    thr = torch.empty(h, dtype=torch.float32, device=z.device)
+    _check(load_library().tardis_neuron_thresholds(h, n, z.data_ptr(), z.stride(0), _ptr(b1), _ptr(lo), _ptr(hi), int(act),
+                                                   float(t_layer), float(t_min), float(t_max), _ptr(err), _ptr(thr),
+                                                   _stream(stream)), "tardis_neuron_thresholds")
+    return err, thr
 
 
 def tardis_stats(handle: int) -> dict:

@@ -233,6 +233,16 @@ tardis_status_t tardis_range_search(int32_t d_ff, int32_t n_cal, const float* z,
                              reinterpret_cast<cudaStream_t>(stream));
 }
 
+tardis_status_t tardis_neuron_thresholds(int32_t d_ff, int32_t n_cal, const float* z, int64_t ldz, const float* b1, const float* lo,
+                                         const float* hi, int32_t act, double t_layer, double t_min, double t_max, float* err,
+                                         float* thresholds, tardis_stream_t stream) {
+  if (d_ff <= 0 || n_cal <= 0 || !z || ldz < n_cal || !lo || !hi || !err || !thresholds) return TARDIS_ERR_INVALID_ARG;
+  if (!(t_min >= 0.0 && t_min <= t_layer && t_layer <= t_max && t_max <= 1.0)) return TARDIS_ERR_INVALID_ARG;
+  if (act != TARDIS_ACT_GELU_TANH && act != TARDIS_ACT_GELU_ERF && act != TARDIS_ACT_RELU) return TARDIS_ERR_INVALID_ARG;
+  return launch_neuron_thresholds(d_ff, n_cal, z, ldz, b1, lo, hi, act, t_layer, t_min, t_max, err, thresholds,
+                                  reinterpret_cast<cudaStream_t>(stream));
+}
+
 tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
   Handle* H = check(handle);
   if (!H || !out) return TARDIS_ERR_INVALID_ARG;

@@ -236,7 +236,85 @@ k_range_search(const float* __restrict__ z, long long ldz, const float* __restri
   fit_and_store(keys, n, lo_f, hi_f, act, red, j, lo, hi, a, c);
 }
 
+// Error contribution of every neuron (Section 5.1.1, the E of the neuron-level thresholds): the mean squared residual of
+// the least-squares line over the neuron's samples inside its range [lo_j, hi_j), as Algorithm 1's approx_error measures it.
+__global__ void __launch_bounds__(NT)
+k_neuron_error(const float* __restrict__ z, long long ldz, const float* __restrict__ b1, int n, int npad, int act,
+               const float* __restrict__ lo, const float* __restrict__ hi, float* __restrict__ err) {
+  extern __shared__ __align__(16) unsigned char smem_err[];
+  double* gs = reinterpret_cast<double*>(smem_err);                // [n] activation of the sorted samples
+  float* keys = reinterpret_cast<float*>(gs + n);                  // [npad] sorted samples
+  __shared__ double red[2 * (NT / 32)];
+  const int j = blockIdx.x, tid = threadIdx.x;
+  load_and_sort(z, ldz, b1, j, n, npad, keys);
+  for (int i = tid; i < n; i += NT) gs[i] = gelu_f64(double(keys[i]), act);
+  __syncthreads();
+  auto lower = [&](double v) {
+    int l = 0, r = n;
+    while (l < r) { const int m = (l + r) >> 1; if (double(keys[m]) < v) l = m + 1; else r = m; }
+    return l;
+  };
+  const int i0 = lower(double(lo[j])), i1 = lower(double(hi[j]));
+  const int cnt = i1 - i0;
+  double e = 0.0;
+  if (cnt >= 2) {                                           // (uniform over the CTA)
+    const double q = 1.0 / double(cnt);
+    double sz = 0.0, sg = 0.0;
+    for (int i = i0 + tid; i < i1; i += NT) { sz += double(keys[i]); sg += gs[i]; }
+    block_sum2(sz, sg, red);
+    const double mz = sz * q, mg = sg * q;
+    double vzz = 0.0, vzg = 0.0;
+    for (int i = i0 + tid; i < i1; i += NT) { const double dz = double(keys[i]) - mz; vzz += dz * dz; vzg += dz * (gs[i] - mg); }
+    block_sum2(vzz, vzg, red);
+    vzz *= q; vzg *= q;
+    if (vzz > 1e-30) {
+      const double sl = vzg / vzz;
+      double rr = 0.0, dummy = 0.0;
+      for (int i = i0 + tid; i < i1; i += NT) { const double r = (gs[i] - mg) - sl * (double(keys[i]) - mz); rr += r * r; }
+      block_sum2(rr, dummy, red);
+      e = rr * q;
+    }
+  }
+  if (tid == 0) err[j] = float(e);
+}
+
+// Neuron-level thresholds (Section 5.1.1): minimise sum_j E_j t_j subject to sum_j t_j = t_layer h, read with the box
+// t_min <= t_j <= t_max.  A linear objective over a box with one equality: every neuron starts at t_min and the budget
+// (t_layer - t_min) h goes, t_max - t_min each, to the neurons in order of increasing error (the smaller index first among
+// equals).  A thread finds its neuron's place in that order by counting, then takes its share of what is left for it.
+__global__ void __launch_bounds__(NT)
+k_neuron_thresholds(const float* __restrict__ err, int h, double t_layer, double t_min, double t_max, float* __restrict__ t) {
+  __shared__ float tile[NT];
+  const int j = blockIdx.x * NT + threadIdx.x;
+  const float ej = j < h ? err[j] : 0.f;
+  int rank = 0;
+  for (int base = 0; base < h; base += NT) {
+    __syncthreads();
+    tile[threadIdx.x] = base + threadIdx.x < h ? err[base + threadIdx.x] : 0.f;
+    __syncthreads();
+    const int m = min(NT, h - base);
+    for (int i = 0; i < m; ++i) rank += (tile[i] < ej || (tile[i] == ej && base + i < j)) ? 1 : 0;
+  }
+  if (j >= h) return;
+  const double cap = t_max - t_min, budget = (t_layer - t_min) * double(h);
+  const double give = fmin(cap, fmax(0.0, budget - double(rank) * cap));
+  t[j] = float(t_min + give);
+}
+
 }  // namespace cal
+
+tardis_status_t launch_neuron_thresholds(int h, int n, const float* z, long long ldz, const float* b1, const float* lo, const float* hi,
+                                         int act, double t_layer, double t_min, double t_max, float* err, float* t, cudaStream_t s) {
+  if (n < 1 || n > cal::kMaxSearchSamples) return TARDIS_ERR_UNSUPPORTED;
+  int npad = 2;
+  while (npad < n) npad <<= 1;
+  const size_t smem = size_t(n) * sizeof(double) + size_t(npad) * sizeof(float);
+  cal::k_neuron_error<<<h, cal::NT, smem, s>>>(z, ldz, b1, n, npad, act, lo, hi, err);
+  TARDIS_CUDA_TRY(cudaGetLastError());
+  cal::k_neuron_thresholds<<<(h + cal::NT - 1) / cal::NT, cal::NT, 0, s>>>(err, h, t_layer, t_min, t_max, t);
+  TARDIS_CUDA_TRY(cudaGetLastError());
+  return TARDIS_OK;
+}
 
 tardis_status_t launch_calibrate(int h, int n, const float* z, long long ldz, const float* b1, double q_lo, double q_hi, int act,
                                  float* lo, float* hi, float* a, float* c, cudaStream_t s) {

@@ -105,6 +105,8 @@ template <> __device__ __forceinline__ float from_f32<float>(float v) { return v
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 // offline statistics (calibrate.cu)
+tardis_status_t launch_neuron_thresholds(int h, int n, const float* z, long long ldz, const float* b1, const float* lo, const float* hi,
+                                         int act, double t_layer, double t_min, double t_max, float* err, float* t, cudaStream_t s);
 tardis_status_t launch_calibrate(int h, int n, const float* z, long long ldz, const float* b1, double q_lo, double q_hi, int act,
                                  float* lo, float* hi, float* a, float* c, cudaStream_t s);
 

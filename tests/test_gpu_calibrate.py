@@ -212,6 +212,45 @@ def test_greedy_range_search_full_layer_shape_sampled():
     assert float(cov.min()) >= 0.85 - 1e-6 and float(cov.mean()) < 0.87
 
 
+# ---- neuron-level thresholds (tardis_neuron_thresholds) ----
+@pytest.mark.parametrize("h,n,act", [(96, 257, W.ACT_GELU_TANH), (300, 1000, W.ACT_GELU_ERF), (1024, 2048, W.ACT_RELU), (5, 16, W.ACT_GELU_TANH)])
+def test_neuron_thresholds_match_oracle(h, n, act):
+    """Errors: each neuron's approx_error of the oracle within the rounding of a float32 and of sums taken in another order.
+    Thresholds: the oracle's allocation on its own errors (rounded to float32, the precision the order is taken in); a
+    neuron may differ only where its error is so close to the error at which the budget runs out that the two sides
+    can order it differently, and then both values must be valid ones (t_min or t_max).  The mean threshold is t_layer."""
+    g = torch.Generator().manual_seed(31 * h + n)
+    z = (torch.randn(h, n, generator=g) * torch.linspace(0.3, 3.0, h)[:, None] + torch.linspace(-1, 1, h)[:, None]).cuda()
+    b1 = (0.1 * torch.randn(h, generator=g)).cuda()
+    lo, hi, _, _ = T.tardis_range_search(z, b1, 0.85, 0.05, act)
+    for (t_layer, t_min, t_max) in [(0.85, 0.7, 0.95), (0.8, 0.8, 0.9), (0.9, 0.5, 0.9), (0.77, 0.6, 1.0)]:
+        err, thr = T.tardis_neuron_thresholds(z, b1, lo, hi, act, t_layer, t_min, t_max)
+        torch.cuda.synchronize()
+        zc = z.cpu().numpy() + b1.cpu().numpy()[:, None]
+        lo_c, hi_c = lo.cpu().numpy().astype(np.float64), hi.cpu().numpy().astype(np.float64)
+        e_ref = np.array([O.approx_error(zc[j], lo_c[j], hi_c[j], act) for j in range(h)])
+        e_gpu = err.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(e_gpu - e_ref) <= 1e-6 * np.abs(e_ref) + 1e-30), np.abs(e_gpu - e_ref).max()
+        e32 = e_ref.astype(np.float32).astype(np.float64)
+        t_ref = O.neuron_thresholds(e32, t_layer, t_min, t_max)
+        t_gpu = thr.cpu().numpy().astype(np.float64)
+        assert abs(t_gpu.mean() - t_layer) <= 1e-6
+        assert np.all(t_gpu >= t_min - 1e-7) and np.all(t_gpu <= t_max + 1e-7)
+        diff = np.abs(t_gpu - t_ref) > 1e-6
+        if diff.any():
+            order = np.argsort(e32, kind="stable")
+            funded = int(np.floor((t_layer - t_min) * h / (t_max - t_min) + 1e-9)) if t_max > t_min else 0
+            cut = e32[order[min(funded, h - 1)]]
+            assert np.all(np.abs(e32[diff] - cut) <= 2e-6 * abs(cut) + 1e-30), "thresholds differ away from the cut-off error"
+    # a layer whose neurons all have the same error: the smaller index is funded first
+    same = torch.zeros(8, 64).cuda()
+    same[:, ::2] = 1.0
+    err, thr = T.tardis_neuron_thresholds(same, None, torch.full((8,), -5.0).cuda(), torch.full((8,), 5.0).cuda(), W.ACT_RELU, 0.75, 0.5, 1.0)
+    assert np.allclose(thr.cpu().numpy(), [1, 1, 1, 1, 0.5, 0.5, 0.5, 0.5])
+    with pytest.raises(T.TardisError):
+        T.tardis_neuron_thresholds(same, None, err, err, 0, 0.5, 0.6, 0.9)      # t_layer below t_min
+
+
 # ---- the predictor built on the GPU (tardis_build_predictor) ----
 def _upper_factor(X, damp=0.01):
     """Upper Cholesky factor of the inverse of H = (2/N) X^T X + damp mean(diag H) I, by numpy's routines in float64."""
