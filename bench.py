@@ -580,7 +580,7 @@ def run_studies(args, T, W, torch, dev):
     base = W.CONFIGS["decode_7b"]
     x = W.make_tokens(base, 64, seed=3, device=dev)
     sweep = {}
-    for bits in (2, 4, 8):
+    for bits in (2, 3, 4, 8):
         cfg = dataclasses.replace(base, bits=bits)
         L = W.make_layer(cfg, seed=11, device=dev)
         hd = T.fold_layer(L)

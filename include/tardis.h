@@ -66,12 +66,16 @@ typedef struct {
   const float* a;             /* device [d_ff]; linear fit a*z + c on the range           */
   const float* c;             /* device [d_ff]                                            */
   int32_t pred_bits;          /* bits per predictor code: 2 (the paper's setting, Section 6;
-                                 every path), 4 (batched and generic paths) or 8 (generic
-                                 kernels only); the paper sweeps this size in Section 7.6  */
+                                 every path), 3 or 4 (batched and generic paths; 3 needs
+                                 d_model % 32 == 0) or 8 (generic kernels only); the paper
+                                 sweeps this size in Section 7.6                           */
   int32_t pred_group;         /* G: channels per quantisation group; multiple of 16       */
-  const uint32_t* pred_codes; /* device [d_ff, d_model*pred_bits/32]; with p = 32/pred_bits
-                                 codes per word, channel k of row j sits in word k/p, bits
-                                 pred_bits*(k%p) upwards                                  */
+  const uint32_t* pred_codes; /* device [d_ff, d_model*pred_bits/32]: row j is one bit stream
+                                 over its words, lowest bits first; channel k holds its bits
+                                 [pred_bits k, pred_bits (k + 1)) (word pred_bits k / 32,
+                                 from bit pred_bits k % 32 upwards; with 2, 4 or 8 bits a
+                                 code stays inside one word, a 3-bit code may go on in the
+                                 lowest bits of the next word)                            */
   const void* pred_scale;     /* device [d_ff, d_model/G], type `dtype`                   */
   const uint8_t* pred_zero;   /* device [d_ff, d_model/G], integer zero-point 0..2^pred_bits-1 */
   uint32_t flags;             /* 0, or one of the TARDIS_FOLD_* study modes below          */
@@ -117,7 +121,7 @@ typedef struct {
  * allocations; *out is valid on return with TARDIS_OK.
  * Errors: INVALID_ARG (NULL desc/out/required array, pointer not 16-byte
  * aligned, d_model % 8, d_model % pred_group, pred_group % 16, d_ff % 32,
- * non-positive sizes, unknown enum, pred_bits outside 1..8), UNSUPPORTED (pred_bits of 1, 3, 5, 6 or 7), ALLOC, CUDA.
+ * non-positive sizes, unknown enum, pred_bits outside 1..8), UNSUPPORTED (pred_bits of 1, 5, 6 or 7), ALLOC, CUDA.
  * Forward calls on the handle must be ordered after `stream` (same stream, or an event): the fold is asynchronous. */
 tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stream,
                             tardis_handle_t* out);
@@ -293,8 +297,8 @@ tardis_status_t tardis_set_deterministic(tardis_handle_t handle, int32_t on);
  *   U      device double [d_model, d_model] row-major, the upper Cholesky factor of the inverse Hessian of the layer's
  *          inputs (U^T U = H^-1, H = (2/N) X^T X plus damping: made by the caller, e.g. with a library Cholesky), only
  *          its upper triangle is read; NULL = identity, which gives plain rounding to nearest;
- *   bits   2, 4 or 8; group a multiple of 64 that divides d_model;
- *   codes  out, device [d_ff, d_model bits / 32] (channel order ascending, lowest bits first);
+ *   bits   2, 3, 4 or 8; group a multiple of 64 that divides d_model;
+ *   codes  out, device [d_ff, d_model bits / 32] (one bit stream per row, channel order ascending, lowest bits first);
  *   scale  out, device [d_ff, d_model / group] in `dtype`; zero out, device bytes of the same shape.
  * The outputs are what tardis_fold_desc_t takes as pred_codes, pred_scale, pred_zero.  The call allocates its scratch
  * (8 d_ff d_model bytes and a little more), runs on `stream` and returns after the stream has finished the work.

@@ -71,19 +71,27 @@ def gelu(z, act=ACT_GELU_TANH):
 def unpack_codes(codes_u32, d, bits=2):
     """Expand packed predictor codes to one integer per weight.
 
-    Packed layout: for neuron j, word w of row j holds the codes of input
-    channels k = w*(32/bits) ... , channel order ascending, lowest bits first.
-    Returns uint8 [h, d]."""
+    Packed layout: row j is one bit stream over its 32-bit words, lowest bits first; input channel k holds the bits
+    [bits k, bits (k + 1)) of it.  With 2, 4 or 8 bits per code that is 32/bits codes per word; a 3-bit code may start in
+    one word and go on in the lowest bits of the next.  Returns uint8 [h, d]."""
     codes_u32 = np.asarray(codes_u32, dtype=np.uint32)
-    per = 32 // bits
     h, nw = codes_u32.shape
-    if nw * per != d:
-        raise ValueError("codes row has %d words, expected %d" % (nw, d // per))
-    q = np.empty((h, d), dtype=np.uint8)
-    mask = np.uint32((1 << bits) - 1)
-    for p in range(per):
-        q[:, p::per] = ((codes_u32 >> np.uint32(bits * p)) & mask).astype(np.uint8)
-    return q
+    if nw * 32 != d * bits:
+        raise ValueError("codes row has %d words, expected %d" % (nw, d * bits // 32))
+    if 32 % bits == 0:                      # a code never leaves its word: 32/bits codes per word
+        per = 32 // bits
+        q = np.empty((h, d), dtype=np.uint8)
+        mask = np.uint32((1 << bits) - 1)
+        for p in range(per):
+            q[:, p::per] = ((codes_u32 >> np.uint32(bits * p)) & mask).astype(np.uint8)
+        return q
+    # the stream as single bits, then `bits` of them per channel, the lowest first
+    stream = (codes_u32[:, :, None] >> np.arange(32, dtype=np.uint32)[None, None, :]) & np.uint32(1)
+    per_code = stream.reshape(h, d, bits).astype(np.uint32)
+    q = np.zeros((h, d), dtype=np.uint32)
+    for b in range(bits):
+        q |= per_code[:, :, b] << np.uint32(b)
+    return q.astype(np.uint8)
 
 
 def predictor_score(x, codes_u32, scale, zero, group, b1=None, bits=2):
@@ -538,12 +546,11 @@ def gptq_quantise(W1, U, group, bits=2, dtype="bf16"):
 
 
 def pack_codes(q, bits=2):
-    """The inverse of unpack_codes: [h, d] codes into [h, d bits / 32] 32-bit words, channel order ascending, lowest bits
-    first."""
-    q = np.asarray(q, dtype=np.uint64)
-    per = 32 // bits
+    """The inverse of unpack_codes: [h, d] codes into [h, d bits / 32] 32-bit words, one bit stream per row, channel order
+    ascending, lowest bits first."""
+    q = np.asarray(q, dtype=np.uint32)
     h, d = q.shape
-    words = np.zeros((h, d // per), dtype=np.uint64)
-    for p in range(per):
-        words |= q[:, p::per] << np.uint64(bits * p)
+    single = (q[:, :, None] >> np.arange(bits, dtype=np.uint32)[None, None, :]) & np.uint32(1)     # [h, d, bits]
+    stream = single.reshape(h, d * bits // 32, 32).astype(np.uint64)
+    words = (stream << np.arange(32, dtype=np.uint64)[None, None, :]).sum(axis=2)
     return words.astype(np.uint32)

@@ -120,8 +120,9 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
   if (desc->act != TARDIS_ACT_GELU_TANH && desc->act != TARDIS_ACT_GELU_ERF && desc->act != TARDIS_ACT_RELU) return TARDIS_ERR_INVALID_ARG;
   if (desc->flags > TARDIS_FOLD_FP32_PLAIN) return TARDIS_ERR_INVALID_ARG;
   if (d % 8 || h % 32 || G % 16 || d % G) return TARDIS_ERR_INVALID_ARG;
-  if (desc->pred_bits != 2 && desc->pred_bits != 4 && desc->pred_bits != 8)
+  if (desc->pred_bits != 2 && desc->pred_bits != 3 && desc->pred_bits != 4 && desc->pred_bits != 8)
     return desc->pred_bits > 0 && desc->pred_bits <= 8 ? TARDIS_ERR_UNSUPPORTED : TARDIS_ERR_INVALID_ARG;
+  if (desc->pred_bits == 3 && d % 32) return TARDIS_ERR_INVALID_ARG;      // (a row of 3-bit codes is a whole number of words)
   const void* required[] = {desc->W1, desc->W2, desc->lo, desc->hi, desc->a, desc->c,
                             desc->pred_codes, desc->pred_scale, desc->pred_zero};
   for (const void* p : required)
@@ -386,7 +387,7 @@ tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_han
   const int d = dims[0], h = dims[1], dtype = dims[2], act = dims[3], G = dims[4], bits = dims[5];
   const bool sane = d > 0 && h > 0 && G > 0 && d <= (1 << 20) && h <= (1 << 24) && (dtype == TARDIS_F32 || dtype == TARDIS_BF16) &&
                     act >= 0 && act <= TARDIS_ACT_RELU && !(d % 8) && !(h % 32) && !(G % 16) && !(d % G) &&
-                    (bits == 2 || bits == 4 || bits == 8);
+                    (bits == 2 || bits == 4 || bits == 8 || (bits == 3 && d % 32 == 0));
   if (!sane) { fclose(f); return TARDIS_ERR_CORRUPT; }
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   Handle* H = nullptr;
@@ -432,7 +433,7 @@ tardis_status_t tardis_debug_fail_alloc(int32_t nth) {
 tardis_status_t tardis_build_predictor(int32_t d_ff, int32_t d_model, tardis_dtype_t dtype, const void* W1, const double* U,
                                        int32_t bits, int32_t group, uint32_t* codes, void* scale, uint8_t* zero, tardis_stream_t stream) {
   if (d_ff < 1 || d_model < 1 || !W1 || !codes || !scale || !zero) return TARDIS_ERR_INVALID_ARG;
-  if (!(dtype == TARDIS_F32 || dtype == TARDIS_BF16) || !(bits == 2 || bits == 4 || bits == 8)) return TARDIS_ERR_INVALID_ARG;
+  if (!(dtype == TARDIS_F32 || dtype == TARDIS_BF16) || !(bits == 2 || bits == 3 || bits == 4 || bits == 8)) return TARDIS_ERR_INVALID_ARG;
   if (group < 64 || group % 64 || d_model % group) return TARDIS_ERR_INVALID_ARG;
   return launch_build_predictor(d_ff, d_model, dtype, W1, U, bits, group, codes, scale, zero, reinterpret_cast<cudaStream_t>(stream));
 }

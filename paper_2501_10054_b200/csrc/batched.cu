@@ -48,7 +48,17 @@ __global__ void k_dequant_split(const uint32_t* __restrict__ codes, const __nv_b
   const int per = 32 / bits;                    // codes per word
   const uint32_t cmask = (1u << bits) - 1u;
   const int j = blockIdx.x, ng = d / G, nwords = d / per;
-  for (int w = threadIdx.x; w < nwords; w += blockDim.x) {
+  if (32 % bits) {                              // 3-bit codes: a bit stream, channel by channel
+    const uint32_t* row = codes + size_t(j) * (size_t(d) * bits / 32);
+    for (int k = threadIdx.x; k < d; k += blockDim.x) {
+      const int g = k / G;
+      const float v = __bfloat162float(scale[size_t(j) * ng + g]) * (float(stream_code(row, k, bits)) - float(zero[size_t(j) * ng + g]));
+      const __nv_bfloat16 h = __float2bfloat16_rn(v);
+      hi[size_t(j) * d + k] = h;
+      lo[size_t(j) * d + k] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+  }
+  for (int w = threadIdx.x; w < nwords && 32 % bits == 0; w += blockDim.x) {
     const uint32_t word = codes[size_t(j) * nwords + w];
     const int g = (w * per) / G;
     const float s = __bfloat162float(scale[size_t(j) * ng + g]);

@@ -1,15 +1,45 @@
 // Exact fp64 predictor sums (Section 5.3: s[j,g] (q - zp) x over the channels of neuron j, without the bias) from the
-// packed codes (2, 4 or 8 bits each): what decides a flag when a fast score is too close to a range end.
+// packed codes (2, 3, 4 or 8 bits each): what decides a flag when a fast score is too close to a range end.
 #pragma once
 #include <cuda_bf16.h>
 #include <stdint.h>
 
 namespace tardis {
 
+// Code of channel k in a row of packed codes: the row is one bit stream, channel order ascending, lowest bits first (code k
+// holds bits [k bits, (k + 1) bits) of it).  With 2, 4 or 8 bits a code never leaves its 32-bit word; a 3-bit code may.
+__device__ __forceinline__ uint32_t stream_code(const uint32_t* __restrict__ row, int k, int bits) {
+  const int pos = k * bits, w = pos >> 5, sh = pos & 31;
+  uint32_t v = row[w] >> sh;
+  if (sh + bits > 32) v |= row[w + 1] << (32 - sh);
+  return v & ((1u << bits) - 1u);
+}
+
+// the same sums for code widths that do not divide 32 (3 bits): channel by channel, lane l takes channels 32 i + l
+__device__ inline double exact_score_stream(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
+                                            const uint8_t* __restrict__ zero, const __nv_bfloat16* __restrict__ xt, int j, int d, int G,
+                                            int bits, int first, int stride) {
+  const int ng = d / G;
+  const uint32_t* row = codes + size_t(j) * (size_t(d) * bits / 32);
+  double acc = 0.0;
+  for (int k = first; k < d; k += stride) {
+    const int g = k / G;
+    const double zp = double(zero[size_t(j) * ng + g]);
+    acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * ((double(stream_code(row, k, bits)) - zp) * double(__bfloat162float(xt[k])));
+  }
+  return acc;
+}
+
 // one warp; every lane returns the sum
 __device__ inline double exact_score(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
                               const uint8_t* __restrict__ zero, const __nv_bfloat16* __restrict__ xt, int j, int d, int G,
                               int bits, int lane) {   // one warp; every lane returns the sum
+  if (32 % bits) {
+    double acc = exact_score_stream(codes, scale, zero, xt, j, d, G, bits, lane, 32);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return acc;
+  }
   const int per = 32 / bits;                    // codes per word
   const uint32_t cmask = (1u << bits) - 1u;
   const int nwords = d / per, ng = d / G;
@@ -29,6 +59,7 @@ __device__ inline double exact_score(const uint32_t* __restrict__ codes, const _
 
 __device__ inline double exact_score_single(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
                                      const uint8_t* __restrict__ zero, const __nv_bfloat16* __restrict__ xt, int j, int d, int G, int bits) {
+  if (32 % bits) return exact_score_stream(codes, scale, zero, xt, j, d, G, bits, 0, 1);
   const int per = 32 / bits;                    // codes per word
   const uint32_t cmask = (1u << bits) - 1u;
   const int nwords = d / per, ng = d / G;

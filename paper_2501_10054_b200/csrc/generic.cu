@@ -4,6 +4,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "exact.cuh"
 
 namespace tardis {
 
@@ -27,7 +28,15 @@ __global__ void __launch_bounds__(1024) k_predictor_exact(
   for (int t = 0; t < n; ++t) {
     const T* xt = x + size_t(t) * d;
     double acc = 0.0;
-    for (int w = lane; w < nwords; w += 32) {
+    if (32 % bits) {                            // 3-bit codes: a bit stream, channel by channel
+      const uint32_t* row = codes + size_t(j) * (size_t(d) * bits / 32);
+      for (int k = lane; k < d; k += 32) {
+        const int g = k / G;
+        acc += double(to_f32(scale[size_t(j) * ng + g])) *
+               ((double(stream_code(row, k, bits)) - double(zero[size_t(j) * ng + g])) * double(to_f32(xt[k])));
+      }
+    }
+    for (int w = lane; w < nwords && 32 % bits == 0; w += 32) {
       const uint32_t word = codes[size_t(j) * nwords + w];
       const int g = (w * per) / G;
       const double zp = double(zero[size_t(j) * ng + g]);

@@ -119,13 +119,18 @@ __global__ void __launch_bounds__(256) k_spread(double* __restrict__ Wd, const d
 template <typename T>
 __global__ void k_pack_out(const uint8_t* __restrict__ q, const double* __restrict__ scale64, const double* __restrict__ zero64,
                            int h, int d, int G, int bits, uint32_t* __restrict__ codes, T* __restrict__ scale, uint8_t* __restrict__ zero) {
-  const int per = 32 / bits, nw = d / per, ng = d / G;
+  const int nw = d * bits / 32, ng = d / G;     // the row is one bit stream: code k holds bits [k bits, (k + 1) bits)
   const size_t words = size_t(h) * nw, groups = size_t(h) * ng;
   for (size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x; e < words; e += size_t(gridDim.x) * blockDim.x) {
     const size_t r = e / nw;
     const int wi = int(e - r * nw);
     uint32_t word = 0u;
-    for (int p = 0; p < per; ++p) word |= uint32_t(q[r * d + size_t(wi) * per + p]) << (bits * p);
+    const int k0 = (wi * 32) / bits, k1 = min(d - 1, (wi * 32 + 31) / bits);    // codes with a bit in this word
+    for (int k = k0; k <= k1; ++k) {
+      const int sh = k * bits - wi * 32;                                        // (negative: the code started in the word before)
+      const uint32_t c = q[r * d + k];
+      word |= sh >= 0 ? c << sh : c >> (-sh);
+    }
     codes[e] = word;
   }
   for (size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x; e < groups; e += size_t(gridDim.x) * blockDim.x) {

@@ -64,7 +64,8 @@ def test_invalid_arguments_return_status_before_any_launch(lib):
     assert status(act=5) == 1
     assert status(W1=None) == 1
     assert status(W1=24) == 1                 # misaligned
-    assert status(pred_bits=3) == 2           # valid but not built (2, 4 and 8 are)
+    assert status(pred_bits=5) == 2           # valid but not built (2, 3, 4 and 8 are)
+    assert status(pred_bits=3, d_model=80, pred_group=16) == 1   # a row of 3-bit codes must fill whole words
     assert status(pred_bits=0) == 1
     assert status(flags=7) == 1               # beyond the fold study modes
     assert out.value is None

@@ -279,7 +279,7 @@ def _build_and_compare(W1, U, bits, G, rows=None):
 
 
 @pytest.mark.parametrize("dt", [torch.bfloat16, torch.float32])
-@pytest.mark.parametrize("h,d,G,bits", [(400, 512, 64, 2), (130, 512, 128, 2), (64, 256, 128, 4), (70, 384, 64, 8), (1, 64, 64, 2)])
+@pytest.mark.parametrize("h,d,G,bits", [(400, 512, 64, 2), (130, 512, 128, 2), (64, 256, 128, 4), (70, 384, 64, 8), (1, 64, 64, 2), (50, 320, 64, 3)])
 def test_build_predictor_matches_oracle(h, d, G, bits, dt):
     g = torch.Generator().manual_seed(h * 7 + d + bits)
     W1 = (torch.randn(h, d, generator=g) * 0.05).to(dt).cuda()

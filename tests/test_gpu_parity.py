@@ -94,13 +94,14 @@ def test_batched_path_forced_for_calls_of_a_few_tokens():
     assert 0.02 < info["flag_frac"] < 0.5
 
 
-@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("bits", [3, 4, 8])
 def test_wider_predictor_codes(bits):
-    # 4-bit codes: batched tensor-core path (also for calls of a few tokens) and generic kernels; 8-bit codes: generic
+    # 3- and 4-bit codes: batched tensor-core path (also for calls of a few tokens) and generic kernels; 8-bit codes: generic
     # kernels only.  The paper sweeps the predictor size (Section 7.6); here each width must give the oracle's flags.
+    # (3-bit codes are a bit stream: some cross from one 32-bit word into the next.)
     cfg = W.LayerConfig("bits%d" % bits, 512, 2048, group=64, bits=bits, n_calib=512)
     calls = [1, 3, 20, 8]
-    info = _run(cfg, sum(calls), calls, path=3 if bits == 4 else 0)
+    info = _run(cfg, sum(calls), calls, path=3 if bits <= 4 else 0)
     assert 0.02 < info["flag_frac"] < 0.5
     _run(cfg, 6, [1, 5], path=1)
     cfg32 = W.LayerConfig("bits%d_f32" % bits, 128, 512, dtype="f32", group=32, bits=bits, n_calib=512)

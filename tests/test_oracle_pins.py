@@ -617,6 +617,34 @@ def test_gptq_quantise_identities_and_special_cases():
     w1 = 1.4 - e0 * 0.5
     assert sh[0, 0] == s_ and zh[0, 0] == 0 and qh[0, 0] == 2 and qh[0, 1] == int(np.rint(w1 / s_))
     np.testing.assert_allclose(Eh[0], [e0, (w1 - s_ * qh[0, 1]) / 1.0], rtol=1e-15)
-    for bits in (2, 4, 8):
+    for bits in (2, 3, 4, 8):
         qq = rng.integers(0, 1 << bits, (5, 64)).astype(np.uint8)
         np.testing.assert_array_equal(O.unpack_codes(O.pack_codes(qq, bits), 64, bits), qq)
+
+
+def test_unpack_convention_3_bits_bit_stream():
+    """3-bit codes are a bit stream over the row's words: 32 codes fill three words, code 10 starts at bit 30 of word 0 and
+    ends in bit 0 of word 1, code 21 starts at bit 31 of word 1.  Words written out by hand from the codes 0..7 repeating
+    (k mod 8), and a scalar-loop score on them."""
+    codes = [k % 8 for k in range(32)]
+    bits_str = "".join("".join(str((c >> b) & 1) for b in range(3)) for c in codes)       # the stream, first bit first
+    words = [int(bits_str[32 * w:32 * (w + 1)][::-1], 2) for w in range(3)]
+    # by hand: codes 0,1,2,...: word 0 = 0b10_110_101_100_011_010_001_000 ... the low 9 bits are 0b010_001_000 = 0x88
+    assert words[0] & 0x1FF == 0b010001000
+    # code 10 (= 2 = 0b010): bits 30, 31 of word 0 are 0, 1; bit 0 of word 1 is 0
+    assert (words[0] >> 30) & 3 == 0b10 and words[1] & 1 == 0
+    # code 21 (= 5 = 0b101): bit 31 of word 1 is 1, bits 0, 1 of word 2 are 0, 1
+    assert (words[1] >> 31) & 1 == 1 and words[2] & 3 == 0b10
+    q = O.unpack_codes(np.array([words], dtype=np.uint32), 32, 3)
+    assert q.tolist() == [codes]
+    assert O.pack_codes(np.array([codes], dtype=np.uint8), 3).tolist() == [words]
+    x = np.arange(1.0, 33.0)[None, :] / 7.0
+    scale, zero = np.array([[0.25, 0.5]]), np.array([[3.0, 4.0]])
+    z = O.predictor_score(x, np.array([words], dtype=np.uint32), scale, zero, 16, np.array([0.125]), 3)
+    ref = 0.125
+    for g in range(2):
+        inner = 0.0
+        for k in range(16 * g, 16 * g + 16):
+            inner += (codes[k] - zero[0, g]) * x[0, k]
+        ref += scale[0, g] * inner
+    assert abs(z[0, 0] - ref) < 1e-12

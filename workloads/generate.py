@@ -289,13 +289,14 @@ def quantise_gptq(W1: torch.Tensor, xcal: torch.Tensor, group: int, bits: int,
 
 
 def pack_codes(q: torch.Tensor, bits: int = 2) -> torch.Tensor:
-    """[h,d] codes -> [h, d*bits/32] 32-bit words, channel order ascending, lowest
-    bits first.  Returned as int32 holding the uint32 bit pattern."""
+    """[h,d] codes -> [h, d*bits/32] 32-bit words: one bit stream per row, channel order
+    ascending, lowest bits first (a 3-bit code may cross into the next word).  Returned as
+    int32 holding the uint32 bit pattern."""
     h, d = q.shape
-    per = 32 // bits
-    w = q.to(torch.int64).reshape(h, d // per, per)
-    shifts = (torch.arange(per, device=q.device, dtype=torch.int64) * bits)[None, None, :]
-    word = (w << shifts).sum(-1)
+    q64 = q.to(torch.int64)
+    single = (q64[:, :, None] >> torch.arange(bits, device=q.device, dtype=torch.int64)[None, None, :]) & 1
+    stream = single.reshape(h, d * bits // 32, 32)
+    word = (stream << torch.arange(32, device=q.device, dtype=torch.int64)[None, None, :]).sum(-1)
     word = torch.where(word >= 2 ** 31, word - 2 ** 32, word)
     return word.to(torch.int32)
 
