@@ -373,8 +373,18 @@ tardis_status_t tardis_clear_error(tardis_handle_t handle);
 /* For testing what the library does when the device allocator says no, without exhausting a GPU: after this call the next
  * `nth` device allocations of the library (process-wide, any thread) succeed and the one after them fails once, as
  * cudaMalloc would with no memory left; nth < 0 switches the injection off.  The entry point that hits the failure
- * returns TARDIS_ERR_ALLOC and must leave nothing allocated behind.  (The paper has no counterpart of this call.) */
+ * returns TARDIS_ERR_ALLOC and must leave nothing allocated behind.  (The paper has no counterpart of these two calls.) */
 tardis_status_t tardis_debug_fail_alloc(int32_t nth);
+/* How many device allocations of the library are alive in this process, and their bytes (guard areas not counted): what a
+ * test compares before and after a failed call. */
+tardis_status_t tardis_debug_live_allocations(int64_t* count, int64_t* bytes);
+
+/* Every device buffer a handle owns lies between two guard areas of 256 bytes holding a fixed pattern; tardis_stats reads
+ * the guards of the handle's buffers back and returns TARDIS_ERR_CORRUPT (device_error = 2) when one has changed, i.e. when
+ * some kernel wrote past an end of a buffer.  tardis_debug_damage_guard changes (repair = 0) or restores (repair = 1) the
+ * four guard bytes in front of (front = 1) or behind (front = 0) the handle's fp32 accumulator, so that this report can be
+ * tested; the write stays inside the allocation and faults nothing.  (The paper has no counterpart of this call.) */
+tardis_status_t tardis_debug_damage_guard(tardis_handle_t handle, int32_t front, int32_t repair);
 
 /* Frees everything the handle owns (synchronises the device first). */
 tardis_status_t tardis_destroy(tardis_handle_t handle);

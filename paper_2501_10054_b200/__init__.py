@@ -22,7 +22,7 @@ TARDIS_ACT_GELU_TANH, TARDIS_ACT_GELU_ERF, TARDIS_ACT_RELU = 0, 1, 2
 
 EXPORTS = ["tardis_fold", "tardis_ffn_forward", "tardis_ffn_forward_static", "tardis_gemm_bf16", "tardis_stats",
            "tardis_set_debug_capture", "tardis_export_folded", "tardis_set_path", "tardis_set_deterministic", "tardis_stack_forward", "tardis_build_predictor", "tardis_destroy", "tardis_calibrate",
-           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_neuron_thresholds", "tardis_debug_wait_timeout", "tardis_clear_error", "tardis_debug_fail_alloc",
+           "tardis_debug_phase_stamps", "tardis_range_search", "tardis_neuron_thresholds", "tardis_debug_wait_timeout", "tardis_clear_error", "tardis_debug_fail_alloc", "tardis_debug_live_allocations", "tardis_debug_damage_guard",
            "tardis_save", "tardis_load", "tardis_status_string", "tardis_last_error"]
 
 
@@ -85,6 +85,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.tardis_neuron_thresholds.argtypes = [i32, i32, vp, i64, vp, vp, vp, i32, ctypes.c_double, ctypes.c_double, ctypes.c_double, vp, vp, vp]
     lib.tardis_clear_error.argtypes = [vp]
     lib.tardis_debug_fail_alloc.argtypes = [i32]
+    lib.tardis_debug_live_allocations.argtypes = [ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.tardis_debug_damage_guard.argtypes = [vp, i32, i32]
     lib.tardis_save.argtypes = [vp, ctypes.c_char_p]
     lib.tardis_load.argtypes = [ctypes.c_char_p, vp, ctypes.POINTER(vp)]
     for name in EXPORTS[:-2]:
@@ -296,6 +298,18 @@ def tardis_stack_forward(handles, x: torch.Tensor, y: torch.Tensor, gammas=None,
     kb = keep.numel() * keep.element_size() if keep is not None else 0
     _check(load_library().tardis_stack_forward(ctypes.byref(desc), _ptr(x), _ptr(y), _ptr(work), wb, _ptr(keep), kb, n,
                                                _stream(stream)), "tardis_stack_forward")
+
+
+def tardis_debug_damage_guard(handle: int, front: bool, repair: bool):
+    """Changes (or restores) four guard bytes next to the handle's fp32 accumulator; tardis_stats then reports CORRUPT."""
+    _check(load_library().tardis_debug_damage_guard(handle, 1 if front else 0, 1 if repair else 0), "tardis_debug_damage_guard")
+
+
+def tardis_debug_live_allocations():
+    """(count, bytes) of the library's live device allocations in this process."""
+    c, b = ctypes.c_int64(), ctypes.c_int64()
+    _check(load_library().tardis_debug_live_allocations(ctypes.byref(c), ctypes.byref(b)), "tardis_debug_live_allocations")
+    return c.value, b.value
 
 
 def tardis_debug_fail_alloc(nth: int):

@@ -6,6 +6,9 @@
 #include <new>
 
 #include <atomic>
+#include <mutex>
+#include <unordered_map>
+#include <vector>
 #include "common.cuh"
 #include "gemm.cuh"
 
@@ -29,12 +32,67 @@ static Handle* check(tardis_handle_t h) {
 // current would launch there against this handle's pointers.
 static std::atomic<int> g_fail_alloc{-1};   // >= 0: that many allocations still succeed, the next one fails (once)
 
+// Every allocation carries 256 guard bytes of a fixed pattern in front of and behind what the caller gets; tardis_stats
+// looks at the guards of the handle's allocations and reports TARDIS_ERR_CORRUPT when a kernel has written past an end.
+constexpr size_t kGuard = 256;
+constexpr int kGuardByte = 0xA5;
+struct Allocation { char* base; size_t bytes; const void* owner; int device; };
+static std::mutex g_alloc_mutex;
+static std::unordered_map<const void*, Allocation> g_allocs;        // keyed by the pointer handed out
+static thread_local const void* g_alloc_owner = nullptr;            // the handle whose entry point is running on this thread
+struct OwnerScope {
+  explicit OwnerScope(const void* o) { g_alloc_owner = o; }
+  ~OwnerScope() { g_alloc_owner = nullptr; }
+};
+
 cudaError_t dev_malloc_raw(void** p, size_t bytes) {
-  if (g_fail_alloc.load() >= 0 && g_fail_alloc.fetch_sub(1) == 0) {
-    *p = nullptr;
-    return cudaErrorMemoryAllocation;
+  *p = nullptr;
+  if (g_fail_alloc.load() >= 0 && g_fail_alloc.fetch_sub(1) == 0) return cudaErrorMemoryAllocation;
+  char* base = nullptr;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&base), bytes + 2 * kGuard);
+  if (e != cudaSuccess) return e;
+  e = cudaMemset(base, kGuardByte, kGuard);
+  if (e == cudaSuccess) e = cudaMemset(base + kGuard + bytes, kGuardByte, kGuard);
+  if (e != cudaSuccess) { cudaFree(base); return e; }
+  int dev = -1;
+  cudaGetDevice(&dev);
+  {
+    std::lock_guard<std::mutex> lock(g_alloc_mutex);
+    g_allocs[base + kGuard] = Allocation{base, bytes, g_alloc_owner, dev};
   }
-  return cudaMalloc(p, bytes);
+  *p = base + kGuard;
+  return cudaSuccess;
+}
+
+void dev_free(void* p) {
+  if (!p) return;
+  char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_alloc_mutex);
+    auto it = g_allocs.find(p);
+    if (it != g_allocs.end()) { base = it->second.base; g_allocs.erase(it); }
+  }
+  cudaFree(base ? static_cast<void*>(base) : p);
+}
+
+// Number of damaged guards among the allocations of `owner` (both guards of every allocation are read back); -1 on a CUDA error.
+static int damaged_guards(const void* owner) {
+  std::vector<Allocation> mine;
+  {
+    std::lock_guard<std::mutex> lock(g_alloc_mutex);
+    for (const auto& kv : g_allocs)
+      if (kv.second.owner == owner) mine.push_back(kv.second);
+  }
+  int bad = 0;
+  unsigned char buf[2 * kGuard];
+  for (const Allocation& al : mine) {
+    if (cudaMemcpy(buf, al.base, kGuard, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+    if (cudaMemcpy(buf + kGuard, al.base + kGuard + al.bytes, kGuard, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+    bool ok = true;
+    for (size_t i = 0; i < 2 * kGuard; ++i) ok = ok && buf[i] == kGuardByte;
+    bad += ok ? 0 : 1;
+  }
+  return bad;
 }
 
 static bool on_handle_device(const Handle* H) {
@@ -63,7 +121,7 @@ static void free_all(Handle* H) {
   void* ptrs[] = {H->W1, H->W2T, H->C, H->bf, H->lo, H->hi, H->a, H->c, H->b1, H->codes, H->scale,
                   H->zero, H->yacc, H->bitmap, H->counters};
   for (void* p : ptrs)
-    if (p) cudaFree(p);
+    if (p) dev_free(p);
   H->magic = 0;
   delete H;
 }
@@ -74,6 +132,7 @@ static tardis_status_t new_handle(int d, int h, int dtype, int act, int G, int b
   Handle* H = new (std::nothrow) Handle();
   if (!H) return TARDIS_ERR_ALLOC;
   memset(H, 0, sizeof(*H));
+  g_alloc_owner = H;                                   // (the entry point that called this resets it when it returns)
   H->magic = kMagic;
   H->d = d; H->h = h; H->dtype = dtype; H->act = act; H->G = G; H->ngroups = d / G;
   H->bits = bits;
@@ -133,6 +192,7 @@ tardis_status_t tardis_fold(const tardis_fold_desc_t* desc, tardis_stream_t stre
 
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   Handle* H = nullptr;
+  OwnerScope scope(nullptr);                           // new_handle names the owner of the allocations that follow
   tardis_status_t st = new_handle(d, h, desc->dtype, desc->act, G, desc->pred_bits, s, &H);
   if (st != TARDIS_OK) return st;
 
@@ -261,6 +321,9 @@ tardis_status_t tardis_stats(tardis_handle_t handle, tardis_stats_t* out) {
   out->launches = H->launches;
   if (ctr[CTR_ERROR] == 1) return TARDIS_ERR_TIMEOUT;
   if (ctr[CTR_ERROR] != 0) return TARDIS_ERR_CORRUPT;
+  const int bad = damaged_guards(H);
+  if (bad < 0) { set_last_error(cudaGetLastError(), "guard check"); return TARDIS_ERR_CUDA; }
+  if (bad > 0) { out->device_error = 2; return TARDIS_ERR_CORRUPT; }
   return TARDIS_OK;
 }
 
@@ -391,6 +454,7 @@ tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_han
   if (!sane) { fclose(f); return TARDIS_ERR_CORRUPT; }
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   Handle* H = nullptr;
+  OwnerScope scope(nullptr);                           // new_handle names the owner of the allocations that follow
   tardis_status_t st = new_handle(d, h, dtype, act, G, bits, s, &H);
   if (st != TARDIS_OK) { fclose(f); return st; }
   const size_t chunk = size_t(8) << 20;
@@ -422,6 +486,31 @@ tardis_status_t tardis_load(const char* path, tardis_stream_t stream, tardis_han
   if (st == TARDIS_OK && bf16) st = batched_finish(H, nullptr, s);
   if (st != TARDIS_OK) { cudaStreamSynchronize(s); free_all(H); return st; }
   *out = reinterpret_cast<tardis_handle_t>(H);
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_debug_damage_guard(tardis_handle_t handle, int32_t front, int32_t repair) {
+  Handle* H = check(handle);
+  if (!H || !on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
+  TARDIS_CUDA_TRY(cudaStreamSynchronize(H->last_stream));
+  Allocation al{};
+  {
+    std::lock_guard<std::mutex> lock(g_alloc_mutex);
+    auto it = g_allocs.find(H->yacc);
+    if (it == g_allocs.end()) return TARDIS_ERR_INVALID_ARG;
+    al = it->second;
+  }
+  char* at = front ? al.base + kGuard - 4 : al.base + kGuard + al.bytes;   // the four guard bytes next to the buffer
+  TARDIS_CUDA_TRY(cudaMemset(at, repair ? kGuardByte : 0, 4));
+  return TARDIS_OK;
+}
+
+tardis_status_t tardis_debug_live_allocations(int64_t* count, int64_t* bytes) {
+  if (!count || !bytes) return TARDIS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_alloc_mutex);
+  *count = int64_t(g_allocs.size());
+  *bytes = 0;
+  for (const auto& kv : g_allocs) *bytes += int64_t(kv.second.bytes);
   return TARDIS_OK;
 }
 
@@ -467,6 +556,7 @@ tardis_status_t tardis_set_deterministic(tardis_handle_t handle, int32_t on) {
   if (!on_handle_device(H)) return TARDIS_ERR_INVALID_ARG;
   if (on && !H->fscratch && !(H->bstate != nullptr && H->bits <= 4)) return TARDIS_ERR_UNSUPPORTED;
   if (on) {
+    OwnerScope scope(H);
     const tardis_status_t st = fused_set_deterministic(H, true);
     if (st != TARDIS_OK) return st;
   }

@@ -300,7 +300,7 @@ void batched_release(Handle* H) {
   if (!S) return;
   void* ptrs[] = {S->Wf, S->W2, S->What_hi, S->What_lo, S->smaxrow, S->zhat, S->yacc, S->x1, S->delta, S->bitmap, S->rlist, S->rcount};
   for (void* q : ptrs)
-    if (q) cudaFree(q);
+    if (q) dev_free(q);
   delete S;
   H->bstate = nullptr;
 }

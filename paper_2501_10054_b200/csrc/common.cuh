@@ -57,9 +57,11 @@ struct Handle {
 void set_last_error(cudaError_t e, const char* where);
 
 // Every device allocation of the library goes through here: cudaMalloc, or the failure that tardis_debug_fail_alloc
-// has asked for (so that the clean-up after a failed allocation can be tested without exhausting a GPU).
+// has asked for (so that the clean-up after a failed allocation can be tested without exhausting a GPU).  The memory
+// handed out sits between two guard areas that tardis_stats checks.
 cudaError_t dev_malloc_raw(void** p, size_t bytes);
 template <typename T> inline cudaError_t dev_malloc(T** p, size_t bytes) { return dev_malloc_raw(reinterpret_cast<void**>(p), bytes); }
+void dev_free(void* p);   // what dev_malloc gave (null is fine)
 
 #define TARDIS_CUDA_TRY(expr)                                  \
   do {                                                         \

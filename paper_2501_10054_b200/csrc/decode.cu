@@ -988,7 +988,7 @@ void decode_release(Handle* H) {
   if (!S) return;
   void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl, S->rowexp, S->Cp};
   for (void* q : ptrs)
-    if (q) cudaFree(q);
+    if (q) dev_free(q);
   delete S;
   H->dscratch = nullptr;
   H->codes_mma = nullptr;

@@ -1207,7 +1207,7 @@ void fused_release(Handle* H) {
   if (!S) return;
   void* ptrs[] = {S->pblocks, S->plan, S->smax, S->yacc, S->ctl, S->Cp, S->dpart};
   for (void* q : ptrs)
-    if (q) cudaFree(q);
+    if (q) dev_free(q);
   delete S;
   H->fscratch = nullptr;
 }

@@ -147,7 +147,7 @@ tardis_status_t launch_build_predictor(int h, int d, int dtype, const void* W1, 
   double *Wd = nullptr, *Eb = nullptr, *scale64 = nullptr, *zero64 = nullptr;
   uint8_t* q = nullptr;
   auto release = [&]() {
-    cudaFree(Wd); cudaFree(Eb); cudaFree(scale64); cudaFree(zero64); cudaFree(q);
+    dev_free(Wd); dev_free(Eb); dev_free(scale64); dev_free(zero64); dev_free(q);
   };
   cudaError_t e = dev_malloc(&Wd, size_t(h) * d * sizeof(double));
   if (e == cudaSuccess) e = dev_malloc(&Eb, size_t(h) * QB * sizeof(double));

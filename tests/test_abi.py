@@ -77,6 +77,8 @@ def test_invalid_arguments_return_status_before_any_launch(lib):
     assert lib.tardis_stack_forward(None, None, None, None, 0, None, 0, 1, None) == 1
     assert lib.tardis_build_predictor(8, 64, 1, None, None, 2, 64, None, None, None, None) == 1
     assert lib.tardis_debug_fail_alloc(-1) == 0
+    assert lib.tardis_debug_damage_guard(None, 0, 0) == 1
+    assert lib.tardis_debug_live_allocations(None, None) == 1
     assert lib.tardis_neuron_thresholds(4, 4, None, 4, None, None, None, 0, 0.8, 0.7, 0.9, None, None, None) == 1
     # the dense product: an output that is not 16-byte aligned (a view that starts at an odd column) is refused
     assert lib.tardis_gemm_bf16(8, 8, 8, 16, 8, 16, 8, 20, 8, None) == 1

@@ -332,10 +332,7 @@ def test_allocation_failures_return_a_status_and_leak_nothing(dtype, d, h):
     cfg = W.LayerConfig("allocfail", d, h, n_calib=512, dtype=dtype)
     L = _layer(cfg)
     torch.cuda.synchronize()
-    hd = T.fold_layer(L)
-    T.tardis_destroy(hd)                                     # (first use: one-off allocations of the CUDA runtime settle)
-    torch.cuda.synchronize()
-    free0 = torch.cuda.mem_get_info()[0]
+    live0 = T.tardis_debug_live_allocations()               # (other tests' handles are all destroyed: normally (0, 0))
     failed = 0
     try:
         for nth in range(200):
@@ -345,8 +342,7 @@ def test_allocation_failures_return_a_status_and_leak_nothing(dtype, d, h):
             except T.TardisError as e:
                 assert e.status == 3, e.status
                 failed += 1
-                torch.cuda.synchronize()
-                assert torch.cuda.mem_get_info()[0] >= free0, "allocation %d: %d bytes left behind" % (nth, free0 - torch.cuda.mem_get_info()[0])
+                assert T.tardis_debug_live_allocations() == live0, "allocation %d: something left behind" % nth
                 continue
             break                                            # nth is past the last allocation of a fold: it went through
         else:
@@ -367,27 +363,54 @@ def test_allocation_failures_return_a_status_and_leak_nothing(dtype, d, h):
         T.tardis_save(hd, path)
         T.tardis_destroy(hd)
         hd = None
-        torch.cuda.synchronize()
-        free1 = torch.cuda.mem_get_info()[0]
+        assert T.tardis_debug_live_allocations() == live0
         for nth in (0, 3, 9):
             T.tardis_debug_fail_alloc(nth)
             with pytest.raises(T.TardisError) as e:
                 T.tardis_load(path)
             assert e.value.status == 3
-            torch.cuda.synchronize()
-            assert torch.cuda.mem_get_info()[0] >= free1
+            assert T.tardis_debug_live_allocations() == live0
         for nth in range(5):
             T.tardis_debug_fail_alloc(nth)
             with pytest.raises(T.TardisError) as e:
                 T.tardis_build_predictor(L.W1, None, 2, 64)
             assert e.value.status == 3
         T.tardis_debug_fail_alloc(-1)
-        torch.cuda.synchronize()
-        assert torch.cuda.mem_get_info()[0] >= free1
+        assert T.tardis_debug_live_allocations() == live0
     finally:
         T.tardis_debug_fail_alloc(-1)
         if hd:
             T.tardis_destroy(hd)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_guard_areas_report_a_write_past_a_buffer(dtype):
+    """The buffers of a handle lie between guard areas that tardis_stats checks: untouched after real work on every path,
+    reported as TARDIS_ERR_CORRUPT once four guard bytes in front of or behind a buffer have changed (changed here by
+    tardis_debug_damage_guard, inside the allocation), and fine again after they are restored."""
+    cfg = W.LayerConfig("guards", 512, 2048, n_calib=512, dtype=dtype)
+    L = _layer(cfg)
+    h = T.fold_layer(L)
+    try:
+        x = W.make_tokens(cfg, 70, 2).cuda()
+        y = torch.empty_like(x)
+        for n in (1, 4, 9, 70):
+            T.tardis_ffn_forward(h, x[:n], y[:n])
+        for path in (1, 3, 4, 0):
+            T.tardis_set_path(h, path)
+            T.tardis_ffn_forward(h, x[:5], y[:5])
+        assert T.tardis_stats(h)["device_error"] == 0          # (reads every guard back)
+        for front in (True, False):
+            T.tardis_debug_damage_guard(h, front, False)
+            with pytest.raises(T.TardisError) as e:
+                T.tardis_stats(h)
+            assert e.value.status == 6
+            T.tardis_debug_damage_guard(h, front, True)
+            assert T.tardis_stats(h)["device_error"] == 0
+        T.tardis_ffn_forward(h, x[:3], y[:3])
+        assert T.tardis_stats(h)["device_error"] == 0
+    finally:
+        T.tardis_destroy(h)
 
 
 def test_batched_path_chunk_boundary_nan_token_and_empty_ranges():
