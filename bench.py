@@ -464,7 +464,8 @@ def main():
             out.setdefault("notes", []).append("stack graph capture failed: %s" % str(e)[:120])
         out["stack_context"] = {"layers": 32, "batch": 1, "us_per_layer": ms_s * 1e3 / 32,
                                 "us_per_layer_graph": None if ms_g is None else ms_g * 1e3 / 32,
-                                "what": "tardis_stack_forward: per layer k_layernorm, the fused kernel, k_stream_update"}
+                                "what": "tardis_stack_forward: per layer k_update_norm (stream update + layer normalisation) and the fused kernel, "
+                                        "chained by programmatic dependent launch"}
 
         def dense_step():
             for i in range(NT // B):

@@ -3,8 +3,11 @@
 // stream.  The paper has no counterpart of this call (it replaces the FFN block inside an existing model, Section 6);
 // it is the shape in which a decoder hands the FFN blocks of consecutive layers to this library, without attention.
 //
-// Two small kernels live here: the normalisation (one CTA per token, two passes over the row in registers, fp32) and the
-// residual addition.  Everything else is the per-layer forward.
+// Two small kernels live here.  k_update_norm (one CTA per token, the row in registers, fp32) adds the previous layer's
+// output to the stream and normalises the result for the next layer in one pass; k_stream_update adds the last layer's
+// output.  Both take part in the programmatic hand-over between launches: they let the next launch start at once
+// (the fused decode kernel then loads its predictor blocks while the row is being normalised) and wait for the launch
+// before them only where they first touch its results.  Everything else is the per-layer forward.
 #include "common.cuh"
 
 namespace tardis {
@@ -26,19 +29,42 @@ __device__ __forceinline__ float block_sum(float v, float* sh) {
   return t;
 }
 
-// out[t][i] = (x[t][i] - mean_t) / sqrt(var_t + eps) * gamma[i] + beta[i]; mean and variance (1/d, not 1/(d-1)) over the row
+// stream[t][:] takes the previous layer's output f[t][:] (update: added when `residual`, else copied), then
+// out[t][i] = (stream[t][i] - mean_t) / sqrt(var_t + eps) * gamma[i] + beta[i]; mean and variance (1/d, not 1/(d-1)) over the
+// row; without `normalise` out is the stream itself.
 template <typename T>
-__global__ void __launch_bounds__(LN_THREADS) k_layernorm(const T* __restrict__ x, T* __restrict__ out, const float* __restrict__ gamma,
-                                                          const float* __restrict__ beta, int d, float eps) {
+__global__ void __launch_bounds__(LN_THREADS) k_update_norm(T* __restrict__ stream, const T* __restrict__ f, int update, int residual,
+                                                            int normalise, T* __restrict__ out, const float* __restrict__ gamma,
+                                                            const float* __restrict__ beta, int d, float eps) {
   __shared__ float sh[LN_THREADS / 32];
-  const T* row = x + size_t(blockIdx.x) * d;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");          // the launch before wrote f (or the stream)
+  T* row = stream + size_t(blockIdx.x) * d;
+  const T* frow = f + size_t(blockIdx.x) * d;
   float v[LN_MAXPER];
   float s = 0.f;
 #pragma unroll
   for (int e = 0; e < LN_MAXPER; ++e) {
     const int i = threadIdx.x + e * LN_THREADS;
-    v[e] = i < d ? to_f32<T>(row[i]) : 0.f;
+    v[e] = 0.f;
+    if (i < d) {
+      if (update) {
+        const T nv = residual ? from_f32<T>(to_f32<T>(row[i]) + to_f32<T>(frow[i])) : frow[i];   // rounded as it is stored
+        row[i] = nv;
+        v[e] = to_f32<T>(nv);
+      } else {
+        v[e] = to_f32<T>(row[i]);
+      }
+    }
     s += v[e];
+  }
+  if (!normalise) {
+#pragma unroll
+    for (int e = 0; e < LN_MAXPER; ++e) {
+      const int i = threadIdx.x + e * LN_THREADS;
+      if (i < d) out[size_t(blockIdx.x) * d + i] = from_f32<T>(v[e]);
+    }
+    return;
   }
   const float mean = block_sum(s, sh) / float(d);
   float q = 0.f;
@@ -56,11 +82,24 @@ __global__ void __launch_bounds__(LN_THREADS) k_layernorm(const T* __restrict__ 
   }
 }
 
-// stream += f (residual) or stream = f
+// stream += f (residual) or stream = f: after the last layer
 template <typename T>
 __global__ void k_stream_update(T* __restrict__ stream, const T* __restrict__ f, size_t count, int residual) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < count; i += size_t(gridDim.x) * blockDim.x)
     stream[i] = residual ? from_f32<T>(to_f32<T>(stream[i]) + to_f32<T>(f[i])) : f[i];
+}
+
+template <typename... Args>
+cudaError_t launch_chained(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 template <typename T>
@@ -70,27 +109,26 @@ tardis_status_t run_stack(const tardis_stack_desc_t* desc, const void* x, void* 
   const size_t count = size_t(n) * d;
   T* stream = static_cast<T*>(y);
   if (x != y) TARDIS_CUDA_TRY(cudaMemcpyAsync(y, x, count * sizeof(T), cudaMemcpyDeviceToDevice, s));
-  const bool norm = desc->normalise != 0;
+  const int norm = desc->normalise != 0 ? 1 : 0;
+  T* fprev = nullptr;
   for (int l = 0; l < desc->n_layers; ++l) {
-    // with `keep`, the layer's input and output stay where the caller can read them; else two work buffers take turns
+    // with `keep`, the layer's input and output stay where the caller can read them; else two buffers for the inputs take
+    // turns with one for the output (the update of layer l + 1 reads the output of layer l while writing its own input)
     T* xin = keep ? static_cast<T*>(keep) + size_t(2 * l) * count : static_cast<T*>(work);
     T* fout = keep ? static_cast<T*>(keep) + size_t(2 * l + 1) * count : static_cast<T*>(work) + count;
     const T* layer_in = stream;
-    if (norm) {
-      k_layernorm<T><<<unsigned(n), LN_THREADS, 0, s>>>(stream, xin, desc->ln_gamma ? desc->ln_gamma[l] : nullptr,
-                                                       desc->ln_beta ? desc->ln_beta[l] : nullptr, d, desc->ln_eps);
-      TARDIS_CUDA_TRY(cudaGetLastError());
-      layer_in = xin;
-    } else if (keep) {
-      TARDIS_CUDA_TRY(cudaMemcpyAsync(xin, stream, count * sizeof(T), cudaMemcpyDeviceToDevice, s));
+    if (norm || keep || l > 0) {
+      TARDIS_CUDA_TRY(launch_chained(k_update_norm<T>, dim3(unsigned(n)), dim3(LN_THREADS), s, stream, static_cast<const T*>(fprev ? fprev : stream),
+                                     l > 0 ? 1 : 0, desc->residual, norm, xin, norm && desc->ln_gamma ? desc->ln_gamma[l] : static_cast<const float*>(nullptr),
+                                     norm && desc->ln_beta ? desc->ln_beta[l] : static_cast<const float*>(nullptr), d, desc->ln_eps));
       layer_in = xin;
     }
     const tardis_status_t st = tardis_ffn_forward(desc->layers[l], layer_in, fout, n, reinterpret_cast<tardis_stream_t>(s));
     if (st != TARDIS_OK) return st;
-    const unsigned blocks = unsigned((count + 255) / 256 < 4096 ? (count + 255) / 256 : 4096);
-    k_stream_update<T><<<blocks, 256, 0, s>>>(stream, fout, count, desc->residual);
-    TARDIS_CUDA_TRY(cudaGetLastError());
+    fprev = fout;
   }
+  const unsigned blocks = unsigned((count + 255) / 256 < 4096 ? (count + 255) / 256 : 4096);
+  TARDIS_CUDA_TRY(launch_chained(k_stream_update<T>, dim3(blocks), dim3(256), s, stream, static_cast<const T*>(fprev), count, desc->residual));
   return TARDIS_OK;
 }
 
