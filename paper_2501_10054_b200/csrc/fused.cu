@@ -743,7 +743,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   }
   const int nks = d >> 4;                                           // 16-channel steps of a row (= 16-column tiles of an output)
   FZ_STAMP_VALUE(tid == 0, ST_NFL, nun);
-  // -- pre-activations and deltas: steps over the W1 rows, NG steps at a time --
+  // -- pre-activations and deltas: steps over the W1 rows, as many at a time as there are buffers of partial sums (NG at most) --
   {
     // x as the B operand (column g = token g): the warp's k-steps are the same in every step, so their operands are
     // loaded once
