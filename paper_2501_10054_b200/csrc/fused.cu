@@ -254,6 +254,12 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   } else if (lane == 0 && warp < p.nbuf && warp < NQ) {
     issue_unit(warp % NU, warp);
   }
+  // tiles that have to wait for a buffer are asked into L2 meanwhile: their copies then do not queue behind the folded matrix
+  if (!resident && NU > p.nbuf) {
+    const char* base = reinterpret_cast<const char*>(p.pblocks + size_t(plan.x + p.nbuf) * p.unit_bytes);
+    const int lines = ((NU - p.nbuf) * p.unit_bytes + 127) / 128;
+    for (int i = tid; i < lines; i += NTH) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + size_t(i) * 128));
+  }
   const float smax_f = *p.smax;                    // constant state of the layer: fetched before the wait
 
   // From here on the kernel touches what earlier work in the stream may still be writing (x, the
