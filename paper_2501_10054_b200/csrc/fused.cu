@@ -98,7 +98,7 @@ struct Scratch {           // handle-owned device memory of this path
 // the result fixing.
 struct SmemLayout {
   size_t zeros, sx2, tab, fl_j, fl_mask, fl_delta, rc, flagbits, red, bars, misc, xh, wz, wz_end, pbuf, xq, zpart, pred_end, slots_end;
-  int xstride, xq_stride, wz_groups;
+  int xstride, xq_stride, wz_groups, ztok;
   __host__ __device__ SmemLayout(int dpad, int ngroups, int tiles_max, int nbuf, int buf_bytes, int ntok, size_t total_bytes) {
     size_t o = 0;
     auto take = [&](size_t bytes, size_t align) { o = (o + align - 1) / align * align; size_t r = o; o += bytes; return r; };
@@ -118,8 +118,9 @@ struct SmemLayout {
     misc = take(64 * sizeof(int), 8);
     xh = take(size_t(ntok) * xstride * 2, 16);
     pbuf = take(size_t(nbuf) * buf_bytes, 128);
-    xq = take(size_t(2) * 4 * xq_stride, 128);             // limbs of two tokens
-    zpart = take(size_t(tiles_max) * NWP * 2 * 16 * sizeof(float), 16);
+    ztok = ntok < 2 ? ntok : 2;                            // tokens of a predictor pass
+    xq = take(size_t(ztok) * 4 * xq_stride, 128);          // limbs of the tokens of a pass
+    zpart = take(size_t(tiles_max) * NWP * ztok * 16 * sizeof(float), 16);
     pred_end = o;
     // the partial pre-activations of the result fixing sit at the very end: they are not needed while the predictor runs,
     // so they do not compete with its buffers for room.  One buffer per step of MAXGS neurons; as many buffers as fit behind
@@ -525,8 +526,8 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
       // limbs 2,3 (odd t4) weigh 65536 times limbs 0,1; lanes t4 = 0 / 2 store the partial score of token 0 / 1
       auto store_partial = [&](int u, float fa0, float fa1) {
         const float o0 = __shfl_xor_sync(0xffffffffu, fa0, 1), o1 = __shfl_xor_sync(0xffffffffu, fa1, 1);
-        if (!(t4 & 1)) {
-          float* zp = zpart + size_t((u * NWP + warp) * 2 + (t4 >> 1)) * 16;
+        if (!(t4 & 1) && (t4 >> 1) < L.ztok) {
+          float* zp = zpart + size_t((u * NWP + warp) * L.ztok + (t4 >> 1)) * 16;
           zp[g] = fmaf(65536.f, o0, fa0);
           zp[g + 8] = fmaf(65536.f, o1, fa1);
         }
@@ -613,7 +614,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
         const double tau = 1.01 * 3.0 * smax * (double(rs) * unit + 12.0 * 5.9604644775390625e-08 * (double(l1) + double(rs) * unit));
         double s = 0.0;
 #pragma unroll
-        for (int w = 0; w < NWP; ++w) s += double(zpart[size_t((tile * NWP + w) * 2 + tl) * 16 + rr]);
+        for (int w = 0; w < NWP; ++w) s += double(zpart[size_t((tile * NWP + w) * L.ztok + tl) * 16 + rr]);
         const double b1 = double(tab[2 * TR + r]);
         double zhat = b1 + s * (unit * 0.015625);
         const double lo = double(tab[r]), hi = double(tab[TR + r]);
