@@ -550,8 +550,10 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
       };
       if (FAST) {
         // every tile is in shared memory behind one barrier, and a warp has the same one or two pairs in every tile:
-        // their x operands stay in registers
-        const bool two = npairs == 2 * NWP;
+        // their x operands stay in registers; pairs beyond 2 NWP (fewer than NWP of them) go round the warps from tile to tile
+        // (only rows longer than 16 chunks, CT > 8, have such pairs: the loop over them folds away otherwise)
+        const bool two = npairs >= 2 * NWP;
+        const int extra = (CT > 8 && two) ? npairs - 2 * NWP : 0;
         const bool usable = wait_unit(0, 0u);
         uint4 xa0, xa1, xc0 = make_uint4(0u, 0u, 0u, 0u), xc1 = xc0;
         int sa0, sa1, sc0 = 0, sc1 = 0;
@@ -562,6 +564,13 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
           float fa0 = 0.f, fa1 = 0.f, fc0 = 0.f, fc1 = 0.f;
           item(ubase, warp, xa0, xa1, sa0, sa1, fa0, fa1);
           if (two) item(ubase, warp + NWP, xc0, xc1, sc0, sc1, fc0, fc1);
+          for (int e = 0; CT > 8 && e < extra; ++e)
+            if ((u * extra + e) % NWP == warp) {
+              uint4 xb0, xb1;
+              int sxa, sxb;
+              load_x(2 * NWP + e, xb0, xb1, sxa, sxb);
+              item(ubase, 2 * NWP + e, xb0, xb1, sxa, sxb, fc0, fc1);
+            }
           store_partial(u, fa0 + fc0, fa1 + fc1);
         }
         q += NU;
@@ -1086,7 +1095,7 @@ tardis_status_t fused_prepare(Handle* H, cudaStream_t s) {
   for (int a = 0; a < 2 && e == cudaSuccess; ++a)
     for (int b = 0; b < 2 && e == cudaSuccess; ++b)
       e = cudaFuncSetAttribute(S->kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-  S->pairs_fit = (p.nkc * 2 == NWP || p.nkc * 2 == 2 * NWP);
+  S->pairs_fit = (p.nkc * 2 == NWP || (p.nkc * 2 >= 2 * NWP && p.nkc * 2 < 3 * NWP));
   if (e != cudaSuccess) { set_last_error(e, "fused_prepare launch"); return fail(TARDIS_ERR_CUDA); }
 
   p.pblocks = S->pblocks; p.plan = S->plan; p.smax = S->smax; p.yacc = S->yacc; p.ctl = S->ctl;
