@@ -715,7 +715,8 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   const uint32_t rowbytes = uint32_t(d) * 2u;
   uint8_t* const slots = smem + L.pbuf;
   const int nslots = int((L.slots_end - L.pbuf) / size_t(p.slot_stride));
-  const int NG = nslots >= 4 * MAXGS ? 4 : (nslots >= 12 ? 3 : 2);
+  // (two groups: with three or four, more rows are asked for at once and the rows needed first arrive later; measured)
+  const int NG = 2;
   const int GS = min(MAXGS, nslots / NG);
   // fills the group of step st: warp `issuer` arms the barrier and its lanes issue one copy each
   auto fill = [&](int st, int nun, int issuer) {
