@@ -50,7 +50,7 @@ constexpr int MAXTILES = 10;      // predictor tiles (of 16 neurons) per CTA
 constexpr int MAXRC = 64;         // exact re-checks per CTA and pass before the list overflows (rest handled in place)
 constexpr int MAXBUF = 10;        // predictor tile buffers in shared memory
 constexpr int MAXGROUPS = 4;      // slot groups (one barrier each, one buffer of partial sums each) of the result fixing
-constexpr int MAXGS = 8;          // rows per slot group (half an MMA tile: the other half of the operand is zero)
+constexpr int MAXGS = 16;         // rows per slot group (one MMA tile)
 constexpr int NREP = 1;           // replicas of the output accumulator (more replicas spread the reductions, but the last CTA
                                   // reads them all: one measured fastest)
 constexpr int CTMAX = 9;          // 16-column output tiles per warp (d <= 32 * 16 * CTMAX = 4608)
@@ -82,6 +82,7 @@ struct Params {
   int nvec;                // 8-column vectors in a row
   int slot_stride;         // result fixing: bytes between row slots
   int smem_total;          // dynamic shared memory of a CTA
+  int gs_cap;              // result fixing: most neurons of a step (16, or 8 where that keeps one more predictor tile in shared memory)
   int nunits;              // folded-matrix units in all
 };
 
@@ -90,6 +91,7 @@ struct Scratch {           // handle-owned device memory of this path
   Params base; size_t smem_bytes; size_t bytes; int grid; const void* kernels[2][2]; bool pairs_fit;
   float* dpart;            // partial outputs of the deterministic mode (allocated when the mode is first switched on)
   int nbuf_n[MAXT + 1];    // tile buffers in shared memory for a call of n tokens
+  int gs_cap_n[MAXT + 1];  // ... and the most neurons of a step of its result fixing
 };
 
 // ---- shared-memory carve-up (host and device agree through this) -----------------------------------
@@ -99,7 +101,7 @@ struct Scratch {           // handle-owned device memory of this path
 struct SmemLayout {
   size_t zeros, sx2, tab, fl_j, fl_mask, fl_delta, rc, flagbits, red, bars, misc, xh, wz, wz_end, pbuf, xq, zpart, pred_end, slots_end;
   int xstride, xq_stride, wz_groups, ztok;
-  __host__ __device__ SmemLayout(int dpad, int ngroups, int tiles_max, int nbuf, int buf_bytes, int ntok, size_t total_bytes) {
+  __host__ __device__ SmemLayout(int dpad, int ngroups, int tiles_max, int nbuf, int buf_bytes, int ntok, size_t total_bytes, int gs_cap) {
     size_t o = 0;
     auto take = [&](size_t bytes, size_t align) { o = (o + align - 1) / align * align; size_t r = o; o += bytes; return r; };
     const size_t rows = size_t(tiles_max) * 16;
@@ -113,7 +115,7 @@ struct SmemLayout {
     fl_delta = take(rows * MAXT * sizeof(float), 16);
     rc = take(MAXRC * sizeof(int), 4);
     flagbits = take(rows * sizeof(int), 4);
-    red = take(size_t(3) * MAXT * 40 * sizeof(float), 4);  // per token and warp round: max |x|, sum |x|, rounding residual
+    red = take(size_t(2) * ntok * 40 * sizeof(float), 4);  // per token and warp round: sum |x|, rounding residual
     bars = take(size_t(MAXBUF + MAXGROUPS) * sizeof(uint64_t), 8);
     misc = take(64 * sizeof(int), 8);
     xh = take(size_t(ntok) * xstride * 2, 16);
@@ -125,7 +127,7 @@ struct SmemLayout {
     // the partial pre-activations of the result fixing sit at the very end: they are not needed while the predictor runs,
     // so they do not compete with its buffers for room.  One buffer per step of MAXGS neurons; as many buffers as fit behind
     // the predictor's state, MAXGROUPS at most (one at least: wz_end tells the caller whether that one fits)
-    const size_t per = size_t(MAXGS) * ntok * 33 * sizeof(float);
+    const size_t per = size_t(gs_cap) * ntok * 33 * sizeof(float);   // (gs_cap: most neurons of a step, 8 or MAXGS)
     size_t nb = total_bytes > o ? (total_bytes - o) / per : 0;
     nb = nb > size_t(MAXGROUPS) ? size_t(MAXGROUPS) : (nb < 1 ? 1 : nb);
     wz_groups = int(nb);
@@ -160,6 +162,13 @@ __device__ __forceinline__ void ldmatrix_x2(uint32_t& r0, uint32_t& r1, uint32_t
 __device__ __forceinline__ void ldmatrix_x2_trans(uint32_t& r0, uint32_t& r1, uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr) : "memory");
 }
+// four 8 x 8 matrices: lanes 8 m .. 8 m + 7 give the row addresses of matrix m, register m receives it
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
 // Exact fp64 predictor sum of one neuron (row r of a tile) from the tile's predictor blocks in shared memory: the same
 // terms in the same order as exact_score, which reads the original arrays in global memory.  Lane `lane` of `nl` takes
 // the code words lane, lane + nl, ...; the caller adds the lanes up.
@@ -193,7 +202,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 template <int G, int CT, int NTK, bool FAST>
 __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   extern __shared__ __align__(128) uint8_t smem[];
-  const SmemLayout L(p.dpad, p.ngroups, p.tiles_max, p.nbuf, p.buf_bytes, p.n, size_t(p.smem_total));
+  const SmemLayout L(p.dpad, p.ngroups, p.tiles_max, p.nbuf, p.buf_bytes, p.n, size_t(p.smem_total), p.gs_cap);
   uint8_t* pbuf = smem + L.pbuf;
   uint8_t* xq = smem + L.xq;
   float* zpart = reinterpret_cast<float*>(smem + L.zpart);
@@ -244,7 +253,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   }
   if (tid < 64) misc[tid] = 0;
   if (tid >= 64 && tid < 128) reinterpret_cast<uint32_t*>(smem + L.zeros)[tid - 64] = 0u;
-  for (int i = tid; i < 3 * MAXT * 40; i += NTH) red[i] = 0.f;
+  for (int i = tid; i < 2 * n * 40; i += NTH) red[i] = 0.f;
   __syncthreads();
   // predictor blocks first: nothing of them depends on x.  When every tile has its own buffer, all copies report to
   // one barrier; else the buffers form a ring with one barrier each.
@@ -295,7 +304,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
       if (lane == 0) {
         atomicMax(const_cast<int*>(&misc[MS_AMAX + t]), __float_as_int(amax));
         if (any_nf) misc[MS_NONFIN + t] = 1;
-        red[(0 * MAXT + t) * 40 + (v >> 5)] = l1;
+        red[t * 40 + (v >> 5)] = l1;
       }
     }
   }
@@ -386,7 +395,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) resid += __shfl_xor_sync(0xffffffffu, resid, o);
-      if (lane == 0) red[(1 * MAXT + t) * 40 + (v >> 5)] = resid;
+      if (lane == 0) red[(n + t) * 40 + (v >> 5)] = resid;
     }
   };
   build_limbs(0, tid, NTH);
@@ -618,7 +627,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
         const int j = plan.x * 16 + r;
         const int E = token_exp(t);
         float rs = 0.f, l1 = 0.f;
-        for (int w = 0; w < (nv >> 5); ++w) { l1 += red[(0 * MAXT + t) * 40 + w]; rs += red[(1 * MAXT + t) * 40 + w]; }
+        for (int w = 0; w < (nv >> 5); ++w) { l1 += red[t * 40 + w]; rs += red[(n + t) * 40 + w]; }
         const double unit = __longlong_as_double((long long)(1023 + E) << 52);   // 2^E
         const double tau = 1.01 * 3.0 * smax * (double(rs) * unit + 12.0 * 5.9604644775390625e-08 * (double(l1) + double(rs) * unit));
         double s = 0.0;
@@ -717,7 +726,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
   const int nslots = int((L.slots_end - L.pbuf) / size_t(p.slot_stride));
   // (two groups: with three or four, more rows are asked for at once and the rows needed first arrive later; measured)
   const int NG = 2;
-  const int GS = min(MAXGS, nslots / NG);
+  const int GS = min(p.gs_cap, nslots / NG);
   // fills the group of step st: warp `issuer` arms the barrier and its lanes issue one copy each
   auto fill = [&](int st, int nun, int issuer) {
     const int nA = (nun + GS - 1) / GS;                             // steps over W1 rows (as many again over W2^T rows)
@@ -778,7 +787,7 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
         }
       }
     }
-    const int wzstride = MAXGS * n * 33;                            // floats per buffer of partial sums
+    const int wzstride = p.gs_cap * n * 33;                         // floats per buffer of partial sums
     const int NCH = min(NG, L.wz_groups);                           // steps summed up together
     for (int c0 = 0; c0 < nA; c0 += NCH) {
       const int c1 = min(nA, c0 + NCH);
@@ -787,22 +796,27 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
         const bool landed = wait_group(st);
         const uint32_t gbase = smem_u32(slots + size_t((st % NG) * GS) * p.slot_stride);
         float c[4] = {0.f, 0.f, 0.f, 0.f};
-        // only rows 0..7 of the MMA tile are in use: lane l < 16 gives ldmatrix row l & 7, channels + 8 (l >> 3)
-        const uint32_t abase = gbase + uint32_t(min(lane & 7, nw1 - 1)) * p.slot_stride + ((lane >> 3) & 1) * 16 + warp * 32;
+        // A operand = up to 16 W1 rows x 16 channels: lanes 0..7 address rows 0..7, lanes 8..15 rows 8..15 (channels 0..7 of the
+        // step), lanes 16..31 the same rows at channels 8..15; a row the step does not have reads the step's last row instead
+        // (its sums are not used)
+        const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+        const uint32_t abase = gbase + uint32_t(min(a_row, nw1 - 1)) * p.slot_stride + ((lane >> 4) & 1) * 16 + warp * 32;
 #pragma unroll
         for (int e2 = 0; e2 < CT; e2 += 2) {                        // two tiles in flight
-          uint32_t a0[2], a2[2];
+          uint32_t a0[2], a1[2], a2[2], a3[2];
 #pragma unroll
           for (int e = 0; e < 2; ++e)
-            if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) ldmatrix_x2(a0[e], a2[e], abase + (e2 + e) * (NW * 32));
+            if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) ldmatrix_x4(a0[e], a1[e], a2[e], a3[e], abase + (e2 + e) * (NW * 32));
 #pragma unroll
           for (int e = 0; e < 2; ++e)
-            if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) mma_bf16(c, a0[e], 0u, a2[e], 0u, xb0[e2 + e], xb1[e2 + e]);
+            if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) mma_bf16(c, a0[e], a1[e], a2[e], a3[e], xb0[e2 + e], xb1[e2 + e]);
         }
         // the partial sum of (row, token) pair q = n row + token goes to [33 q + warp]: stores and loads without bank conflicts
+        // (c[0], c[1]: row g; c[2], c[3]: row g + 8)
         float* const wzs = wz + size_t(st - c0) * wzstride;
-        if (2 * t4 < n) wzs[(n * g + 2 * t4) * 33 + warp] = c[0];
-        if (2 * t4 + 1 < n) wzs[(n * g + 2 * t4 + 1) * 33 + warp] = c[1];
+        const bool upper = g + 8 < GS;                              // (a buffer holds the sums of GS rows)
+        if (2 * t4 < n) { wzs[(n * g + 2 * t4) * 33 + warp] = c[0]; if (upper) wzs[(n * (g + 8) + 2 * t4) * 33 + warp] = c[2]; }
+        if (2 * t4 + 1 < n) { wzs[(n * g + 2 * t4 + 1) * 33 + warp] = c[1]; if (upper) wzs[(n * (g + 8) + 2 * t4 + 1) * 33 + warp] = c[3]; }
       }
       __syncthreads();                                              // partial sums complete; the rows are used
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -836,30 +850,31 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
 #pragma unroll
   for (int ci = 0; ci < CT; ++ci) acc[ci][0] = acc[ci][1] = acc[ci][2] = acc[ci][3] = 0.f;
   {
-    // W2^T tiles (transposed on load): only neurons 0..7 of the MMA tile are in use: lane l < 16 gives neuron l & 7,
-    // columns + 8 (l >> 3)
-    const int w2_row = lane & 7, w2_cofs = ((lane >> 3) & 1) * 8;
+    // W2^T tiles (transposed on load), up to 16 neurons x 16 output columns: lanes 0..7 address neurons 0..7 at columns 0..7,
+    // lanes 8..15 the same neurons at columns 8..15, lanes 16..31 neurons 8..15 likewise
+    const int w2_row = (lane & 7) + ((lane >> 4) & 1) * 8, w2_cofs = ((lane >> 3) & 1) * 8;
     for (int st = nA; st < 2 * nA; ++st) {
       const int l0 = (st - nA) * GS, nw2 = min(GS, nun - l0);
       const bool landed = wait_group(st);
       const uint32_t gbase = smem_u32(slots + size_t((st % NG) * GS) * p.slot_stride);
-      // B operand: delta of the step's neurons, columns 0..3 the leading bf16 term of tokens 0..3, columns 4..7 the rest
-      float dv[2];
+      // B operand: delta of the step's neurons (k = neuron), columns 0..3 the leading bf16 term of tokens 0..3, columns 4..7 the
+      // rest; b0 holds neurons 2 t4, 2 t4 + 1, b1 neurons 2 t4 + 8, 2 t4 + 9 (a neuron the step does not have counts as 0)
+      float dv[4];
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int kk = 2 * t4 + e;
+      for (int e = 0; e < 4; ++e) {
+        const int kk = 2 * t4 + (e & 1) + (e >> 1) * 8;
         const float v = (kk < nw2 && (g & 3) < n) ? fl_delta[(l0 + kk) * MAXT + (g & 3)] : 0.f;
         const float hi = __bfloat162float(__float2bfloat16_rn(v));
         dv[e] = (g >> 2) ? v - hi : hi;
       }
-      const uint32_t b0 = pack_bf16(dv[0], dv[1]), b1 = 0u;          // (neurons 8..15: none)
+      const uint32_t b0 = pack_bf16(dv[0], dv[1]), b1 = pack_bf16(dv[2], dv[3]);
       const uint32_t abase = gbase + uint32_t(min(w2_row, nw2 - 1)) * p.slot_stride + w2_cofs * 2;
 #pragma unroll
       for (int ci = 0; ci < CT; ++ci) {
         if (warp + ci * NW < nks && landed) {
-          uint32_t a0, a1;
-          ldmatrix_x2_trans(a0, a1, abase + (warp + ci * NW) * 32);
-          mma_bf16(acc[ci], a0, a1, 0u, 0u, b0, b1);
+          uint32_t a0, a1, a2, a3;
+          ldmatrix_x4_trans(a0, a1, a2, a3, abase + (warp + ci * NW) * 32);
+          mma_bf16(acc[ci], a0, a1, a2, a3, b0, b1);
         }
       }
       if (st + NG < 2 * nA) {
@@ -1042,10 +1057,15 @@ tardis_status_t fused_prepare(Handle* H, cudaStream_t s) {
   for (int nt = 1; nt <= MAXT; ++nt) {
     const size_t need_slots = size_t(nt) * dpad * 4 > size_t(4) * p.slot_stride ? size_t(nt) * dpad * 4 : size_t(4) * p.slot_stride;
     S->nbuf_n[nt] = 0;
-    for (int nbuf = tiles_max < MAXBUF ? tiles_max : MAXBUF; nbuf >= 1; --nbuf) {
-      const SmemLayout L(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes, nt, size_t(max_smem));
-      if (L.pred_end <= size_t(max_smem) && L.wz_end <= size_t(max_smem) && L.slots_end - L.pbuf >= need_slots) { S->nbuf_n[nt] = nbuf; break; }
-    }
+    // steps of up to 16 neurons need twice the room for partial sums: they give way where that room buys another tile buffer
+    for (int nbuf = tiles_max < MAXBUF ? tiles_max : MAXBUF; nbuf >= 1 && S->nbuf_n[nt] == 0; --nbuf)
+      for (int cap = MAXGS; cap >= 8; cap -= 8) {
+        const SmemLayout L(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes, nt, size_t(max_smem), cap);
+        if (L.pred_end <= size_t(max_smem) && L.wz_end <= size_t(max_smem) && L.slots_end - L.pbuf >= need_slots) {
+          S->nbuf_n[nt] = nbuf; S->gs_cap_n[nt] = cap;
+          break;
+        }
+      }
     if (S->nbuf_n[nt] == 0) { delete S; return TARDIS_OK; }
   }
   p.tiles_max = tiles_max; p.buf_bytes = p.unit_bytes; S->smem_bytes = size_t(max_smem); p.smem_total = max_smem;
@@ -1161,6 +1181,7 @@ tardis_status_t launch_fused_forward(Handle* H, const void* x, void* y, int n, c
     Params p = S->base;
     p.n = nt;
     p.nbuf = S->nbuf_n[nt];
+    p.gs_cap = S->gs_cap_n[nt];
     p.x = static_cast<const __nv_bfloat16*>(x) + size_t(t0) * H->d;
     p.y = static_cast<__nv_bfloat16*>(y) + size_t(t0) * H->d;
     p.dbg_bitmap = H->dbg_bitmap ? H->dbg_bitmap + size_t(t0) * (H->h / 32) : nullptr;
