@@ -796,27 +796,46 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
         const bool landed = wait_group(st);
         const uint32_t gbase = smem_u32(slots + size_t((st % NG) * GS) * p.slot_stride);
         float c[4] = {0.f, 0.f, 0.f, 0.f};
-        // A operand = up to 16 W1 rows x 16 channels: lanes 0..7 address rows 0..7, lanes 8..15 rows 8..15 (channels 0..7 of the
-        // step), lanes 16..31 the same rows at channels 8..15; a row the step does not have reads the step's last row instead
-        // (its sums are not used)
-        const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
-        const uint32_t abase = gbase + uint32_t(min(a_row, nw1 - 1)) * p.slot_stride + ((lane >> 4) & 1) * 16 + warp * 32;
-#pragma unroll
-        for (int e2 = 0; e2 < CT; e2 += 2) {                        // two tiles in flight
-          uint32_t a0[2], a1[2], a2[2], a3[2];
-#pragma unroll
-          for (int e = 0; e < 2; ++e)
-            if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) ldmatrix_x4(a0[e], a1[e], a2[e], a3[e], abase + (e2 + e) * (NW * 32));
-#pragma unroll
-          for (int e = 0; e < 2; ++e)
-            if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) mma_bf16(c, a0[e], a1[e], a2[e], a3[e], xb0[e2 + e], xb1[e2 + e]);
+        if constexpr (NTK == 1) {
+          // A operand = up to 16 W1 rows x 16 channels: lanes 0..7 address rows 0..7, lanes 8..15 rows 8..15 (channels 0..7 of the
+          // step), lanes 16..31 the same rows at channels 8..15; a row the step does not have reads the step's last row instead
+          // (its sums are not used)
+          const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+          const uint32_t abase = gbase + uint32_t(min(a_row, nw1 - 1)) * p.slot_stride + ((lane >> 4) & 1) * 16 + warp * 32;
+  #pragma unroll
+          for (int e2 = 0; e2 < CT; e2 += 2) {                        // two tiles in flight
+            uint32_t a0[2], a1[2], a2[2], a3[2];
+  #pragma unroll
+            for (int e = 0; e < 2; ++e)
+              if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) ldmatrix_x4(a0[e], a1[e], a2[e], a3[e], abase + (e2 + e) * (NW * 32));
+  #pragma unroll
+            for (int e = 0; e < 2; ++e)
+              if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) mma_bf16(c, a0[e], a1[e], a2[e], a3[e], xb0[e2 + e], xb1[e2 + e]);
+          }
+          // the partial sum of (row, token) pair q = n row + token goes to [33 q + warp]: stores and loads without bank conflicts
+          // (c[0], c[1]: row g; c[2], c[3]: row g + 8)
+          float* const wzs = wz + size_t(st - c0) * wzstride;
+          const bool upper = g + 8 < GS;                              // (a buffer holds the sums of GS rows)
+          if (2 * t4 < n) { wzs[(n * g + 2 * t4) * 33 + warp] = c[0]; if (upper) wzs[(n * (g + 8) + 2 * t4) * 33 + warp] = c[2]; }
+          if (2 * t4 + 1 < n) { wzs[(n * g + 2 * t4 + 1) * 33 + warp] = c[1]; if (upper) wzs[(n * (g + 8) + 2 * t4 + 1) * 33 + warp] = c[3]; }
+        } else {
+          // only rows 0..7 of the MMA tile are in use: lane l < 16 gives ldmatrix row l & 7, channels + 8 (l >> 3)
+          const uint32_t abase = gbase + uint32_t(min(lane & 7, nw1 - 1)) * p.slot_stride + ((lane >> 3) & 1) * 16 + warp * 32;
+  #pragma unroll
+          for (int e2 = 0; e2 < CT; e2 += 2) {                        // two tiles in flight
+            uint32_t a0[2], a2[2];
+  #pragma unroll
+            for (int e = 0; e < 2; ++e)
+              if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) ldmatrix_x2(a0[e], a2[e], abase + (e2 + e) * (NW * 32));
+  #pragma unroll
+            for (int e = 0; e < 2; ++e)
+              if (e2 + e < CT && warp + (e2 + e) * NW < nks && landed) mma_bf16(c, a0[e], 0u, a2[e], 0u, xb0[e2 + e], xb1[e2 + e]);
+          }
+          // the partial sum of (row, token) pair q = n row + token goes to [33 q + warp]: stores and loads without bank conflicts
+          float* const wzs = wz + size_t(st - c0) * wzstride;
+          if (2 * t4 < n) wzs[(n * g + 2 * t4) * 33 + warp] = c[0];
+          if (2 * t4 + 1 < n) wzs[(n * g + 2 * t4 + 1) * 33 + warp] = c[1];
         }
-        // the partial sum of (row, token) pair q = n row + token goes to [33 q + warp]: stores and loads without bank conflicts
-        // (c[0], c[1]: row g; c[2], c[3]: row g + 8)
-        float* const wzs = wz + size_t(st - c0) * wzstride;
-        const bool upper = g + 8 < GS;                              // (a buffer holds the sums of GS rows)
-        if (2 * t4 < n) { wzs[(n * g + 2 * t4) * 33 + warp] = c[0]; if (upper) wzs[(n * (g + 8) + 2 * t4) * 33 + warp] = c[2]; }
-        if (2 * t4 + 1 < n) { wzs[(n * g + 2 * t4 + 1) * 33 + warp] = c[1]; if (upper) wzs[(n * (g + 8) + 2 * t4 + 1) * 33 + warp] = c[3]; }
       }
       __syncthreads();                                              // partial sums complete; the rows are used
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -850,9 +869,12 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
 #pragma unroll
   for (int ci = 0; ci < CT; ++ci) acc[ci][0] = acc[ci][1] = acc[ci][2] = acc[ci][3] = 0.f;
   {
-    // W2^T tiles (transposed on load), up to 16 neurons x 16 output columns: lanes 0..7 address neurons 0..7 at columns 0..7,
-    // lanes 8..15 the same neurons at columns 8..15, lanes 16..31 neurons 8..15 likewise
-    const int w2_row = (lane & 7) + ((lane >> 4) & 1) * 8, w2_cofs = ((lane >> 3) & 1) * 8;
+    // W2^T tiles (transposed on load), 16 output columns x the neurons of the step.  Calls of one token (steps of up to 16
+    // neurons): lanes 0..7 address neurons 0..7 at columns 0..7, lanes 8..15 the same neurons at columns 8..15, lanes 16..31
+    // neurons 8..15 likewise.  Calls of several tokens (steps of up to 8 neurons): lanes 0..15 only, the other half of the
+    // operand is zero.
+    constexpr bool WIDE = NTK == 1;
+    const int w2_row = (lane & 7) + (WIDE ? ((lane >> 4) & 1) * 8 : 0), w2_cofs = ((lane >> 3) & 1) * 8;
     for (int st = nA; st < 2 * nA; ++st) {
       const int l0 = (st - nA) * GS, nw2 = min(GS, nun - l0);
       const bool landed = wait_group(st);
@@ -863,17 +885,18 @@ __global__ void __launch_bounds__(NTH, 1) k_fused(const Params p) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int kk = 2 * t4 + (e & 1) + (e >> 1) * 8;
-        const float v = (kk < nw2 && (g & 3) < n) ? fl_delta[(l0 + kk) * MAXT + (g & 3)] : 0.f;
+        const float v = ((WIDE || e < 2) && kk < nw2 && (g & 3) < n) ? fl_delta[(l0 + kk) * MAXT + (g & 3)] : 0.f;
         const float hi = __bfloat162float(__float2bfloat16_rn(v));
         dv[e] = (g >> 2) ? v - hi : hi;
       }
-      const uint32_t b0 = pack_bf16(dv[0], dv[1]), b1 = pack_bf16(dv[2], dv[3]);
+      const uint32_t b0 = pack_bf16(dv[0], dv[1]), b1 = WIDE ? pack_bf16(dv[2], dv[3]) : 0u;
       const uint32_t abase = gbase + uint32_t(min(w2_row, nw2 - 1)) * p.slot_stride + w2_cofs * 2;
 #pragma unroll
       for (int ci = 0; ci < CT; ++ci) {
         if (warp + ci * NW < nks && landed) {
-          uint32_t a0, a1, a2, a3;
-          ldmatrix_x4_trans(a0, a1, a2, a3, abase + (warp + ci * NW) * 32);
+          uint32_t a0, a1, a2 = 0u, a3 = 0u;
+          if constexpr (WIDE) ldmatrix_x4_trans(a0, a1, a2, a3, abase + (warp + ci * NW) * 32);
+          else ldmatrix_x2_trans(a0, a1, abase + (warp + ci * NW) * 32);
           mma_bf16(acc[ci], a0, a1, a2, a3, b0, b1);
         }
       }
@@ -1059,7 +1082,7 @@ tardis_status_t fused_prepare(Handle* H, cudaStream_t s) {
     S->nbuf_n[nt] = 0;
     // steps of up to 16 neurons need twice the room for partial sums: they give way where that room buys another tile buffer
     for (int nbuf = tiles_max < MAXBUF ? tiles_max : MAXBUF; nbuf >= 1 && S->nbuf_n[nt] == 0; --nbuf)
-      for (int cap = MAXGS; cap >= 8; cap -= 8) {
+      for (int cap = nt == 1 ? MAXGS : 8; cap >= 8; cap -= 8) {   // (calls of several tokens: 8, measured)
         const SmemLayout L(dpad, p.ngroups, tiles_max, nbuf, p.unit_bytes, nt, size_t(max_smem), cap);
         if (L.pred_end <= size_t(max_smem) && L.wz_end <= size_t(max_smem) && L.slots_end - L.pbuf >= need_slots) {
           S->nbuf_n[nt] = nbuf; S->gs_cap_n[nt] = cap;
