@@ -320,7 +320,7 @@ def main():
     dur_s = ms * 1e-3 / calls_per_step
     achieved = alg / dur_s / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": peak_src, "kernel": "k_fused" if B <= 12 else "k_gemm (batched path)",
+                "traffic": None, "peak_source": peak_src, "kernel": "k_fused" if B <= 16 else "k_gemm (batched path)",
                 "algorithmic_bytes_per_launch": alg, "avg_launch_us": dur_s * 1e6,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
     # DRAM bytes per launch from the committed ncu summary of this kernel (null when there is none)
@@ -378,7 +378,7 @@ def main():
                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                                  "frac_of_nominal_8TBs": gbs / 8000.0}}
 
-        # the same layers at other batch sizes (one launch of the fused kernel up to 4 tokens, several up to 12, the
+        # the same layers at other batch sizes (one launch of the fused kernel up to 4 tokens, several up to 16, the
         # tensor-core path beyond)
         for bsz in (4, 16, 64):
             if NT % bsz == 0 and B != bsz:

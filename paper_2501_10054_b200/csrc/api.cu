@@ -225,7 +225,7 @@ tardis_status_t tardis_ffn_forward(tardis_handle_t handle, const void* x, void* 
   tardis_status_t st;
   // (deterministic mode: only the kernels of fused.cu and the tensor-core products without a split channel range qualify)
   const bool has_fused = H->fscratch != nullptr || (H->codes_mma != nullptr && !H->deterministic);
-  const bool fused = has_fused && ((H->path_override == 0 && n_tokens <= (H->fscratch ? kDecodeMaxTokens : 8)) || (H->path_override == 2 && n_tokens <= 4096));
+  const bool fused = has_fused && ((H->path_override == 0 && n_tokens <= (H->fscratch ? H->fused_max_tokens : 8)) || (H->path_override == 2 && n_tokens <= 4096));
   // (8-bit codes times a bf16 scale do not fit the exact two-term bf16 form the batched scores rely on)
   const bool batched = ((H->path_override == 0 && !fused) || H->path_override == 3) && H->bstate != nullptr && H->bits <= 4;
   if (H->deterministic && !fused && !batched) return TARDIS_ERR_UNSUPPORTED;

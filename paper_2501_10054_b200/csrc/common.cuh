@@ -10,7 +10,8 @@ namespace tardis {
 
 constexpr uint64_t kMagic = 0x7A2D15F01DULL;
 constexpr int kGenericChunk = 256;   // tokens per pass of the generic kernels (scratch is sized for this)
-constexpr int kDecodeMaxTokens = 12; // largest batch the fused decode kernels take (the newer one 4 tokens per launch)
+constexpr int kDecodeMaxTokens = 16; // largest batch the fused decode kernel takes (4 tokens per launch) on layers of up to 4096
+                                     // channels; 13 on wider ones (measured against the batched path, see fused_max_tokens)
 constexpr int kStaticMaxTokens = 64; // largest batch of the forward that keeps its scratch in the library image
 
 // device counter slots
@@ -39,6 +40,7 @@ struct Handle {
   uint32_t* bitmap;      // [kGenericChunk, h/32]
   unsigned long long* counters;  // [CTR_COUNT]
   void* fscratch;        // fused decode state for calls of 1..4 tokens per launch (see fused.cu); null when not built
+  int fused_max_tokens;  // calls of up to this many tokens go to that kernel when the path is chosen automatically
   void* dscratch;        // fused decode scratch (see decode.cu)
   size_t dscratch_bytes;
   void* bstate;          // batched / prefill state and scratch (see batched.cu); null when not built

@@ -233,7 +233,7 @@ def test_deterministic_mode_same_bits_run_to_run(d, h, G):
                 T.tardis_ffn_forward(other, x, yo)            # unrelated work between the repetitions
             for y in outs[1:]:
                 assert torch.equal(y.view(torch.int16), outs[0].view(torch.int16)), "n = %d" % n
-            assert T.tardis_stats(hd)["last_path"] == (2 if n <= 12 else 3)
+            assert T.tardis_stats(hd)["last_path"] == (2 if n <= 16 else 3)
             yg, F, S = Hp.gpu_forward(hd, L, x, [n])
             assert torch.equal(yg.view(torch.int16), outs[0].view(torch.int16))
             keep = np.arange(n)[: 6]
