@@ -44,13 +44,31 @@ __device__ inline double exact_score(const uint32_t* __restrict__ codes, const _
   const uint32_t cmask = (1u << bits) - 1u;
   const int nwords = d / per, ng = d / G;
   double acc = 0.0;
-  for (int w = lane; w < nwords; w += 32) {
-    const uint32_t word = codes[size_t(j) * nwords + w];
-    const int g = (w * per) / G;
-    const double zp = double(zero[size_t(j) * ng + g]);
-    double inner = 0.0;
-    for (int q = 0; q < per; ++q) inner += (double((word >> (bits * q)) & cmask) - zp) * double(__bfloat162float(xt[w * per + q]));
-    acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
+  if (bits == 2 && (reinterpret_cast<uintptr_t>(xt) & 15u) == 0) {
+    // the 16 channels of a word come in as two 128-bit loads (same terms in the same order as the general loop below)
+    for (int w = lane; w < nwords; w += 32) {
+      const uint32_t word = codes[size_t(j) * nwords + w];
+      const int g = (w * 16) / G;
+      const double zp = double(zero[size_t(j) * ng + g]);
+      const uint4 xa = *reinterpret_cast<const uint4*>(xt + w * 16), xb = *reinterpret_cast<const uint4*>(xt + w * 16 + 8);
+      const uint32_t xw[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+      double inner = 0.0;
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        const float xf = __uint_as_float((q & 1) ? (xw[q >> 1] & 0xffff0000u) : (xw[q >> 1] << 16));
+        inner += (double((word >> (2 * q)) & 3u) - zp) * double(xf);
+      }
+      acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
+    }
+  } else {
+    for (int w = lane; w < nwords; w += 32) {
+      const uint32_t word = codes[size_t(j) * nwords + w];
+      const int g = (w * per) / G;
+      const double zp = double(zero[size_t(j) * ng + g]);
+      double inner = 0.0;
+      for (int q = 0; q < per; ++q) inner += (double((word >> (bits * q)) & cmask) - zp) * double(__bfloat162float(xt[w * per + q]));
+      acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
