@@ -45,20 +45,39 @@ __device__ inline double exact_score(const uint32_t* __restrict__ codes, const _
   const int nwords = d / per, ng = d / G;
   double acc = 0.0;
   if (bits == 2 && (reinterpret_cast<uintptr_t>(xt) & 15u) == 0) {
-    // the 16 channels of a word come in as two 128-bit loads (same terms in the same order as the general loop below)
-    for (int w = lane; w < nwords; w += 32) {
-      const uint32_t word = codes[size_t(j) * nwords + w];
-      const int g = (w * 16) / G;
-      const double zp = double(zero[size_t(j) * ng + g]);
-      const uint4 xa = *reinterpret_cast<const uint4*>(xt + w * 16), xb = *reinterpret_cast<const uint4*>(xt + w * 16 + 8);
-      const uint32_t xw[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-      double inner = 0.0;
+    // the 16 channels of a word come in as two 128-bit loads, and the loads of four words go out before the first is used
+    // (same terms in the same order as the general loop below)
+    for (int w0 = lane; w0 < nwords; w0 += 128) {
+      uint32_t word[4];
+      uint8_t zr[4];
+      __nv_bfloat16 sr[4];
+      uint4 xa[4], xb[4];
 #pragma unroll
-      for (int q = 0; q < 16; ++q) {
-        const float xf = __uint_as_float((q & 1) ? (xw[q >> 1] & 0xffff0000u) : (xw[q >> 1] << 16));
-        inner += (double((word >> (2 * q)) & 3u) - zp) * double(xf);
+      for (int u = 0; u < 4; ++u) {
+        const int w = w0 + 32 * u;
+        if (w < nwords) {
+          const int g = (w * 16) / G;
+          word[u] = codes[size_t(j) * nwords + w];
+          zr[u] = zero[size_t(j) * ng + g];
+          sr[u] = scale[size_t(j) * ng + g];
+          xa[u] = *reinterpret_cast<const uint4*>(xt + w * 16);
+          xb[u] = *reinterpret_cast<const uint4*>(xt + w * 16 + 8);
+        }
       }
-      acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (w0 + 32 * u < nwords) {
+          const double zp = double(zr[u]);
+          const uint32_t xw[8] = {xa[u].x, xa[u].y, xa[u].z, xa[u].w, xb[u].x, xb[u].y, xb[u].z, xb[u].w};
+          double inner = 0.0;
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            const float xf = __uint_as_float((q & 1) ? (xw[q >> 1] & 0xffff0000u) : (xw[q >> 1] << 16));
+            inner += (double((word[u] >> (2 * q)) & 3u) - zp) * double(xf);
+          }
+          acc += double(__bfloat162float(sr[u])) * inner;
+        }
+      }
     }
   } else {
     for (int w = lane; w < nwords; w += 32) {
