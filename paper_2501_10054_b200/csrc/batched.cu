@@ -113,7 +113,7 @@ __global__ void k_recheck(const uint2* __restrict__ rlist, const unsigned int* _
   for (unsigned int e = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; e < total; e += nwarps) {
     const uint2 pr = rlist[e];
     const int t = int(pr.x), j = int(pr.y);
-    const double z = exact_score(codes, scale, zero, x + size_t(t) * d, j, d, G, bits, lane) + double(b1[j]);
+    const double z = exact_score_wide(codes, scale, zero, x + size_t(t) * d, j, d, G, bits, lane) + double(b1[j]);
     if (lane == 0) {
       const bool inside = (double(lo[j]) <= z) && (z < double(hi[j]));
       uint32_t* wp = bitmap + size_t(t) * (h / 32) + (j >> 5);

@@ -44,7 +44,29 @@ __device__ inline double exact_score(const uint32_t* __restrict__ codes, const _
   const uint32_t cmask = (1u << bits) - 1u;
   const int nwords = d / per, ng = d / G;
   double acc = 0.0;
-  if (bits == 2 && (reinterpret_cast<uintptr_t>(xt) & 15u) == 0) {
+  for (int w = lane; w < nwords; w += 32) {
+    const uint32_t word = codes[size_t(j) * nwords + w];
+    const int g = (w * per) / G;
+    const double zp = double(zero[size_t(j) * ng + g]);
+    double inner = 0.0;
+    for (int q = 0; q < per; ++q) inner += (double((word >> (bits * q)) & cmask) - zp) * double(__bfloat162float(xt[w * per + q]));
+    acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  return acc;
+}
+
+// The same sums for a kernel that does nothing else (k_recheck): with 2-bit codes the 16 channels of a word come in as two
+// 128-bit loads and the loads of four words go out before the first is used; same terms in the same order as exact_score.
+// (Kept apart from exact_score: inside the fused kernels its registers would spill.)
+__device__ inline double exact_score_wide(const uint32_t* __restrict__ codes, const __nv_bfloat16* __restrict__ scale,
+                                          const uint8_t* __restrict__ zero, const __nv_bfloat16* __restrict__ xt, int j, int d, int G,
+                                          int bits, int lane) {
+  if (bits != 2 || (reinterpret_cast<uintptr_t>(xt) & 15u) != 0) return exact_score(codes, scale, zero, xt, j, d, G, bits, lane);
+  const int nwords = d / 16, ng = d / G;
+  double acc = 0.0;
+  {
     // the 16 channels of a word come in as two 128-bit loads, and the loads of four words go out before the first is used
     // (same terms in the same order as the general loop below)
     for (int w0 = lane; w0 < nwords; w0 += 128) {
@@ -78,15 +100,6 @@ __device__ inline double exact_score(const uint32_t* __restrict__ codes, const _
           acc += double(__bfloat162float(sr[u])) * inner;
         }
       }
-    }
-  } else {
-    for (int w = lane; w < nwords; w += 32) {
-      const uint32_t word = codes[size_t(j) * nwords + w];
-      const int g = (w * per) / G;
-      const double zp = double(zero[size_t(j) * ng + g]);
-      double inner = 0.0;
-      for (int q = 0; q < per; ++q) inner += (double((word >> (bits * q)) & cmask) - zp) * double(__bfloat162float(xt[w * per + q]));
-      acc += double(__bfloat162float(scale[size_t(j) * ng + g])) * inner;
     }
   }
 #pragma unroll
