@@ -251,6 +251,30 @@ def test_neuron_thresholds_match_oracle(h, n, act):
         T.tardis_neuron_thresholds(same, None, err, err, 0, 0.5, 0.6, 0.9)      # t_layer below t_min
 
 
+def test_offline_pipeline_thresholds_feed_the_range_search():
+    """The offline steps of Section 5.1.1 chained on the GPU: a range search at the layer threshold, the neuron-level
+    thresholds from the errors of those ranges, a second search with one threshold per neuron.  Properties that must hold
+    whatever the data: every neuron's final range covers at least its own threshold of its samples (or all of them), a
+    neuron whose threshold went up does not get a narrower range, and the thresholds average to the layer's."""
+    h, n, act = 512, 1024, W.ACT_GELU_TANH
+    g = torch.Generator().manual_seed(77)
+    z = (torch.randn(h, n, generator=g) * torch.linspace(0.4, 2.5, h)[:, None] + torch.linspace(-0.5, 0.5, h)[:, None]).cuda()
+    lo0, hi0, _, _ = T.tardis_range_search(z, None, 0.85, 0.05, act)
+    err, thr = T.tardis_neuron_thresholds(z, None, lo0, hi0, act, 0.85, 0.75, 0.95)
+    lo1, hi1, a1, c1 = T.tardis_range_search(z, None, thr, 0.05, act)
+    torch.cuda.synchronize()
+    inside = ((z >= lo1[:, None]) & (z < hi1[:, None])).float().mean(dim=1)
+    assert bool((inside >= thr - 1e-6).all())
+    assert abs(float(thr.mean()) - 0.85) < 1e-5
+    up = thr > 0.85 + 1e-6
+    assert bool(((hi1 - lo1)[up] >= (hi0 - lo0)[up] - 1e-6).all())
+    down = thr < 0.85 - 1e-6
+    assert bool(((hi1 - lo1)[down] <= (hi0 - lo0)[down] + 1e-6).all())
+    # the neurons with the smallest errors are the ones that were given the widest coverage
+    order = torch.argsort(err, stable=True)
+    assert bool((thr[order[:h // 4]] >= thr[order[-h // 4:]].max() - 1e-6).all())
+
+
 # ---- the predictor built on the GPU (tardis_build_predictor) ----
 def _upper_factor(X, damp=0.01):
     """Upper Cholesky factor of the inverse of H = (2/N) X^T X + damp mean(diag H) I, by numpy's routines in float64."""
