@@ -457,11 +457,12 @@ def main():
         def stack_step():
             T.tardis_stack_forward(chain, xs1, ys1, None, None, 1e-5, True, True, work=wk)
         ms_s = timed(stack_step, max(3, args.steps // 2), 3)
-        try:
-            ms_g = timed(stack_step, max(3, args.steps // 2), 3, graph=True)
-        except Exception as e:      # capture refused: reported, not fatal
-            ms_g = None
-            out.setdefault("notes", []).append("stack graph capture failed: %s" % str(e)[:120])
+        ms_g = None
+        if world == 1:              # (a capture that fails on one rank only would leave the others in a barrier)
+            try:
+                ms_g = timed(stack_step, max(3, args.steps // 2), 3, graph=True)
+            except Exception as e:  # capture refused: reported, not fatal
+                out.setdefault("notes", []).append("stack graph capture failed: %s" % str(e)[:120])
         out["stack_context"] = {"layers": 32, "batch": 1, "us_per_layer": ms_s * 1e3 / 32,
                                 "us_per_layer_graph": None if ms_g is None else ms_g * 1e3 / 32,
                                 "what": "tardis_stack_forward: per layer k_update_norm (stream update + layer normalisation) and the fused kernel, "
